@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the isomorphic neighbourhood all-to-all on one B200 (or N independent
+replicas, one per GPU).
+
+A step is one `Iso_Start` of the whole schedule on the workload (default: all-to-all on a
+32x32x32 torus, Moore neighbourhood of radius 1, 64-byte fp32 blocks).  The headline value
+is the effective bandwidth over the bytes the message-combining schedule actually moves
+(read + written), device timed with CUDA events; the same line carries the payload rate,
+the one-pass direct kernel for comparison, the roofline fraction, the end-to-end rate with
+host buffers and the CPU oracle timed on the host cores.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--sweep]
+    python bench.py --impl reference ...      # times the CPU oracle instead
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "neighbor-alltoall effective GB/s (device-timed) and % of B200 HBM peak, combining vs direct"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+L2_FLUSH_BYTES = 512 << 20
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while running."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.2] or [r for _, r in self.rows]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower() == "active":
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def tukey_median(xs):
+    """Median after removing outliers beyond 3 x IQR (the paper's protocol, Section IV)."""
+    xs = sorted(xs)
+    if len(xs) < 4:
+        return statistics.median(xs)
+    q1, q3 = np.percentile(xs, [25, 75])
+    lo, hi = q1 - 3 * (q3 - q1), q3 + 3 * (q3 - q1)
+    kept = [x for x in xs if lo <= x <= hi]
+    return statistics.median(kept or xs)
+
+
+def init_distributed(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        import torch
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        dist_mod.init_process_group(backend=backend, rank=rank, world_size=world)
+        dist = dist_mod
+    return rank, world, local, dist
+
+
+# ------------------------------------------------------------------------ reference arm
+def oracle_run(w, send):
+    """One pass of the CPU oracle over the whole workload (only the CPU-baseline leg and the
+    reference arm call this)."""
+    import oracle
+    from paper_1606_07676_b200 import workloads as wl
+    lens, sd, rd, ss, rs = wl.layout(w)
+    if w.collective == "alltoall":
+        return oracle.alltoall(w.dims, w.offsets, w.block_bytes, send)
+    if w.collective == "allgather":
+        return oracle.allgather(w.dims, w.offsets, w.block_bytes, send)
+    return oracle.alltoallv(w.dims, w.offsets, lens, sd, rd, ss, rs, send)
+
+
+def run_reference(args):
+    """Times the CPU oracle, as it stands, on the same workload and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_1606_07676_b200 import workloads as wl
+
+    w = wl.config(args.workload)
+    lens, sd, rd, ss, rs = wl.layout(w)
+    send = wl.send_buffer_np(w, ss)
+    bytes_min = 2 * w.P * int(lens.sum())
+    for _ in range(max(1, args.warmup)):
+        oracle_run(w, send)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_run(w, send)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = bytes_min / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.workload, "P": w.P, "s": w.s, "note": "CPU oracle (direct definition), "
+                   "one host thread, whole workload per step; bytes = one read + one write of every block"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                         "sample": "the whole workload, %d steps" % args.steps},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------ our arm
+class Bound:
+    """A workload bound to device buffers through the C-ABI binding."""
+
+    def __init__(self, torch, iso, wl, name, seed=None):
+        self.torch, self.iso = torch, iso
+        self.w = wl.config(name) if seed is None else wl.config(name, seed)
+        w = self.w
+        self.lens, self.sd, self.rd, self.ss, self.rs = wl.layout(w)
+        self.send = wl.payload_torch(w.kind, w.seed, 0, w.P * self.ss, "cuda")
+        self.recv = torch.empty(w.P * self.rs, dtype=torch.uint8, device="cuda")
+        self.comm = iso.Iso_neighborhood_create(w.dims, w.offsets)
+        if w.collective == "alltoall":
+            self.req = iso.Iso_neighbor_alltoall_init(self.send, w.block_bytes, 1, self.recv, w.block_bytes, 1, self.comm)
+        elif w.collective == "allgather":
+            self.req = iso.Iso_neighbor_allgather_init(self.send, w.block_bytes, 1, self.recv, w.block_bytes, 1, self.comm)
+        else:
+            self.req = iso.Iso_neighbor_alltoallv_init(self.send, self.lens, self.sd, 1, self.recv, self.lens, self.rd, 1, self.comm)
+
+    def set(self, alg, fusion):
+        self.iso.Iso_request_set_algorithm(self.req, alg, fusion)
+        self.iso.Iso_Start(self.req, self.torch.cuda.current_stream())    # materialise outside the timed region
+        self.iso.Iso_wait(self.req)
+        return self.iso.Iso_request_get_stats(self.req)
+
+    def close(self):
+        self.iso.Iso_request_free(self.req)
+        self.iso.Iso_comm_free(self.comm)
+
+
+def time_steps(torch, fn, steps, warmup, flush):
+    """Per-step device times (ms) of `fn`, CUDA events on the current stream; between steps
+    the L2 is flushed by overwriting a buffer larger than it (outside the timed spans)."""
+    for _ in range(warmup):
+        if flush is not None:
+            flush.add_(1)
+        fn()
+    torch.cuda.synchronize()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    for k in range(steps):
+        if flush is not None:
+            flush.add_(1)
+        starts[k].record()
+        fn()
+        ends[k].record()
+    torch.cuda.synchronize()
+    return [s.elapsed_time(e) for s, e in zip(starts, ends)]
+
+
+def cpu_baseline(w, seconds=10.0):
+    """The oracle, as it stands, on this host: repeated runs of the whole workload for a
+    bounded time; returns GB/s over one read + one write of every delivered block."""
+    from paper_1606_07676_b200 import workloads as wl
+    lens, sd, rd, ss, rs = wl.layout(w)
+    send = wl.send_buffer_np(w, ss)
+    bytes_min = 2 * w.P * int(lens.sum())
+    oracle_run(w, send)
+    times = []
+    t_end = time.perf_counter() + seconds
+    while len(times) < 3 or (time.perf_counter() < t_end and len(times) < 50):
+        t0 = time.perf_counter()
+        oracle_run(w, send)
+        times.append(time.perf_counter() - t0)
+    dt = statistics.median(times)
+    return {"value": bytes_min / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": "the whole workload (%d processes x %d blocks), median of %d runs" % (w.P, w.s, len(times)),
+            "ms": dt * 1e3}
+
+
+def run_ours(args):
+    import torch
+    rank, world, local, dist = init_distributed(args.gpus)
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    from paper_1606_07676_b200 import binding as iso
+    from paper_1606_07676_b200 import workloads as wl
+    iso.load_library()
+
+    peak, peak_kind = measured_peak()
+    flush = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device="cuda")
+    b = Bound(torch, iso, wl, args.workload)
+    stream = torch.cuda.current_stream()
+
+    def start():
+        iso.Iso_Start(b.req, stream)
+
+    # ---- headline: message-combining schedule, one launch per dimension ----------------
+    st = b.set(iso.ISO_ALG_COMBINING, args.fusion)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local) if rank == 0 else None
+    t0 = time.time()
+    times = time_steps(torch, start, args.steps, args.warmup, flush)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    ms = sum(times) / len(times)
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    moved, minimum = st["bytes_moved"], st["bytes_min"]
+    value = world * moved / (ms * 1e-3) / 1e9
+    per_gpu = moved / (ms * 1e-3) / 1e9
+
+    detail = {"combining": {"fusion_level": args.fusion, "rounds": st["rounds"], "launches": st["launches"],
+                            "bytes_moved": moved, "bytes_min": minimum, "ms_cold": ms,
+                            "ms_cold_median": tukey_median(times), "gbs_moved": per_gpu,
+                            "gbs_payload": minimum / (ms * 1e-3) / 1e9}}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.workload, "collective": b.w.collective, "dims": list(b.w.dims), "s": b.w.s,
+                   "P": b.w.P, "block_bytes": b.w.block_bytes or None, "schedule": "combining (Section V), fusion level %d" % args.fusion,
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "flushed between steps (512 MiB overwrite, outside the timed spans)",
+                   "bytes": "value = bytes read + written by the schedule / device time"},
+        "gpu_launches": st["launches"] * args.steps,
+        "frac_of_nominal_8TBs": per_gpu / NOMINAL_HBM_GBS,
+    }
+
+    if rank == 0 and world == 1:
+        # warm (back to back, no flush) timing of the same schedule
+        warm = time_steps(torch, start, args.steps, args.warmup, None)
+        detail["combining"]["ms_warm"] = tukey_median(warm)
+        # per-round launches (the paper's schedule, one launch per round) and the direct kernel
+        for key, alg, fusion in (("combining_per_round", iso.ISO_ALG_COMBINING, 0), ("direct", iso.ISO_ALG_DIRECT, 1)):
+            s2 = b.set(alg, fusion)
+            tt = time_steps(torch, start, args.steps, args.warmup, flush)
+            m2 = sum(tt) / len(tt)
+            detail[key] = {"launches": s2["launches"], "bytes_moved": s2["bytes_moved"], "ms_cold": m2,
+                           "gbs_moved": s2["bytes_moved"] / (m2 * 1e-3) / 1e9,
+                           "gbs_payload": s2["bytes_min"] / (m2 * 1e-3) / 1e9,
+                           "frac_of_peak_moved": s2["bytes_moved"] / (m2 * 1e-3) / 1e9 / peak}
+        st = b.set(iso.ISO_ALG_COMBINING, args.fusion)
+
+        # ---- end to end: host buffers in, host buffers out, through the C-ABI -----------
+        hs = torch.empty(b.w.P * b.ss, dtype=torch.uint8).pin_memory()
+        hs.copy_(b.send.cpu())
+        hr = torch.empty(b.w.P * b.rs, dtype=torch.uint8).pin_memory()
+
+        def start_host():
+            iso.Iso_Start_host(b.req, hs, hr, stream)
+
+        e2e_steps = max(3, min(args.steps, 20))
+        te = time_steps(torch, start_host, e2e_steps, 3, None)
+        me = sum(te) / len(te)
+        line["e2e"] = {"value": moved / (me * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": me,
+                       "h2d_bytes_per_step": int(hs.numel()), "d2h_bytes_per_step": int(hr.numel()),
+                       "payload_gbs": minimum / (me * 1e-3) / 1e9}
+
+        # ---- roofline of the dominant kernel ------------------------------------------
+        launches = max(1, st["launches"])
+        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_vec<16,4>"
+        line["roofline"] = {
+            "bound": "hbm", "kernel": kernel, "achieved": per_gpu, "peak": peak, "unit": "GB/s",
+            "frac": per_gpu / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
+            "bytes_per_launch": moved // launches, "avg_launch_ms": ms / launches,
+            "traffic": args.traffic,
+            "note": "achieved = bytes read+written per launch / (step time / launches per step); "
+                    "launch gaps are inside the step time",
+        }
+        line["cpu_baseline"] = cpu_baseline(b.w, args.cpu_seconds)
+
+        if args.sweep:
+            detail["sweep"] = sweep(torch, iso, wl, flush, peak, args)
+    elif rank == 0:
+        line["e2e"] = None
+        line["roofline"] = {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s",
+                            "frac": per_gpu / peak, "traffic": None, "peak_kind": "%s copy bandwidth" % peak_kind}
+
+    line["clocks"] = clocks
+    line["detail"] = detail
+    b.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def sweep(torch, iso, wl, flush, peak, args):
+    """Every named workload, combining (fusion level 1) and direct: for the results table."""
+    out = {}
+    names = [n for n in wl.CONFIG_NAMES]
+    for name in names:
+        b = Bound(torch, iso, wl, name)
+        stream = torch.cuda.current_stream()
+        row = {}
+        for key, alg, fusion in (("combining", iso.ISO_ALG_COMBINING, 1), ("combining_per_round", iso.ISO_ALG_COMBINING, 0),
+                                 ("direct", iso.ISO_ALG_DIRECT, 1)):
+            st = b.set(alg, fusion)
+            steps = 20 if st["bytes_moved"] < (4 << 30) else 5
+            tt = time_steps(torch, lambda: iso.Iso_Start(b.req, stream), steps, 3, flush)
+            tw = time_steps(torch, lambda: iso.Iso_Start(b.req, stream), steps, 3, None)
+            ms, msw = tukey_median(tt), tukey_median(tw)
+            row[key] = {"rounds": st["rounds"], "launches": st["launches"], "bytes_moved": st["bytes_moved"],
+                        "bytes_min": st["bytes_min"], "bulk_bytes": st["bulk_bytes"], "ms_cold": ms, "ms_warm": msw,
+                        "gbs_moved": st["bytes_moved"] / ms / 1e6, "gbs_payload": st["bytes_min"] / ms / 1e6,
+                        "frac_moved_of_peak": st["bytes_moved"] / ms / 1e6 / peak,
+                        "frac_moved_of_8TBs": st["bytes_moved"] / ms / 1e6 / NOMINAL_HBM_GBS}
+        out[name] = row
+        b.close()
+        del b
+        torch.cuda.empty_cache()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2_alltoall")
+    ap.add_argument("--fusion", type=int, default=1)
+    ap.add_argument("--sweep", action="store_true", help="also time every named workload")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture, if one is current")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

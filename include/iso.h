@@ -1,0 +1,257 @@
+/*
+ * iso.h - isomorphic, sparse neighbourhood collectives for P virtual processes on a
+ * d-dimensional periodic torus, all resident in the memory of one CUDA device.
+ *
+ * The interface follows the persistent interface of the paper "Message-Combining
+ * Algorithms for Isomorphic, Sparse Collective Communication" (Listings 1, 2 and 4):
+ * a neighbourhood is created once from a list of relative coordinate vectors, an
+ * `..._init` call binds buffers and precomputes a schedule, and `Iso_Start` runs it any
+ * number of times.  MPI communicators and datatypes are replaced by plain integers.
+ *
+ * Model.  There are P = p_0 * ... * p_{d-1} processes; the process of rank r has the
+ * coordinates of r written in the mixed radix (p_0, ..., p_{d-1}) with dimension d-1
+ * varying fastest (the order of an MPI Cartesian communicator; the paper leaves it to
+ * that communicator).  A buffer argument is a DEVICE pointer to the buffers of all P
+ * processes, process-major: the buffer of process r starts `r * stride` bytes after the
+ * pointer, where the stride is
+ *     regular all-to-all : s * count * size            (s blocks back to back, Section II)
+ *     allgather          : count * size   (send side), s * count * size (receive side)
+ *     irregular          : max_i(displ_i + count_i * size), rounded up to a multiple of 16
+ * `Iso_request_get_stats` reports the strides in use.
+ *
+ * Result (Section II).  With C^i the i-th relative coordinate vector and (-) the
+ * component-wise subtraction modulo p_j, after `Iso_Start` + `Iso_wait`
+ *     all-to-all : block i of process R's receive buffer = block i of the send buffer of R (-) C^i
+ *     allgather  : block i of process R's receive buffer = the send block of R (-) C^i.
+ *
+ * Every function returns ISO_SUCCESS (0) or a positive ISO_ERR_* code; no exception or
+ * abort crosses this boundary and output arguments are left untouched on failure.
+ * Unless stated otherwise all pointer arguments other than buffers are HOST pointers that
+ * are only read during the call.  The library is not thread safe per object: use one
+ * request from one host thread at a time.
+ */
+#ifndef ISO_H
+#define ISO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ISO_MAX_DIMS 8
+
+typedef struct Iso_comm_s *Iso_comm;       /* neighbourhood object, library owned */
+typedef struct Iso_request_s *Iso_request; /* persistent collective, library owned */
+
+/* Basic datatypes only carry a size: the payload is moved as opaque bytes.  Any positive
+ * value is accepted and read as "bytes per element". */
+typedef int Iso_datatype;
+#define ISO_BYTE 1
+#define ISO_INT32 4
+#define ISO_FLOAT 4
+#define ISO_DOUBLE 8
+
+enum {
+    ISO_SUCCESS = 0,
+    ISO_ERR_ARG = 1,     /* null pointer, negative count, unknown enum value, bad handle */
+    ISO_ERR_DIMS = 2,    /* d outside 1..ISO_MAX_DIMS, a dimension size < 1, P too large */
+    ISO_ERR_COUNT = 3,   /* send and receive block sizes differ, or a size overflows */
+    ISO_ERR_ALIGN = 4,   /* reserved: no supported input is rejected for alignment */
+    ISO_ERR_NOMEM = 5,   /* host or device allocation failed */
+    ISO_ERR_CUDA = 6,    /* a CUDA call failed; see Iso_last_cuda_error */
+    ISO_ERR_OVERLAP = 7, /* receive blocks overlap each other, or send and receive buffers overlap */
+    ISO_ERR_STATE = 8,   /* call not valid in this state (e.g. request bound to no buffers) */
+    ISO_ERR_TIMEOUT = 9  /* a bounded wait inside a kernel expired; the result is incomplete */
+};
+
+/* Schedules. */
+enum {
+    ISO_ALG_COMBINING = 0, /* Section V: message combining with direct communication along
+                              the dimensions, one round per distinct non-zero coordinate */
+    ISO_ALG_DIRECT = 1,    /* Listing 3: every block straight from its source, here in one pass */
+    ISO_ALG_TORUS = 2      /* Section III, Algorithm 1: hop-by-hop between immediate neighbours */
+};
+
+enum { ISO_KIND_ALLTOALL = 0, ISO_KIND_ALLGATHER = 1, ISO_KIND_ALLTOALLV = 2 };
+enum { ISO_BUF_SEND = 0, ISO_BUF_RECV = 1, ISO_BUF_INTER = 2 };
+
+typedef struct Iso_stats {
+    int kind;             /* ISO_KIND_* */
+    int algorithm;        /* ISO_ALG_* */
+    int fusion_level;
+    int d;
+    int s;
+    int rounds;           /* communication rounds of the schedule (Sections III-A and V) */
+    int max_rounds_per_dim; /* the factor N of the bound "at most N*d rounds" */
+    int phases;           /* groups of rounds that run without an ordering point between them */
+    int launches;         /* kernel launches per Iso_Start */
+    int parts;            /* block transmissions per process: sum of hops (all-to-all),
+                             trie edges that move a block (allgather) */
+    int local_copies;     /* blocks whose source is the process itself (no hop) */
+    int64_t P;
+    int64_t send_stride;  /* bytes between consecutive processes' send buffers */
+    int64_t recv_stride;
+    int64_t inter_stride; /* same for the library's intermediate buffer (0: none needed) */
+    int64_t bytes_min;    /* 2 * P * sum_i m_i: every delivered block read once, written once */
+    int64_t bytes_moved;  /* bytes read + written by one Iso_Start with this schedule */
+    int64_t bulk_bytes;   /* part of bytes_moved handled by the bulk-copy kernel */
+} Iso_stats;
+
+/* One line of a schedule as it is executed: in phase `phase`, every process r copies
+ * `len` bytes from byte `src_off` of buffer `src_buf` of process r (-) shift to byte
+ * `dst_off` of its own buffer `dst_buf`.  `slot` is the neighbour index i the bytes belong
+ * to; `round` numbers the paper's communication rounds (-1 for a local copy). */
+typedef struct Iso_part {
+    int phase;
+    int round;
+    int slot;
+    int src_buf;          /* ISO_BUF_* */
+    int dst_buf;
+    int kernel;           /* 0: vector copy kernel, 1: bulk copy kernel */
+    int width;            /* bytes per vector unit (vector kernel) */
+    int reserved;
+    int64_t src_off;
+    int64_t dst_off;
+    int64_t len;
+    int shift[ISO_MAX_DIMS]; /* per dimension, reduced to [0, p_j) */
+} Iso_part;
+
+/*
+ * Neighbourhood set-up (Listing 1, Section II).  `dims[0..d-1]` are the torus sizes,
+ * `relative_coordinates` holds s*d integers, neighbour-major (vector i occupies entries
+ * i*d .. i*d+d-1).  Any integers are allowed: repetitions, the zero vector, coordinates
+ * whose magnitude exceeds the torus size.  The order of the vectors fixes the order of
+ * the blocks in the buffers.  s = 0 is valid.  The arrays are copied.
+ * Errors: ISO_ERR_ARG (null pointer, s < 0), ISO_ERR_DIMS, ISO_ERR_NOMEM.
+ */
+int Iso_neighborhood_create(int d, const int dims[], int s, const int relative_coordinates[],
+                            Iso_comm *isocomm);
+
+/* Releases the neighbourhood; requests created from it keep it alive until they are freed.
+ * `*isocomm` is set to NULL. */
+int Iso_comm_free(Iso_comm *isocomm);
+
+/*
+ * Regular all-to-all (Listing 2, Section II): s blocks of sendcount * sendtype bytes per
+ * process, stored consecutively in neighbour order in both buffers.  The block sizes in
+ * bytes on the send and receive side must be equal (ISO_ERR_COUNT otherwise).
+ * The schedule (Section V with the buffer alternation of Algorithm 1) is computed here, on
+ * the host; device resources (the intermediate buffer and the index tables) are created by
+ * the first Iso_Start.  `sendbuf` and `recvbuf` are device pointers owned by the caller,
+ * must not overlap, must stay valid while the request is in use; the send buffer is never
+ * written.  Both may be NULL: the request can then be inspected (statistics, parts) but
+ * not started.
+ */
+int Iso_neighbor_alltoall_init(const void *sendbuf, int sendcount, Iso_datatype sendtype,
+                               void *recvbuf, int recvcount, Iso_datatype recvtype,
+                               Iso_comm isocomm, Iso_request *request);
+
+/*
+ * Allgather (Listing 2, Sections II and III-B): every process contributes ONE block of
+ * sendcount * sendtype bytes and receives s blocks in neighbour order.  The schedule is
+ * the prefix-trie schedule of Section III-B in its direct-communication form (Section V).
+ * Buffer rules as for the all-to-all.
+ */
+int Iso_neighbor_allgather_init(const void *sendbuf, int sendcount, Iso_datatype sendtype,
+                                void *recvbuf, int recvcount, Iso_datatype recvtype,
+                                Iso_comm isocomm, Iso_request *request);
+
+/*
+ * Irregular all-to-all (Listing 4, Section II): block i has sendcounts[i] elements at
+ * byte displacement senddispls[i] of a process's send buffer and arrives at byte
+ * displacement recvdispls[i] of the receiver's buffer.  Counts and displacements (s
+ * entries each, host arrays, copied) are the same on every process and block sizes must
+ * match pairwise in bytes (ISO_ERR_COUNT).  Displacements must be >= 0; receive blocks
+ * must not overlap each other (ISO_ERR_OVERLAP); send blocks may.  "It uses the same
+ * schedules as in the regular case" (Section IV).
+ */
+int Iso_neighbor_alltoallv_init(const void *sendbuf, const int sendcounts[],
+                                const int64_t senddispls[], Iso_datatype sendtype,
+                                void *recvbuf, const int recvcounts[],
+                                const int64_t recvdispls[], Iso_datatype recvtype,
+                                Iso_comm isocomm, Iso_request *request);
+
+/*
+ * Irregular allgather (Listing 4): one send block of sendcount * sendtype bytes per
+ * process; the copy received from neighbour i is stored at byte displacement
+ * recvdispls[i]; recvcounts[i] * recvtype must equal the send block size for every i.
+ */
+int Iso_neighbor_allgatherv_init(const void *sendbuf, int sendcount, Iso_datatype sendtype,
+                                 void *recvbuf, const int recvcounts[],
+                                 const int64_t recvdispls[], Iso_datatype recvtype,
+                                 Iso_comm isocomm, Iso_request *request);
+
+/*
+ * Chooses the schedule.  `alg` is an ISO_ALG_* value.  `fusion_level` applies to
+ * ISO_ALG_COMBINING: 0 = one kernel launch per communication round; 1 (the default) = all
+ * rounds of one dimension in one launch (same bytes moved: within a dimension every block
+ * moves at most once); g >= 2 = the dimensions are taken in groups of g consecutive ones and
+ * a block's hops inside a group are composed into a single shift (Section V: "all blocks
+ * going to the same relative neighbor ... can be combined"), so fewer intermediate copies
+ * pass through memory; g >= d moves exactly the bytes of ISO_ALG_DIRECT.
+ * May be called at any time between starts; the schedule is rebuilt and the device tables
+ * are replaced by the next Iso_Start.  Errors: ISO_ERR_ARG.
+ */
+int Iso_request_set_algorithm(Iso_request request, int alg, int fusion_level);
+
+/* Parts of at least `bytes` bytes whose addresses and length are multiples of 16 are moved
+ * by the bulk-copy kernel (asynchronous bulk copies staged through shared memory), the rest
+ * by the vector kernel.  Default 1024; 0 disables the bulk kernel. */
+int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes);
+
+/*
+ * Non-periodic dimensions (Section VII: "our schedules can easily be extended to
+ * non-periodic tori").  periodic[j] = 0 makes dimension j a mesh: a block whose source
+ * R - C^i falls outside the mesh is not delivered and the receive slot keeps its previous
+ * contents.  Only ISO_ALG_DIRECT supports meshes.  Default: all dimensions periodic.
+ */
+int Iso_comm_set_periodic(Iso_comm isocomm, const int periodic[]);
+
+/*
+ * Runs the collective: enqueues the schedule's kernels on `cuda_stream` (a cudaStream_t
+ * cast to void*, NULL = the default stream) and returns without waiting (the non-blocking
+ * start proposed in Section VII).  The first start after an init or a set_* call also
+ * allocates the intermediate buffer and uploads the index tables (cudaMalloc and a blocking
+ * copy), so it must not happen inside a stream capture.
+ * Errors: ISO_ERR_STATE (request has no buffers), ISO_ERR_NOMEM, ISO_ERR_CUDA.
+ */
+int Iso_Start(Iso_request request, void *cuda_stream);
+
+/* Same with HOST buffers holding all P processes' send / receive buffers in the layout
+ * above: copies `host_sendbuf` to the request's device send buffer, runs the schedule and
+ * copies the device receive buffer to `host_recvbuf`, all on `cuda_stream`.  The copies are
+ * asynchronous when the host memory is page-locked.  Complete after Iso_wait. */
+int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_recvbuf,
+                   void *cuda_stream);
+
+/* Local completion (Section VII): blocks until the last start has finished and returns
+ * ISO_ERR_TIMEOUT if a kernel gave up a bounded wait, ISO_ERR_CUDA on a CUDA error. */
+int Iso_wait(Iso_request request);
+
+/* Statistics of the current schedule.  Host only; valid before the first start. */
+int Iso_request_get_stats(Iso_request request, Iso_stats *out);
+
+/* Copies up to `capacity` executed parts (in execution order) to `out` and stores the
+ * total number in `*count`.  Needs no device; meant for validation of schedules. */
+int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int *count);
+
+/* Frees the request, its device memory and its reference on the neighbourhood; waits for
+ * work in flight first.  `*request` is set to NULL. */
+int Iso_request_free(Iso_request *request);
+
+/* Static text for an ISO_ERR_* code. */
+const char *Iso_error_string(int code);
+
+/* The cudaError_t value of the CUDA call that last failed inside the library on this
+ * host thread (0 if none). */
+int Iso_last_cuda_error(void);
+
+/* Host-side consistency checks of the library's integer helpers (exact division by
+ * multiplication, alignment classes).  Returns ISO_SUCCESS or ISO_ERR_STATE.  No device. */
+int Iso_selftest(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ISO_H */

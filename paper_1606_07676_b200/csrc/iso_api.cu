@@ -1,0 +1,584 @@
+// C-ABI of the isomorphic neighbourhood collectives (declared in include/iso.h):
+// argument checking, object lifetime, device tables and kernel launches.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "iso.h"
+#include "iso_internal.h"
+#include "iso_kernels.cuh"
+
+using namespace iso;
+
+struct Iso_comm_s : public Comm {};
+struct Iso_request_s : public Request {};
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    (void)cudaGetLastError();  // clear the sticky flag of non-fatal errors
+    return e == cudaErrorMemoryAllocation ? ISO_ERR_NOMEM : ISO_ERR_CUDA;
+}
+
+#define ISO_CUDA(call)                               \
+    do {                                             \
+        cudaError_t e_ = (call);                     \
+        if (e_ != cudaSuccess) return cuda_fail(e_); \
+    } while (0)
+
+void release_device(Request &r)
+{
+    if (r.d_blob) cudaFree(r.d_blob);
+    if (r.d_inter) cudaFree(r.d_inter);
+    if (r.d_err) cudaFree(r.d_err);
+    if (r.h_err) cudaFreeHost(r.h_err);
+    r.d_blob = nullptr;
+    r.d_inter = nullptr;
+    r.d_err = nullptr;
+    r.h_err = nullptr;
+    r.d_inter_bytes = 0;
+    r.dirty = true;
+}
+
+void comm_unref(Comm *c)
+{
+    if (c && --c->refcount == 0) delete static_cast<Iso_comm_s *>(c);
+}
+
+bool mul_overflows(int64_t a, int64_t b)
+{
+    if (a == 0 || b == 0) return false;
+    return a > INT64_MAX / b;
+}
+
+// Common tail of the init calls: strides are set, block layout is in r.
+int finish_init(Iso_request_s *r, Iso_request *out)
+{
+    const Comm &c = *r->comm;
+    if (mul_overflows(c.P, r->send_stride) || mul_overflows(c.P, r->recv_stride)) {
+        comm_unref(r->comm);
+        delete r;
+        return ISO_ERR_COUNT;
+    }
+    // receive blocks must not overlap each other
+    {
+        std::vector<std::pair<int64_t, int64_t>> iv;
+        for (int i = 0; i < r->s; ++i)
+            if (r->len[i] > 0) iv.push_back({r->rdispl[i], r->rdispl[i] + r->len[i]});
+        std::sort(iv.begin(), iv.end());
+        for (size_t k = 1; k < iv.size(); ++k)
+            if (iv[k].first < iv[k - 1].second) {
+                comm_unref(r->comm);
+                delete r;
+                return ISO_ERR_OVERLAP;
+            }
+    }
+    // the two user buffers must not overlap
+    if (r->send && r->recv) {
+        const unsigned char *s0 = r->send, *s1 = r->send + c.P * r->send_stride;
+        const unsigned char *d0 = r->recv, *d1 = r->recv + c.P * r->recv_stride;
+        if (s0 < d1 && d0 < s1 && s0 != s1 && d0 != d1) {
+            comm_unref(r->comm);
+            delete r;
+            return ISO_ERR_OVERLAP;
+        }
+    }
+    int rc = build_schedule(*r);
+    if (rc == ISO_SUCCESS) rc = lower_schedule(*r, (uintptr_t)r->send, (uintptr_t)r->recv, 0);
+    if (rc != ISO_SUCCESS) {
+        comm_unref(r->comm);
+        delete r;
+        return rc;
+    }
+    *out = r;
+    return ISO_SUCCESS;
+}
+
+Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *recvbuf)
+{
+    Iso_request_s *r = new (std::nothrow) Iso_request_s();
+    if (!r) return nullptr;
+    r->comm = comm;
+    comm->refcount++;
+    r->kind = kind;
+    r->send = static_cast<const unsigned char *>(sendbuf);
+    r->recv = static_cast<unsigned char *>(recvbuf);
+    r->s = comm->s;
+    r->len.assign(comm->s, 0);
+    r->sdispl.assign(comm->s, 0);
+    r->rdispl.assign(comm->s, 0);
+    return r;
+}
+
+int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
+
+// Uploads the lowered schedule and allocates the intermediate buffer.
+int materialise(Request &r)
+{
+    const Comm &c = *r.comm;
+    // device tables depend on the alignment of the intermediate buffer: allocate it first
+    const int64_t inter_bytes = c.P * r.inter_stride;
+    if (inter_bytes > r.d_inter_bytes) {
+        if (r.d_inter) cudaFree(r.d_inter);
+        r.d_inter = nullptr;
+        r.d_inter_bytes = 0;
+        ISO_CUDA(cudaMalloc((void **)&r.d_inter, (size_t)inter_bytes));
+        r.d_inter_bytes = inter_bytes;
+    }
+    int rc = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
+    if (rc != ISO_SUCCESS) return rc;
+
+    size_t bytes = 0;
+    for (LaunchPlan &L : r.launches) {
+        L.parts_off = bytes;
+        bytes += L.parts.size() * sizeof(PartDev);
+        L.lookup_off = bytes;
+        bytes += (L.lookup.size() * sizeof(uint16_t) + 15) / 16 * 16;
+    }
+    std::vector<unsigned char> blob(bytes ? bytes : 16, 0);
+    for (const LaunchPlan &L : r.launches) {
+        int used_index[ISO_MAX_DIMS];
+        for (int j = 0; j < ISO_MAX_DIMS; ++j) used_index[j] = -1;
+        for (int k = 0; k < L.n_used; ++k) used_index[L.used_dim[k]] = k;
+        PartDev *pd = reinterpret_cast<PartDev *>(blob.data() + L.parts_off);
+        for (size_t t = 0; t < L.parts.size(); ++t) {
+            const LoweredPart &lp = L.parts[t];
+            PartDev d{};
+            d.src_off = lp.p.src_off;
+            d.dst_off = lp.p.dst_off;
+            d.len = lp.p.len;
+            d.first_unit = lp.first_unit;
+            d.units = lp.units;
+            d.src_buf = (uint8_t)lp.p.src_buf;
+            d.dst_buf = (uint8_t)lp.p.dst_buf;
+            long long delta = 0;
+            int nnz = 0;
+            for (int j = 0; j < c.d; ++j) {
+                if (!lp.p.shift[j]) continue;
+                delta -= (long long)lp.p.shift[j] * c.rank_stride[j];
+                d.dim[nnz] = (uint8_t)used_index[j];
+                d.c[nnz] = lp.p.shift[j];
+                ++nnz;
+            }
+            d.nnz = (uint8_t)nnz;
+            d.rank_delta = delta;
+            pd[t] = d;
+        }
+        if (!L.lookup.empty())
+            std::memcpy(blob.data() + L.lookup_off, L.lookup.data(), L.lookup.size() * sizeof(uint16_t));
+    }
+    if (r.d_blob) cudaFree(r.d_blob);
+    r.d_blob = nullptr;
+    ISO_CUDA(cudaMalloc(&r.d_blob, blob.size()));
+    ISO_CUDA(cudaMemcpy(r.d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice));
+    if (!r.d_err) {
+        ISO_CUDA(cudaMalloc((void **)&r.d_err, sizeof(int)));
+        ISO_CUDA(cudaMemset(r.d_err, 0, sizeof(int)));
+    }
+    if (!r.h_err) {
+        ISO_CUDA(cudaMallocHost((void **)&r.h_err, sizeof(int)));
+        *r.h_err = 0;
+    }
+    // opt in to large dynamic shared memory once per kernel
+    static bool attrs_set = false;
+    if (!attrs_set) {
+        ISO_CUDA(cudaFuncSetAttribute(iso_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attrs_set = true;
+    }
+    r.dirty = false;
+    return ISO_SUCCESS;
+}
+
+LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
+{
+    const Comm &c = *r.comm;
+    LaunchDev a{};
+    a.parts = reinterpret_cast<const PartDev *>(static_cast<unsigned char *>(r.d_blob) + L.parts_off);
+    a.lookup = reinterpret_cast<const uint16_t *>(static_cast<unsigned char *>(r.d_blob) + L.lookup_off);
+    a.buf[ISO_BUF_SEND] = const_cast<unsigned char *>(r.send);
+    a.buf[ISO_BUF_RECV] = r.recv;
+    a.buf[ISO_BUF_INTER] = r.d_inter;
+    a.buf_stride[ISO_BUF_SEND] = r.send_stride;
+    a.buf_stride[ISO_BUF_RECV] = r.recv_stride;
+    a.buf_stride[ISO_BUF_INTER] = r.inter_stride;
+    a.P = c.P;
+    a.err = r.d_err;
+    a.nparts = (uint32_t)L.parts.size();
+    a.units_per_proc = L.units_per_proc;
+    a.uniform_units = L.uniform_units;
+    a.lookup_shift = (uint32_t)L.lookup_shift;
+    a.width = (uint32_t)L.width;
+    a.tile_procs = L.tile_procs;
+    a.n_used = L.n_used;
+    a.mesh_mask = 0;
+    FastDiv f = make_fastdiv(L.units_per_proc);
+    a.div_units = FastDivDev{f.m, f.s1, f.s2, f.div};
+    f = make_fastdiv(L.uniform_units ? L.uniform_units : 1);
+    a.div_uniform = FastDivDev{f.m, f.s1, f.s2, f.div};
+    for (int k = 0; k < L.n_used; ++k) {
+        const int j = L.used_dim[k];
+        a.used_dim[k] = j;
+        a.used_size[k] = (uint32_t)c.dims[j];
+        a.used_rstride[k] = c.rank_stride[j];
+        if (!c.periodic[j]) a.mesh_mask |= 1 << k;
+    }
+    return a;
+}
+
+int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream)
+{
+    if (L.grid == 0 || L.units_per_proc == 0) return ISO_SUCCESS;
+    LaunchDev a = make_launch_args(r, L);
+    dim3 grid((unsigned)L.grid), block((unsigned)L.threads);
+    if (L.kernel == KERNEL_BULK) {
+        iso_gather_bulk<<<grid, block, L.smem, stream>>>(a);
+    } else {
+        switch (L.width) {
+        case 16: iso_gather_vec<16, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 8: iso_gather_vec<8, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 4: iso_gather_vec<4, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 2: iso_gather_vec<2, 4><<<grid, block, L.smem, stream>>>(a); break;
+        default: iso_gather_vec<1, 4><<<grid, block, L.smem, stream>>>(a); break;
+        }
+    }
+    ISO_CUDA(cudaGetLastError());
+    return ISO_SUCCESS;
+}
+
+int check_handle(Iso_request request)
+{
+    return request && request->comm ? ISO_SUCCESS : ISO_ERR_ARG;
+}
+
+}  // namespace
+
+extern "C" {
+
+int Iso_neighborhood_create(int d, const int dims[], int s, const int relative_coordinates[], Iso_comm *isocomm)
+{
+    if (!isocomm || !dims || s < 0 || (s > 0 && !relative_coordinates)) return ISO_ERR_ARG;
+    if (d < 1 || d > ISO_MAX_DIMS) return ISO_ERR_DIMS;
+    int64_t P = 1;
+    for (int j = 0; j < d; ++j) {
+        if (dims[j] < 1) return ISO_ERR_DIMS;
+        if (P > (int64_t)0x7fffffff / dims[j]) return ISO_ERR_DIMS;  // ranks are kept below 2^31
+        P *= dims[j];
+    }
+    Iso_comm_s *c = new (std::nothrow) Iso_comm_s();
+    if (!c) return ISO_ERR_NOMEM;
+    c->d = d;
+    c->s = s;
+    c->P = P;
+    int64_t stride = 1;
+    for (int j = d - 1; j >= 0; --j) {
+        c->dims[j] = dims[j];
+        c->periodic[j] = 1;
+        c->rank_stride[j] = stride;
+        stride *= dims[j];
+    }
+    try {
+        c->coords.assign(relative_coordinates, relative_coordinates + (size_t)s * d);
+    } catch (...) {
+        delete c;
+        return ISO_ERR_NOMEM;
+    }
+    *isocomm = c;
+    return ISO_SUCCESS;
+}
+
+int Iso_comm_set_periodic(Iso_comm isocomm, const int periodic[])
+{
+    if (!isocomm || !periodic) return ISO_ERR_ARG;
+    for (int j = 0; j < isocomm->d; ++j) isocomm->periodic[j] = periodic[j] ? 1 : 0;
+    return ISO_SUCCESS;
+}
+
+int Iso_comm_free(Iso_comm *isocomm)
+{
+    if (!isocomm || !*isocomm) return ISO_ERR_ARG;
+    comm_unref(*isocomm);
+    *isocomm = nullptr;
+    return ISO_SUCCESS;
+}
+
+int Iso_neighbor_alltoall_init(const void *sendbuf, int sendcount, Iso_datatype sendtype, void *recvbuf,
+                               int recvcount, Iso_datatype recvtype, Iso_comm isocomm, Iso_request *request)
+{
+    if (!isocomm || !request || sendcount < 0 || recvcount < 0 || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
+    if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
+    const int64_t m = (int64_t)sendcount * sendtype;
+    if (m != (int64_t)recvcount * recvtype) return ISO_ERR_COUNT;
+    Iso_request_s *r = new_request(isocomm, ISO_KIND_ALLTOALL, sendbuf, recvbuf);
+    if (!r) return ISO_ERR_NOMEM;
+    for (int i = 0; i < r->s; ++i) {
+        r->len[i] = m;
+        r->sdispl[i] = r->rdispl[i] = (int64_t)i * m;
+    }
+    r->send_stride = r->recv_stride = (int64_t)r->s * m;
+    return finish_init(r, request);
+}
+
+int Iso_neighbor_allgather_init(const void *sendbuf, int sendcount, Iso_datatype sendtype, void *recvbuf,
+                                int recvcount, Iso_datatype recvtype, Iso_comm isocomm, Iso_request *request)
+{
+    if (!isocomm || !request || sendcount < 0 || recvcount < 0 || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
+    if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
+    const int64_t m = (int64_t)sendcount * sendtype;
+    if (m != (int64_t)recvcount * recvtype) return ISO_ERR_COUNT;
+    Iso_request_s *r = new_request(isocomm, ISO_KIND_ALLGATHER, sendbuf, recvbuf);
+    if (!r) return ISO_ERR_NOMEM;
+    for (int i = 0; i < r->s; ++i) {
+        r->len[i] = m;
+        r->sdispl[i] = 0;
+        r->rdispl[i] = (int64_t)i * m;
+    }
+    r->send_stride = m;
+    r->recv_stride = (int64_t)r->s * m;
+    return finish_init(r, request);
+}
+
+int Iso_neighbor_alltoallv_init(const void *sendbuf, const int sendcounts[], const int64_t senddispls[],
+                                Iso_datatype sendtype, void *recvbuf, const int recvcounts[],
+                                const int64_t recvdispls[], Iso_datatype recvtype, Iso_comm isocomm,
+                                Iso_request *request)
+{
+    if (!isocomm || !request || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
+    if (isocomm->s > 0 && (!sendcounts || !senddispls || !recvcounts || !recvdispls)) return ISO_ERR_ARG;
+    if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
+    for (int i = 0; i < isocomm->s; ++i) {
+        if (sendcounts[i] < 0 || recvcounts[i] < 0 || senddispls[i] < 0 || recvdispls[i] < 0) return ISO_ERR_ARG;
+        if ((int64_t)sendcounts[i] * sendtype != (int64_t)recvcounts[i] * recvtype) return ISO_ERR_COUNT;
+    }
+    Iso_request_s *r = new_request(isocomm, ISO_KIND_ALLTOALLV, sendbuf, recvbuf);
+    if (!r) return ISO_ERR_NOMEM;
+    int64_t se = 0, re = 0;
+    for (int i = 0; i < r->s; ++i) {
+        r->len[i] = (int64_t)sendcounts[i] * sendtype;
+        r->sdispl[i] = senddispls[i];
+        r->rdispl[i] = recvdispls[i];
+        se = std::max(se, senddispls[i] + r->len[i]);
+        re = std::max(re, recvdispls[i] + r->len[i]);
+    }
+    r->send_stride = round_up16(se);
+    r->recv_stride = round_up16(re);
+    return finish_init(r, request);
+}
+
+int Iso_neighbor_allgatherv_init(const void *sendbuf, int sendcount, Iso_datatype sendtype, void *recvbuf,
+                                 const int recvcounts[], const int64_t recvdispls[], Iso_datatype recvtype,
+                                 Iso_comm isocomm, Iso_request *request)
+{
+    if (!isocomm || !request || sendcount < 0 || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
+    if (isocomm->s > 0 && (!recvcounts || !recvdispls)) return ISO_ERR_ARG;
+    if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
+    const int64_t m = (int64_t)sendcount * sendtype;
+    for (int i = 0; i < isocomm->s; ++i) {
+        if (recvcounts[i] < 0 || recvdispls[i] < 0) return ISO_ERR_ARG;
+        if ((int64_t)recvcounts[i] * recvtype != m) return ISO_ERR_COUNT;
+    }
+    Iso_request_s *r = new_request(isocomm, ISO_KIND_ALLGATHER, sendbuf, recvbuf);
+    if (!r) return ISO_ERR_NOMEM;
+    int64_t re = 0;
+    for (int i = 0; i < r->s; ++i) {
+        r->len[i] = m;
+        r->sdispl[i] = 0;
+        r->rdispl[i] = recvdispls[i];
+        re = std::max(re, recvdispls[i] + m);
+    }
+    r->send_stride = round_up16(m);
+    r->recv_stride = round_up16(re);
+    return finish_init(r, request);
+}
+
+int Iso_request_set_algorithm(Iso_request request, int alg, int fusion_level)
+{
+    if (check_handle(request)) return ISO_ERR_ARG;
+    if (alg != ISO_ALG_COMBINING && alg != ISO_ALG_DIRECT && alg != ISO_ALG_TORUS) return ISO_ERR_ARG;
+    if (fusion_level < 0) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    const int old_alg = request->alg, old_fusion = request->fusion;
+    request->alg = alg;
+    request->fusion = fusion_level;
+    int rc = build_schedule(*request);
+    if (rc == ISO_SUCCESS)
+        rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
+    if (rc != ISO_SUCCESS) {
+        request->alg = old_alg;
+        request->fusion = old_fusion;
+        build_schedule(*request);
+        lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
+    }
+    request->dirty = true;
+    return rc;
+}
+
+int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
+{
+    if (check_handle(request) || bytes < 0) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    request->bulk_threshold = bytes;
+    int rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
+    request->dirty = true;
+    return rc;
+}
+
+int Iso_Start(Iso_request request, void *cuda_stream)
+{
+    if (check_handle(request)) return ISO_ERR_ARG;
+    Request &r = *request;
+    if (!r.send || !r.recv) return ISO_ERR_STATE;
+    if (r.dirty) {
+        if (r.started) {
+            int rc = Iso_wait(request);
+            if (rc != ISO_SUCCESS) return rc;
+        }
+        int rc = materialise(r);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (const LaunchPlan &L : r.launches) {
+        int rc = launch_one(r, L, stream);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    r.last_stream = cuda_stream;
+    r.started = true;
+    return ISO_SUCCESS;
+}
+
+int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_recvbuf, void *cuda_stream)
+{
+    if (check_handle(request) || !host_sendbuf || !host_recvbuf) return ISO_ERR_ARG;
+    Request &r = *request;
+    if (!r.send || !r.recv) return ISO_ERR_STATE;
+    const Comm &c = *r.comm;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t sbytes = (size_t)(c.P * r.send_stride), rbytes = (size_t)(c.P * r.recv_stride);
+    if (sbytes)
+        ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send), host_sendbuf, sbytes, cudaMemcpyHostToDevice, stream));
+    int rc = Iso_Start(request, cuda_stream);
+    if (rc != ISO_SUCCESS) return rc;
+    if (rbytes) ISO_CUDA(cudaMemcpyAsync(host_recvbuf, r.recv, rbytes, cudaMemcpyDeviceToHost, stream));
+    return ISO_SUCCESS;
+}
+
+int Iso_wait(Iso_request request)
+{
+    if (check_handle(request)) return ISO_ERR_ARG;
+    Request &r = *request;
+    if (!r.started) return ISO_SUCCESS;
+    cudaStream_t stream = static_cast<cudaStream_t>(r.last_stream);
+    if (r.d_err && r.h_err) {
+        ISO_CUDA(cudaMemcpyAsync(r.h_err, r.d_err, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    }
+    ISO_CUDA(cudaStreamSynchronize(stream));
+    if (r.h_err && *r.h_err) {
+        *r.h_err = 0;
+        cudaMemsetAsync(r.d_err, 0, sizeof(int), stream);
+        return ISO_ERR_TIMEOUT;
+    }
+    return ISO_SUCCESS;
+}
+
+int Iso_request_get_stats(Iso_request request, Iso_stats *out)
+{
+    if (check_handle(request) || !out) return ISO_ERR_ARG;
+    *out = request->stats;
+    return ISO_SUCCESS;
+}
+
+int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int *count)
+{
+    if (check_handle(request) || !count || capacity < 0 || (capacity > 0 && !out)) return ISO_ERR_ARG;
+    int n = 0;
+    for (const LaunchPlan &L : request->launches) {
+        for (const LoweredPart &lp : L.parts) {
+            if (n < capacity) {
+                Iso_part q{};
+                q.phase = lp.p.phase;
+                q.round = lp.p.round;
+                q.slot = lp.p.slot;
+                q.src_buf = lp.p.src_buf;
+                q.dst_buf = lp.p.dst_buf;
+                q.kernel = L.kernel;
+                q.width = L.width;
+                q.src_off = lp.p.src_off;
+                q.dst_off = lp.p.dst_off;
+                q.len = lp.p.len;
+                std::memcpy(q.shift, lp.p.shift, sizeof(q.shift));
+                out[n] = q;
+            }
+            ++n;
+        }
+    }
+    *count = n;
+    return ISO_SUCCESS;
+}
+
+int Iso_request_free(Iso_request *request)
+{
+    if (!request || !*request) return ISO_ERR_ARG;
+    Iso_request_s *r = *request;
+    int rc = ISO_SUCCESS;
+    if (r->started) rc = Iso_wait(r);
+    release_device(*r);
+    comm_unref(r->comm);
+    delete r;
+    *request = nullptr;
+    return rc == ISO_ERR_TIMEOUT ? ISO_SUCCESS : rc;
+}
+
+const char *Iso_error_string(int code)
+{
+    switch (code) {
+    case ISO_SUCCESS: return "success";
+    case ISO_ERR_ARG: return "invalid argument";
+    case ISO_ERR_DIMS: return "invalid torus dimensions";
+    case ISO_ERR_COUNT: return "block sizes do not match or overflow";
+    case ISO_ERR_ALIGN: return "unsupported alignment";
+    case ISO_ERR_NOMEM: return "out of memory";
+    case ISO_ERR_CUDA: return "CUDA call failed";
+    case ISO_ERR_OVERLAP: return "buffers or blocks overlap";
+    case ISO_ERR_STATE: return "call not valid in this state";
+    case ISO_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+    default: return "unknown error code";
+    }
+}
+
+int Iso_last_cuda_error(void) { return g_last_cuda_error; }
+
+int Iso_selftest(void)
+{
+    // exact division by multiplication: edge values and a pseudo-random sweep
+    const uint32_t divisors[] = {1, 2, 3, 5, 7, 9, 10, 36, 81, 162, 255, 256, 257, 1000, 1280, 6144, 65535, 65536, 65537,
+                                 1000003, 0x7fffffffu, 0x80000000u, 0xfffffffeu, 0xffffffffu};
+    uint64_t x = 88172645463325252ull;
+    for (uint32_t d : divisors) {
+        FastDiv f = make_fastdiv(d);
+        const uint32_t edges[] = {0, 1, d - 1, d, d + 1, 2 * d - 1, 2 * d, 0x7fffffffu, 0x80000000u, 0xffffffffu};
+        for (uint32_t n : edges)
+            if (fastdiv_host(f, n) != n / d) return ISO_ERR_STATE;
+        for (int k = 0; k < 20000; ++k) {
+            x ^= x << 13; x ^= x >> 7; x ^= x << 17;
+            uint32_t n = (uint32_t)(x >> 16);
+            if (fastdiv_host(f, n) != n / d) return ISO_ERR_STATE;
+        }
+    }
+    return ISO_SUCCESS;
+}
+
+}  // extern "C"

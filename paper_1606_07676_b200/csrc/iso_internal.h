@@ -1,0 +1,112 @@
+// Internal host-side types of the isomorphic neighbourhood collectives library.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "iso.h"
+
+namespace iso {
+
+struct Comm {
+    int refcount = 1;
+    int d = 0;
+    int s = 0;
+    int dims[ISO_MAX_DIMS] = {0};
+    int periodic[ISO_MAX_DIMS] = {0};
+    int64_t P = 1;
+    int64_t rank_stride[ISO_MAX_DIMS] = {0};  // ranks between neighbours along dimension j
+    std::vector<int> coords;                  // s*d, as given by the caller
+};
+
+// One line of the executed schedule, before it is lowered to kernel launches.
+struct Part {
+    int phase = 0;
+    int round = -1;
+    int slot = 0;
+    int src_buf = ISO_BUF_SEND;
+    int dst_buf = ISO_BUF_RECV;
+    int64_t src_off = 0;
+    int64_t dst_off = 0;
+    int64_t len = 0;
+    int shift[ISO_MAX_DIMS] = {0};  // residue in [0,p_j) for periodic dimensions, signed for mesh ones
+};
+
+// Exact unsigned 32-bit division by an invariant divisor (Granlund & Montgomery 1994,
+// round-up method): q = (t + ((n - t) >> s1)) >> s2 with t = mulhi(m, n).
+struct FastDiv {
+    uint32_t m = 1, s1 = 0, s2 = 0, div = 1;
+};
+FastDiv make_fastdiv(uint32_t divisor);
+inline uint32_t fastdiv_host(const FastDiv &f, uint32_t n)
+{
+    uint32_t t = (uint32_t)(((uint64_t)f.m * n) >> 32);
+    return (t + ((n - t) >> f.s1)) >> f.s2;
+}
+
+// A part as one kernel launch sees it (after splitting into aligned pieces).
+struct LoweredPart {
+    Part p;            // offsets / len of this piece
+    uint32_t first_unit = 0;
+    uint32_t units = 0;
+};
+
+enum { KERNEL_VEC = 0, KERNEL_BULK = 1 };
+
+struct LaunchPlan {
+    int kernel = KERNEL_VEC;
+    int width = 16;       // bytes per unit (vector kernel); chunk bytes (bulk kernel)
+    int phase = 0;
+    std::vector<LoweredPart> parts;
+    uint32_t units_per_proc = 0;
+    uint32_t uniform_units = 0;  // >0: every part has this many units
+    int lookup_shift = 0;
+    std::vector<uint16_t> lookup;  // unit >> lookup_shift -> index of the part holding that unit
+    int tile_procs = 1;
+    int threads = 256;
+    int64_t grid = 0;
+    size_t smem = 0;
+    int n_used = 0;
+    int used_dim[ISO_MAX_DIMS] = {0};
+    // byte offsets of this launch's tables inside the request's device blob
+    size_t parts_off = 0, lookup_off = 0;
+};
+
+struct Request {
+    Comm *comm = nullptr;
+    int kind = ISO_KIND_ALLTOALL;
+    int alg = ISO_ALG_COMBINING;
+    int fusion = 1;
+    int64_t bulk_threshold = 1024;
+    const unsigned char *send = nullptr;
+    unsigned char *recv = nullptr;
+    int s = 0;
+    std::vector<int64_t> len, sdispl, rdispl;
+    int64_t send_stride = 0, recv_stride = 0, inter_stride = 0;
+    std::vector<Part> parts;           // schedule in execution order
+    std::vector<LaunchPlan> launches;  // lowered schedule
+    Iso_stats stats{};
+    // device side (owned by iso_api.cu)
+    bool dirty = true;
+    void *d_blob = nullptr;
+    unsigned char *d_inter = nullptr;
+    int64_t d_inter_bytes = 0;
+    int *d_err = nullptr;
+    int *h_err = nullptr;
+    void *last_stream = nullptr;
+    bool started = false;
+};
+
+// Builds r.parts, r.inter_stride and the schedule statistics from r.comm, r.kind, r.alg,
+// r.fusion and the block layout.  Returns an ISO_* code.
+int build_schedule(Request &r);
+
+// Splits parts into aligned pieces, groups them into kernel launches and fills the launch
+// geometry.  `send_addr` / `recv_addr` / `inter_addr` are only used for their alignment.
+int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr_t inter_addr);
+
+// Checks the executed parts for hazards: every range inside its buffer, no write to the send
+// buffer, and within a phase no written range overlapping another written or any read range.
+int validate_schedule(const Request &r);
+
+}  // namespace iso

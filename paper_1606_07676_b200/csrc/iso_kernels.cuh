@@ -1,0 +1,315 @@
+// Device code of the isomorphic neighbourhood collectives (sm_100a).
+//
+// One launch applies a list of parts to every process (paper, Section V: in a round all
+// processes forward the same relative blocks): for process r and part t
+//     dst_buf[r] + dst_off_t .. + len_t  =  src_buf[r (-) shift_t] + src_off_t .. + len_t
+// Packing, "sending" and unpacking of a combined message are this single gather; nothing
+// is staged through memory in between (the zero-copy goal of Section III-C).
+//
+// Work decomposition shared by both kernels: a CTA owns a tile of consecutive processes.
+// The payload of one process in this launch is cut into units (vector kernel: `width`
+// bytes; bulk kernel: chunks of up to `width` bytes); unit u of tile-local process q has
+// the flat index q * units_per_proc + u, and consecutive threads take consecutive flat
+// indices, so a warp touches consecutive bytes of one part (or of neighbouring parts)
+// whatever the block size is.
+#pragma once
+
+#include <cstdint>
+
+#include "iso.h"
+
+namespace iso {
+
+struct FastDivDev {
+    uint32_t m, s1, s2, div;
+};
+
+struct alignas(16) PartDev {
+    long long src_off;     // byte offset inside a process's source buffer
+    long long dst_off;     // byte offset inside the own destination buffer
+    long long len;         // bytes
+    long long rank_delta;  // source rank = own rank + rank_delta (+ wrap corrections)
+    uint32_t first_unit;   // index of the part's first unit among the launch's units
+    uint32_t units;
+    uint8_t src_buf, dst_buf, nnz, pad0;
+    uint8_t dim[ISO_MAX_DIMS];  // index into the launch's used dimensions
+    int32_t c[ISO_MAX_DIMS];    // coordinate shift along that dimension
+    uint32_t pad1;
+};
+
+struct LaunchDev {
+    const PartDev *parts;
+    const uint16_t *lookup;  // unit >> lookup_shift -> part (unused when uniform_units > 0)
+    unsigned char *buf[3];   // send, recv, inter
+    long long buf_stride[3];
+    long long P;
+    int *err;                // device error flag (bulk kernel time-outs)
+    uint32_t nparts;
+    uint32_t units_per_proc;
+    uint32_t uniform_units;
+    uint32_t lookup_shift;
+    uint32_t width;          // bytes per unit / chunk
+    int tile_procs;
+    int n_used;
+    int mesh_mask;           // bit k set: used dimension k is not periodic
+    FastDivDev div_units;    // division by units_per_proc
+    FastDivDev div_uniform;  // division by uniform_units
+    int used_dim[ISO_MAX_DIMS];
+    uint32_t used_size[ISO_MAX_DIMS];       // p_j of the used dimensions
+    long long used_rstride[ISO_MAX_DIMS];   // ranks per step along the used dimensions
+};
+
+__device__ __forceinline__ uint32_t fastdiv(const FastDivDev &f, uint32_t n)
+{
+    uint32_t t = __umulhi(f.m, n);
+    return (t + ((n - t) >> f.s1)) >> f.s2;
+}
+
+// Coordinates (along the dimensions this launch shifts in) of the tile's processes.
+__device__ __forceinline__ void tile_coordinates(const LaunchDev &L, long long r0, int np, uint32_t *s_coord)
+{
+    for (int x = threadIdx.x; x < np * L.n_used; x += blockDim.x) {
+        int k = x / np, q = x - k * np;
+        unsigned long long r = (unsigned long long)(r0 + q);
+        s_coord[k * L.tile_procs + q] =
+            (uint32_t)((r / (unsigned long long)L.used_rstride[k]) % L.used_size[k]);
+    }
+}
+
+struct UnitAddr {
+    const unsigned char *src;
+    unsigned char *dst;
+    uint32_t bytes;  // bytes of this unit (bulk kernel: the last chunk of a part is shorter)
+    bool valid;      // false: the source lies outside a non-periodic dimension
+};
+
+// Decodes flat unit index `id` of the tile into addresses.
+__device__ __forceinline__ UnitAddr decode_unit(const LaunchDev &L, long long r0, uint32_t id,
+                                                const uint32_t *s_coord)
+{
+    const uint32_t q = fastdiv(L.div_units, id);
+    const uint32_t u = id - q * L.units_per_proc;
+    uint32_t t;
+    if (L.uniform_units) {
+        t = fastdiv(L.div_uniform, u);
+    } else {
+        t = L.lookup[u >> L.lookup_shift];
+        while (t + 1 < L.nparts && __ldg(&L.parts[t + 1].first_unit) <= u) ++t;
+    }
+    const PartDev *p = L.parts + t;
+    const uint32_t k = u - __ldg(&p->first_unit);
+    long long rs = r0 + q + __ldg(&p->rank_delta);
+    bool valid = true;
+    const int nnz = __ldg(&p->nnz);
+    for (int e = 0; e < nnz; ++e) {
+        const int dk = __ldg(&p->dim[e]);
+        const int c = __ldg(&p->c[e]);
+        const int x = (int)s_coord[dk * L.tile_procs + q];
+        if (L.mesh_mask >> dk & 1) {
+            const int y = x - c;
+            valid = valid && y >= 0 && y < (int)L.used_size[dk];
+        } else if (x < c) {
+            rs += (long long)L.used_size[dk] * L.used_rstride[dk];
+        }
+    }
+    const long long within = (long long)k * L.width;
+    const long long len = __ldg(&p->len);
+    UnitAddr a;
+    a.src = L.buf[__ldg(&p->src_buf)] + rs * L.buf_stride[__ldg(&p->src_buf)] + __ldg(&p->src_off) + within;
+    a.dst = L.buf[__ldg(&p->dst_buf)] + (r0 + q) * L.buf_stride[__ldg(&p->dst_buf)] + __ldg(&p->dst_off) + within;
+    const long long rest = len - within;
+    a.bytes = (uint32_t)(rest < (long long)L.width ? rest : (long long)L.width);
+    a.valid = valid;
+    return a;
+}
+
+template <int W> struct VecOf;
+template <> struct VecOf<16> { using type = uint4; };
+template <> struct VecOf<8> { using type = uint2; };
+template <> struct VecOf<4> { using type = uint32_t; };
+template <> struct VecOf<2> { using type = uint16_t; };
+template <> struct VecOf<1> { using type = uint8_t; };
+
+// Vector gather: one W-byte load and store per unit, UNROLL independent units per thread
+// in flight before the first store.
+template <int W, int UNROLL>
+__global__ void __launch_bounds__(256) iso_gather_vec(const __grid_constant__ LaunchDev L)
+{
+    using V = typename VecOf<W>::type;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint32_t *s_coord = reinterpret_cast<uint32_t *>(smem_raw);
+
+    const long long r0 = (long long)blockIdx.x * L.tile_procs;
+    const long long left = L.P - r0;
+    const int np = (int)(left < L.tile_procs ? left : L.tile_procs);
+    tile_coordinates(L, r0, np, s_coord);
+    __syncthreads();
+
+    const uint32_t total = (uint32_t)np * L.units_per_proc;
+    const uint32_t step = blockDim.x * UNROLL;
+    for (uint32_t base = threadIdx.x; base < total; base += step) {
+        V val[UNROLL];
+        V *dst[UNROLL];
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const uint32_t id = base + k * blockDim.x;
+            dst[k] = nullptr;
+            if (id < total) {
+                UnitAddr a = decode_unit(L, r0, id, s_coord);
+                if (a.valid) {
+                    dst[k] = reinterpret_cast<V *>(a.dst);
+                    val[k] = *reinterpret_cast<const V *>(a.src);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k)
+            if (dst[k]) *dst[k] = val[k];
+    }
+}
+
+// ---- asynchronous bulk copies (TMA, untiled form) ------------------------------------
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// global -> shared, completion reported on an mbarrier of this CTA
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(smem_dst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+// shared -> global, tracked by the thread's bulk async-group
+__device__ __forceinline__ void bulk_store(void *gdst, const void *smem_src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_addr(smem_src)),
+                 "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Upper bound on polls of one mbarrier before the kernel gives up and reports an error.
+constexpr uint32_t kBulkWaitPolls = 1u << 22;
+
+// Bulk gather for large parts: every thread drives its own two-stage pipeline of chunks,
+//   global --cp.async.bulk--> shared (mbarrier) --cp.async.bulk--> global (bulk group),
+// so that per thread one load and one store are in flight at any time and the data never
+// passes through registers.  All addresses and sizes are multiples of 16 bytes.
+__global__ void __launch_bounds__(256) iso_gather_bulk(const __grid_constant__ LaunchDev L)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t chunk = L.width;
+    unsigned char *s_data = smem_raw;                                                           // threads * 2 * chunk
+    uint64_t *s_bar = reinterpret_cast<uint64_t *>(smem_raw + (size_t)blockDim.x * 2 * chunk);  // threads * 2
+    uint32_t *s_coord =
+        reinterpret_cast<uint32_t *>(smem_raw + (size_t)blockDim.x * 2 * chunk + (size_t)blockDim.x * 16);
+
+    const long long r0 = (long long)blockIdx.x * L.tile_procs;
+    const long long left = L.P - r0;
+    const int np = (int)(left < L.tile_procs ? left : L.tile_procs);
+    tile_coordinates(L, r0, np, s_coord);
+    uint64_t *bar = s_bar + 2 * threadIdx.x;
+    unsigned char *stage = s_data + (size_t)threadIdx.x * 2 * chunk;
+    mbar_init(&bar[0], 1);
+    mbar_init(&bar[1], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+    __syncthreads();
+
+    const uint32_t total = (uint32_t)np * L.units_per_proc;
+    const uint32_t n = threadIdx.x < total ? (total - threadIdx.x + blockDim.x - 1) / blockDim.x : 0;
+    uint32_t parity_bits = 0;   // bit s: parity the next wait on stage s has to see
+    uint32_t pending_bits = 0;  // bit s: a load into stage s has been issued and not yet awaited
+    bool failed = false;
+
+    auto await = [&](uint32_t s) {
+        uint32_t polls = 0;
+        while (!mbar_try_wait(&bar[s], (parity_bits >> s) & 1u)) {
+            if (++polls >= kBulkWaitPolls) {
+                failed = true;
+                return;
+            }
+        }
+        parity_bits ^= 1u << s;
+        pending_bits &= ~(1u << s);
+    };
+
+    UnitAddr cur{}, nxt{};
+    if (n > 0) {
+        cur = decode_unit(L, r0, threadIdx.x, s_coord);
+        if (cur.valid) {
+            mbar_expect_tx(&bar[0], cur.bytes);
+            bulk_load(stage, cur.src, cur.bytes, &bar[0]);
+            pending_bits |= 1u;
+        }
+    }
+    for (uint32_t k = 0; k < n; ++k) {
+        const uint32_t s = k & 1u;
+        if (k + 1 < n) {
+            bulk_wait_read_all();  // the other stage was last read by the store of item k-1
+            nxt = decode_unit(L, r0, threadIdx.x + (k + 1) * blockDim.x, s_coord);
+            if (nxt.valid && !failed) {
+                mbar_expect_tx(&bar[s ^ 1u], nxt.bytes);
+                bulk_load(stage + (size_t)(s ^ 1u) * chunk, nxt.src, nxt.bytes, &bar[s ^ 1u]);
+                pending_bits |= 1u << (s ^ 1u);
+            }
+        }
+        if (cur.valid && !failed) {
+            await(s);
+            if (!failed) {
+                fence_async_smem();
+                bulk_store(cur.dst, stage + (size_t)s * chunk, cur.bytes);
+                bulk_commit();
+            }
+        }
+        cur = nxt;
+    }
+    // on the error path a load may still be in flight: give it one more bounded wait so that
+    // it does not land in shared memory that has been handed to another CTA
+    for (uint32_t s = 0; s < 2; ++s)
+        if (pending_bits >> s & 1u) {
+            bool keep = failed;
+            failed = false;
+            await(s);
+            failed = failed || keep;
+        }
+    bulk_wait_all();
+    if (failed) atomicExch(L.err, 1);
+}
+
+}  // namespace iso

@@ -1,0 +1,663 @@
+// Host-side schedule computation for the isomorphic neighbourhood collectives.
+//
+// The schedules are those of the paper "Message-Combining Algorithms for Isomorphic,
+// Sparse Collective Communication":
+//   * Section V    - message combining with direct communication along the dimensions:
+//                    per dimension the neighbours are bucketed by their coordinate, one
+//                    round per distinct non-zero coordinate, every block hops once per
+//                    dimension in which its coordinate is non-zero;
+//   * Algorithm 1  - the alternating buffer rule (receive into the user's receive buffer
+//                    when an odd number of hops remains, else into the intermediate
+//                    buffer) and the hop-by-hop torus schedule;
+//   * Section III-B- the prefix trie of the allgather: a block is routed once per
+//                    distinct prefix;
+//   * Listing 3    - the straightforward schedule, every block straight from its source.
+// Because all processes follow the same steps, a schedule is a process-independent list of
+// parts "copy len bytes from (buffer, offset) of the process at -shift to (buffer, offset)
+// of myself"; the kernels apply every part to every process.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <numeric>
+
+#include "iso_internal.h"
+
+namespace iso {
+
+FastDiv make_fastdiv(uint32_t d)
+{
+    FastDiv f;
+    f.div = d ? d : 1;
+    d = f.div;
+    uint32_t l = 0;
+    while (l < 32 && ((uint64_t)1 << l) < d) ++l;  // l = ceil(log2 d)
+    uint64_t two_l = (uint64_t)1 << l;
+    f.m = (uint32_t)((((two_l - d) << 32) / d) + 1);
+    f.s1 = l < 1 ? l : 1;
+    f.s2 = l > 0 ? l - 1 : 0;
+    return f;
+}
+
+namespace {
+
+int reduce_mod(int c, int p)
+{
+    int x = c % p;
+    return x < 0 ? x + p : x;
+}
+
+// representative of smallest magnitude, ties towards the positive one
+int symmetric_rep(int residue, int p) { return 2 * (int64_t)residue <= p ? residue : residue - p; }
+
+struct Geometry {
+    int d, s;
+    std::vector<int> red;  // s*d reduced coordinates
+    const int *at(int i) const { return red.data() + (size_t)i * d; }
+};
+
+// Order of the rounds inside one dimension: positive coordinates by increasing
+// magnitude, then negative ones by increasing magnitude (Algorithm 1 treats the positive
+// coordinates first); keys of fused dimension groups are compared coordinate by coordinate.
+struct RoundOrder {
+    const int *dims;
+    int j0, j1;
+    bool operator()(const std::vector<int> &a, const std::vector<int> &b) const
+    {
+        for (int j = j0; j < j1; ++j) {
+            int sa = symmetric_rep(a[j - j0], dims[j]), sb = symmetric_rep(b[j - j0], dims[j]);
+            if (sa == sb) continue;
+            bool na = sa < 0, nb = sb < 0;
+            if (na != nb) return nb;  // non-negative first
+            return std::abs(sa) < std::abs(sb);
+        }
+        return false;
+    }
+};
+
+struct Groups {
+    int n = 0;
+    int begin[ISO_MAX_DIMS + 1] = {0};
+};
+
+Groups make_groups(int d, int fusion)
+{
+    Groups g;
+    int width = fusion <= 1 ? 1 : fusion;
+    for (int j = 0; j < d; j += width) g.begin[g.n++] = j;
+    g.begin[g.n] = d;
+    return g;
+}
+
+bool group_nonzero(const int *v, int j0, int j1)
+{
+    for (int j = j0; j < j1; ++j)
+        if (v[j]) return true;
+    return false;
+}
+
+int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+void add_local_copy(Request &r, int slot, std::vector<Part> &out)
+{
+    Part p;
+    p.phase = 0;
+    p.round = -1;
+    p.slot = slot;
+    p.src_buf = ISO_BUF_SEND;
+    p.dst_buf = ISO_BUF_RECV;
+    p.src_off = r.sdispl[slot];
+    p.dst_off = r.rdispl[slot];
+    p.len = r.len[slot];
+    out.push_back(p);
+}
+
+// --------------------------------------------------------------------------------------
+// Listing 3, run as one pass: block i comes straight from the process at -C^i.
+int build_direct(Request &r, const Geometry &g)
+{
+    const Comm &c = *r.comm;
+    int locals = 0, parts = 0;
+    for (int i = 0; i < g.s; ++i) {
+        if (r.len[i] == 0) continue;
+        const int *v = g.at(i);
+        bool reachable = true, zero = true;
+        for (int j = 0; j < g.d; ++j) {
+            if (!c.periodic[j] && std::abs((int64_t)v[j]) >= c.dims[j]) reachable = false;
+            if (v[j]) zero = false;
+        }
+        if (!reachable) continue;  // mesh: the source lies outside for every process
+        Part p;
+        p.phase = 0;
+        p.round = i;
+        p.slot = i;
+        p.src_off = r.sdispl[i];
+        p.dst_off = r.rdispl[i];
+        p.len = r.len[i];
+        std::memcpy(p.shift, v, sizeof(int) * g.d);
+        r.parts.push_back(p);
+        if (zero) ++locals; else ++parts;
+    }
+    r.stats.rounds = g.s;
+    r.stats.max_rounds_per_dim = g.s;
+    r.stats.parts = parts;
+    r.stats.local_copies = locals;
+    r.inter_stride = 0;
+    return ISO_SUCCESS;
+}
+
+// Assigns intermediate-buffer offsets to the slots flagged in `needs`; an offset keeps the
+// misalignment (mod 16) of the slot's receive displacement so that copies between the two
+// buffers can use wide accesses.
+std::vector<int64_t> layout_inter(Request &r, const std::vector<char> &needs)
+{
+    std::vector<int64_t> off(needs.size(), -1);
+    int64_t cur = 0;
+    for (size_t i = 0; i < needs.size(); ++i) {
+        if (!needs[i]) continue;
+        int64_t mis = r.len[i] >= 16 ? (r.rdispl[i] & 15) : 0;
+        int64_t a = r.len[i] >= 16 ? 16 : (r.len[i] >= 8 ? 8 : (r.len[i] >= 4 ? 4 : 1));
+        cur = round_up(cur, a) + mis;
+        off[i] = cur;
+        cur += r.len[i];
+    }
+    r.inter_stride = round_up(cur, 16);
+    return off;
+}
+
+int64_t offset_in(const Request &r, int buf, int slot, const std::vector<int64_t> &inter_off)
+{
+    if (buf == ISO_BUF_SEND) return r.sdispl[slot];
+    if (buf == ISO_BUF_RECV) return r.rdispl[slot];
+    return inter_off[slot];
+}
+
+// One hop of slot i under the alternating rule of Algorithm 1.
+void emit_hop(Request &r, int phase, int round, int slot, const int *shift, int d,
+              std::vector<int> &remaining, std::vector<int> &cur_buf,
+              const std::vector<int64_t> &inter_off, std::vector<Part> &out)
+{
+    Part p;
+    p.phase = phase;
+    p.round = round;
+    p.slot = slot;
+    p.src_buf = cur_buf[slot];
+    p.dst_buf = (remaining[slot] & 1) ? ISO_BUF_RECV : ISO_BUF_INTER;
+    p.src_off = offset_in(r, p.src_buf, slot, inter_off);
+    p.dst_off = offset_in(r, p.dst_buf, slot, inter_off);
+    p.len = r.len[slot];
+    std::memcpy(p.shift, shift, sizeof(int) * d);
+    out.push_back(p);
+    remaining[slot] -= 1;
+    cur_buf[slot] = p.dst_buf;
+}
+
+// Section V all-to-all: dimensions (or groups of consecutive dimensions) one after the
+// other; inside a group one round per distinct non-zero projected coordinate vector.
+int build_combining_alltoall(Request &r, const Geometry &g)
+{
+    const Comm &c = *r.comm;
+    const Groups gr = make_groups(g.d, r.fusion);
+    std::vector<int> hops(g.s, 0);
+    for (int i = 0; i < g.s; ++i)
+        for (int k = 0; k < gr.n; ++k)
+            if (group_nonzero(g.at(i), gr.begin[k], gr.begin[k + 1])) ++hops[i];
+    std::vector<char> needs(g.s, 0);
+    for (int i = 0; i < g.s; ++i) needs[i] = r.len[i] > 0 && hops[i] >= 2;
+    std::vector<int64_t> inter_off = layout_inter(r, needs);
+
+    std::vector<int> remaining = hops, cur_buf(g.s, ISO_BUF_SEND);
+    int round = 0, phase = 0, nmax = 0, parts = 0, locals = 0;
+    std::vector<Part> locals_parts;
+    for (int i = 0; i < g.s; ++i)
+        if (r.len[i] > 0 && hops[i] == 0) { add_local_copy(r, i, locals_parts); ++locals; }
+
+    for (int k = 0; k < gr.n; ++k) {
+        const int j0 = gr.begin[k], j1 = gr.begin[k + 1];
+        // bucket the neighbours by their coordinates in this group
+        std::map<std::vector<int>, std::vector<int>, RoundOrder> buckets(RoundOrder{c.dims, j0, j1});
+        for (int i = 0; i < g.s; ++i) {
+            if (r.len[i] == 0 || !group_nonzero(g.at(i), j0, j1)) continue;
+            buckets[std::vector<int>(g.at(i) + j0, g.at(i) + j1)].push_back(i);
+        }
+        nmax = std::max<int>(nmax, (int)buckets.size());
+        const size_t group_begin = r.parts.size();
+        for (auto &b : buckets) {
+            int shift[ISO_MAX_DIMS] = {0};
+            for (int j = j0; j < j1; ++j) shift[j] = b.first[j - j0];
+            for (int i : b.second) {
+                emit_hop(r, phase, round, i, shift, g.d, remaining, cur_buf, inter_off, r.parts);
+                ++parts;
+            }
+            ++round;
+            if (r.fusion == 0) ++phase;
+        }
+        if (r.fusion != 0 && r.parts.size() > group_begin) {
+            // rounds of one group touch disjoint slots: run them together, in slot order
+            std::stable_sort(r.parts.begin() + group_begin, r.parts.end(),
+                             [](const Part &a, const Part &b) { return a.slot < b.slot; });
+            ++phase;
+        }
+    }
+    // blocks for the process itself: one local copy, together with the first phase
+    for (Part &p : locals_parts) p.phase = 0;
+    r.parts.insert(r.parts.begin(), locals_parts.begin(), locals_parts.end());
+    r.stats.rounds = round;
+    r.stats.max_rounds_per_dim = nmax;
+    r.stats.parts = parts;
+    r.stats.local_copies = locals;
+    return ISO_SUCCESS;
+}
+
+// Algorithm 1: hop-by-hop all-to-all between immediate torus neighbours.  Step h of the
+// positive half of dimension j forwards every block with c^i_j > h by one hop; the negative
+// half mirrors it.  A block is read from the send buffer only on its very first hop.
+int build_torus_alltoall(Request &r, const Geometry &g)
+{
+    const Comm &c = *r.comm;
+    std::vector<int> sym((size_t)g.s * g.d), hops(g.s, 0);
+    for (int i = 0; i < g.s; ++i)
+        for (int j = 0; j < g.d; ++j) {
+            sym[(size_t)i * g.d + j] = symmetric_rep(g.at(i)[j], c.dims[j]);
+            hops[i] += std::abs(sym[(size_t)i * g.d + j]);
+        }
+    std::vector<char> needs(g.s, 0);
+    for (int i = 0; i < g.s; ++i) needs[i] = r.len[i] > 0 && hops[i] >= 2;
+    std::vector<int64_t> inter_off = layout_inter(r, needs);
+    std::vector<int> remaining = hops, cur_buf(g.s, ISO_BUF_SEND);
+    int round = 0, nmax = 0, parts = 0, locals = 0;
+    std::vector<Part> locals_parts;
+    for (int i = 0; i < g.s; ++i)
+        if (r.len[i] > 0 && hops[i] == 0) { add_local_copy(r, i, locals_parts); ++locals; }
+    for (int j = 0; j < g.d; ++j) {
+        int per_dim = 0;
+        for (int sign = +1; sign >= -1; sign -= 2) {
+            int reach = 0;
+            for (int i = 0; i < g.s; ++i)
+                if (r.len[i] > 0) reach = std::max(reach, sign * sym[(size_t)i * g.d + j]);
+            for (int h = 0; h < reach; ++h) {
+                int shift[ISO_MAX_DIMS] = {0};
+                shift[j] = reduce_mod(sign, c.dims[j]);
+                for (int i = 0; i < g.s; ++i) {
+                    if (r.len[i] == 0 || sign * sym[(size_t)i * g.d + j] <= h) continue;
+                    emit_hop(r, round, round, i, shift, g.d, remaining, cur_buf, inter_off, r.parts);
+                    ++parts;
+                }
+                ++round;
+                ++per_dim;
+            }
+        }
+        nmax = std::max(nmax, per_dim);
+    }
+    for (Part &p : locals_parts) p.phase = 0;
+    r.parts.insert(r.parts.begin(), locals_parts.begin(), locals_parts.end());
+    r.stats.rounds = round;
+    r.stats.max_rounds_per_dim = nmax;
+    r.stats.parts = parts;
+    r.stats.local_copies = locals;
+    return ISO_SUCCESS;
+}
+
+// Section III-B / V allgather.  A trie node is a distinct prefix of the (reduced) offset
+// vectors; a node whose last coordinate group is non-zero is produced in the round of that
+// coordinate by reading its parent's storage one shift away; a zero edge forwards nothing
+// and shares the parent's storage.  A node is stored in the receive slot of the first
+// neighbour whose vector is the prefix padded with zeros, else in the intermediate buffer.
+int build_combining_allgather(Request &r, const Geometry &g)
+{
+    const Comm &c = *r.comm;
+    const Groups gr = make_groups(g.d, r.fusion);
+    const int64_t m = g.s ? r.len[0] : 0;
+    struct Store { int buf; int64_t off; };
+    std::map<std::vector<int>, int> first_with_vector;  // full vector -> smallest slot
+    for (int i = g.s - 1; i >= 0; --i)
+        first_with_vector[std::vector<int>(g.at(i), g.at(i) + g.d)] = i;
+
+    std::map<std::vector<int>, Store> storage;  // prefix -> where that block lives
+    storage[std::vector<int>()] = Store{ISO_BUF_SEND, 0};
+    int64_t inter_cur = 0;
+    int round = 0, phase = 0, nmax = 0, parts = 0, locals = 0;
+    std::vector<Part> locals_parts;
+    std::vector<char> served(g.s, 0);
+
+    if (m > 0)
+        for (int i = 0; i < g.s; ++i)
+            if (!group_nonzero(g.at(i), 0, g.d)) { add_local_copy(r, i, locals_parts); served[i] = 1; ++locals; }
+
+    for (int k = 0; k < gr.n && m > 0; ++k) {
+        const int j0 = gr.begin[k], j1 = gr.begin[k + 1];
+        // rounds of this group: distinct non-zero coordinate keys
+        std::map<std::vector<int>, int, RoundOrder> round_of(RoundOrder{c.dims, j0, j1});
+        for (int i = 0; i < g.s; ++i)
+            if (group_nonzero(g.at(i), j0, j1)) round_of[std::vector<int>(g.at(i) + j0, g.at(i) + j1)] = 0;
+        nmax = std::max<int>(nmax, (int)round_of.size());
+        for (auto &kv : round_of) kv.second = round++;
+        const size_t group_begin = r.parts.size();
+        for (int i = 0; i < g.s; ++i) {
+            std::vector<int> prefix(g.at(i), g.at(i) + j1), parent(g.at(i), g.at(i) + j0);
+            const Store src = storage.at(parent);
+            if (!group_nonzero(g.at(i), j0, j1)) {
+                storage.emplace(prefix, src);  // zero edge: nothing moves
+                continue;
+            }
+            int shift[ISO_MAX_DIMS] = {0};
+            for (int j = j0; j < j1; ++j) shift[j] = g.at(i)[j];
+            const int rnd = round_of.at(std::vector<int>(g.at(i) + j0, g.at(i) + j1));
+            auto emit = [&](int slot, Store dst) {
+                Part p;
+                p.phase = r.fusion == 0 ? rnd : phase;
+                p.round = rnd;
+                p.slot = slot;
+                p.src_buf = src.buf;
+                p.src_off = src.off;
+                p.dst_buf = dst.buf;
+                p.dst_off = dst.off;
+                p.len = m;
+                std::memcpy(p.shift, shift, sizeof(shift));
+                r.parts.push_back(p);
+                ++parts;
+            };
+            if (!storage.count(prefix)) {
+                // new trie node: choose its storage and produce it
+                std::vector<int> padded(prefix);
+                padded.resize(g.d, 0);
+                auto it = first_with_vector.find(padded);
+                Store dst;
+                int slot = -1;
+                if (it != first_with_vector.end()) {
+                    slot = it->second;
+                    dst = Store{ISO_BUF_RECV, r.rdispl[slot]};
+                    served[slot] = 1;
+                } else {
+                    dst = Store{ISO_BUF_INTER, inter_cur};
+                    inter_cur += round_up(m, 16);
+                }
+                storage.emplace(prefix, dst);
+                emit(slot, dst);
+            }
+            // a neighbour whose vector ends here but whose slot does not hold the node
+            // (a repeated vector) receives its own copy in the same round
+            if (!served[i] && !group_nonzero(g.at(i), j1, g.d)) {
+                emit(i, Store{ISO_BUF_RECV, r.rdispl[i]});
+                served[i] = 1;
+            }
+        }
+        if (r.fusion != 0 && r.parts.size() > group_begin) ++phase;
+    }
+    if (r.fusion == 0) {
+        // per-round launches: parts were emitted in slot order, bring them into round order
+        std::stable_sort(r.parts.begin(), r.parts.end(),
+                         [](const Part &a, const Part &b) { return a.phase < b.phase; });
+    }
+    for (Part &p : locals_parts) p.phase = 0;
+    r.parts.insert(r.parts.begin(), locals_parts.begin(), locals_parts.end());
+    r.inter_stride = inter_cur;
+    r.stats.rounds = round;
+    r.stats.max_rounds_per_dim = nmax;
+    r.stats.parts = parts;
+    r.stats.local_copies = locals;
+    return ISO_SUCCESS;
+}
+
+void compress_phases(std::vector<Part> &parts, int &phases)
+{
+    int next = -1, last = -1;
+    for (Part &p : parts) {
+        if (p.phase != last) { last = p.phase; ++next; }
+        p.phase = next;
+    }
+    phases = next + 1;
+}
+
+}  // namespace
+
+int build_schedule(Request &r)
+{
+    const Comm &c = *r.comm;
+    Geometry g;
+    g.d = c.d;
+    g.s = c.s;
+    g.red.resize((size_t)c.s * c.d);
+    bool mesh = false;
+    for (int j = 0; j < c.d; ++j) mesh |= !c.periodic[j];
+    for (int i = 0; i < c.s; ++i)
+        for (int j = 0; j < c.d; ++j) {
+            int v = c.coords[(size_t)i * c.d + j];
+            g.red[(size_t)i * c.d + j] = c.periodic[j] ? reduce_mod(v, c.dims[j]) : v;
+        }
+    if (mesh && r.alg != ISO_ALG_DIRECT) return ISO_ERR_ARG;
+    const bool gather = r.kind == ISO_KIND_ALLGATHER;
+    if (r.alg == ISO_ALG_TORUS && gather) return ISO_ERR_ARG;
+    if (r.alg != ISO_ALG_COMBINING && r.alg != ISO_ALG_DIRECT && r.alg != ISO_ALG_TORUS) return ISO_ERR_ARG;
+    if (r.fusion < 0) return ISO_ERR_ARG;
+
+    r.parts.clear();
+    r.inter_stride = 0;
+    Iso_stats st{};
+    r.stats = st;
+    int rc;
+    if (r.alg == ISO_ALG_DIRECT) rc = build_direct(r, g);
+    else if (r.alg == ISO_ALG_TORUS) rc = build_torus_alltoall(r, g);
+    else if (gather) rc = build_combining_allgather(r, g);
+    else rc = build_combining_alltoall(r, g);
+    if (rc != ISO_SUCCESS) return rc;
+
+    // phase numbers must be non-decreasing in execution order
+    std::stable_sort(r.parts.begin(), r.parts.end(),
+                     [](const Part &a, const Part &b) { return a.phase < b.phase; });
+    int phases = 0;
+    compress_phases(r.parts, phases);
+
+    int64_t payload = 0, moved = 0;
+    for (int i = 0; i < c.s; ++i) payload += r.len[i];
+    for (const Part &p : r.parts) moved += p.len;
+    r.stats.kind = r.kind;
+    r.stats.algorithm = r.alg;
+    r.stats.fusion_level = r.fusion;
+    r.stats.d = c.d;
+    r.stats.s = c.s;
+    r.stats.phases = phases;
+    r.stats.P = c.P;
+    r.stats.send_stride = r.send_stride;
+    r.stats.recv_stride = r.recv_stride;
+    r.stats.inter_stride = r.inter_stride;
+    r.stats.bytes_min = 2 * c.P * payload;
+    r.stats.bytes_moved = 2 * c.P * moved;
+    return validate_schedule(r);
+}
+
+int validate_schedule(const Request &r)
+{
+    struct Range { int64_t lo, hi; bool write; };
+    const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
+    size_t begin = 0;
+    while (begin < r.parts.size()) {
+        size_t end = begin;
+        while (end < r.parts.size() && r.parts[end].phase == r.parts[begin].phase) ++end;
+        std::vector<Range> ranges[3];
+        for (size_t k = begin; k < end; ++k) {
+            const Part &p = r.parts[k];
+            if (p.len <= 0 || p.src_off < 0 || p.dst_off < 0) return ISO_ERR_STATE;
+            if (p.src_buf < 0 || p.src_buf > 2 || p.dst_buf < 1 || p.dst_buf > 2) return ISO_ERR_STATE;
+            if (p.src_off + p.len > stride[p.src_buf] || p.dst_off + p.len > stride[p.dst_buf]) return ISO_ERR_STATE;
+            ranges[p.src_buf].push_back(Range{p.src_off, p.src_off + p.len, false});
+            ranges[p.dst_buf].push_back(Range{p.dst_off, p.dst_off + p.len, true});
+        }
+        for (auto &v : ranges) {
+            std::sort(v.begin(), v.end(), [](const Range &a, const Range &b) { return a.lo < b.lo; });
+            // a write may not overlap anything else; reads may overlap reads
+            int64_t write_hi = -1, any_hi = -1;
+            for (const Range &x : v) {
+                if (x.lo < write_hi) return ISO_ERR_OVERLAP;
+                if (x.write && x.lo < any_hi) return ISO_ERR_OVERLAP;
+                any_hi = std::max(any_hi, x.hi);
+                if (x.write) write_hi = std::max(write_hi, x.hi);
+            }
+        }
+        begin = end;
+    }
+    return ISO_SUCCESS;
+}
+
+// --------------------------------------------------------------------------------------
+// Lowering to kernel launches.
+namespace {
+
+int pow2_alignment(int64_t x)
+{
+    if (x == 0) return 16;
+    int a = 1;
+    while (a < 16 && (x & a) == 0) a <<= 1;
+    return a;
+}
+
+int common_alignment(std::initializer_list<int64_t> xs)
+{
+    int a = 16;
+    for (int64_t x : xs) a = std::min(a, pow2_alignment(x));
+    return a;
+}
+
+}  // namespace
+
+int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr_t inter_addr)
+{
+    const Comm &c = *r.comm;
+    const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
+    const int64_t addr[3] = {(int64_t)send_addr, (int64_t)recv_addr, (int64_t)inter_addr};
+    r.launches.clear();
+    int64_t bulk_bytes = 0;
+
+    size_t begin = 0;
+    while (begin < r.parts.size()) {
+        size_t end = begin;
+        while (end < r.parts.size() && r.parts[end].phase == r.parts[begin].phase) ++end;
+
+        // split every part into pieces that share one alignment class
+        struct Piece { Part p; int kernel; int width; };
+        std::vector<Piece> pieces;
+        for (size_t k = begin; k < end; ++k) {
+            const Part &p = r.parts[k];
+            const int base = common_alignment({stride[p.src_buf], stride[p.dst_buf], addr[p.src_buf], addr[p.dst_buf]});
+            auto push = [&](int64_t rel, int64_t len) {
+                if (len <= 0) return;
+                Piece q;
+                q.p = p;
+                q.p.src_off = p.src_off + rel;
+                q.p.dst_off = p.dst_off + rel;
+                q.p.len = len;
+                q.width = std::min(base, common_alignment({q.p.src_off, q.p.dst_off, len}));
+                q.kernel = (q.width == 16 && r.bulk_threshold > 0 && len >= r.bulk_threshold) ? KERNEL_BULK : KERNEL_VEC;
+                pieces.push_back(q);
+            };
+            const bool co_aligned = base == 16 && ((p.src_off - p.dst_off) & 15) == 0;
+            if (co_aligned && p.len >= 48 && ((p.src_off & 15) || (p.len & 15))) {
+                int64_t head = (16 - (p.src_off & 15)) & 15;
+                int64_t body = (p.len - head) / 16 * 16;
+                push(0, head);
+                push(head, body);
+                push(head + body, p.len - head - body);
+            } else {
+                push(0, p.len);
+            }
+        }
+
+        // one launch per (kernel, width) class, in a fixed order
+        for (int kernel = 0; kernel < 2; ++kernel) {
+            for (int width = 16; width >= 1; width >>= 1) {
+                std::vector<Piece> cls;
+                for (const Piece &q : pieces)
+                    if (q.kernel == kernel && q.width == width) cls.push_back(q);
+                const size_t max_parts = 60000;
+                for (size_t lo = 0; lo < cls.size(); lo += max_parts) {
+                    size_t hi = std::min(cls.size(), lo + max_parts);
+                    LaunchPlan L;
+                    L.kernel = kernel;
+                    L.phase = r.parts[begin].phase;
+                    int64_t unit = width;
+                    if (kernel == KERNEL_BULK) {
+                        int64_t min_len = INT64_MAX;
+                        for (size_t k = lo; k < hi; ++k) min_len = std::min(min_len, cls[k].p.len);
+                        unit = 256;
+                        while (unit * 2 <= min_len && unit < 2048) unit *= 2;
+                        const char *env = std::getenv("ISO_BULK_CHUNK");
+                        if (env) {
+                            int64_t v = std::atoll(env);
+                            if (v >= 16 && v <= 16384 && v % 16 == 0) unit = v;
+                        }
+                    }
+                    L.width = (int)unit;
+                    uint64_t units = 0;
+                    bool uniform = true;
+                    bool used[ISO_MAX_DIMS] = {false};
+                    for (size_t k = lo; k < hi; ++k) {
+                        LoweredPart lp;
+                        lp.p = cls[k].p;
+                        uint64_t n = (uint64_t)((lp.p.len + unit - 1) / unit);
+                        if (units + n > 0x7fffffffull) return ISO_ERR_COUNT;
+                        lp.first_unit = (uint32_t)units;
+                        lp.units = (uint32_t)n;
+                        units += n;
+                        if (!L.parts.empty() && L.parts[0].units != lp.units) uniform = false;
+                        for (int j = 0; j < c.d; ++j)
+                            if (lp.p.shift[j]) used[j] = true;
+                        L.parts.push_back(lp);
+                        if (kernel == KERNEL_BULK) bulk_bytes += lp.p.len;
+                    }
+                    L.units_per_proc = (uint32_t)units;
+                    L.uniform_units = uniform ? L.parts[0].units : 0;
+                    for (int j = 0; j < c.d; ++j)
+                        if (used[j]) L.used_dim[L.n_used++] = j;
+                    // coarse lookup: unit >> shift -> part
+                    if (!uniform) {
+                        int shift = 0;
+                        while ((units >> shift) + 1 > 16384) ++shift;
+                        L.lookup_shift = shift;
+                        size_t n = (size_t)(units >> shift) + 1;
+                        L.lookup.resize(n);
+                        size_t t = 0;
+                        for (size_t e = 0; e < n; ++e) {
+                            uint64_t u = (uint64_t)e << shift;
+                            while (t + 1 < L.parts.size() && L.parts[t + 1].first_unit <= u) ++t;
+                            L.lookup[e] = (uint16_t)t;
+                        }
+                    }
+                    // geometry
+                    const int64_t bytes_per_proc = (int64_t)units * (kernel == KERNEL_BULK ? unit : width);
+                    int64_t tp;
+                    if (kernel == KERNEL_VEC) {
+                        L.threads = 256;
+                        tp = std::max<int64_t>(1, 32768 / std::max<int64_t>(1, bytes_per_proc));
+                        tp = std::min<int64_t>(tp, 512);
+                        tp = std::min<int64_t>(tp, std::max<int64_t>(1, c.P / (148 * 8)));
+                    } else {
+                        int threads = (int)(196608 / (2 * unit)) / 32 * 32;
+                        L.threads = std::max(32, std::min(256, threads));
+                        tp = std::max<int64_t>(1, (8 * (int64_t)L.threads + (int64_t)units - 1) / (int64_t)units);
+                        tp = std::min<int64_t>(tp, 512);
+                        tp = std::min<int64_t>(tp, std::max<int64_t>(1, c.P / (148 * 2)));
+                    }
+                    while (tp > 1 && (uint64_t)tp * units > 0x7fffffffull) tp /= 2;
+                    const char *env_tp = std::getenv(kernel == KERNEL_VEC ? "ISO_VEC_TILE" : "ISO_BULK_TILE");
+                    if (env_tp) {
+                        int64_t v = std::atoll(env_tp);
+                        if (v >= 1 && v <= 512 && (uint64_t)v * units <= 0x7fffffffull) tp = v;
+                    }
+                    L.tile_procs = (int)tp;
+                    L.grid = (c.P + tp - 1) / tp;
+                    if (L.grid > 0x7fffffff) return ISO_ERR_DIMS;
+                    L.smem = (size_t)L.n_used * (size_t)tp * sizeof(uint32_t);
+                    if (kernel == KERNEL_BULK)
+                        L.smem = (L.smem + 15) / 16 * 16 + (size_t)L.threads * 2 * (size_t)unit + (size_t)L.threads * 2 * 8;
+                    r.launches.push_back(std::move(L));
+                }
+            }
+        }
+        begin = end;
+    }
+    r.stats.launches = (int)r.launches.size();
+    r.stats.bulk_bytes = 2 * c.P * bulk_bytes;
+    return ISO_SUCCESS;
+}
+
+}  // namespace iso

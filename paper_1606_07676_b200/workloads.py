@@ -247,5 +247,28 @@ def config(name: str, seed: int = DEFAULT_SEED) -> Workload:
     raise KeyError(name)
 
 
+def layout(w: Workload):
+    """(lens, send displacements, receive displacements, send stride, receive stride), in
+    bytes, of a workload's buffers under the interface's layout rules: regular blocks back
+    to back; irregular blocks packed, process stride rounded up to 16 bytes."""
+    s = w.s
+    if w.collective == "alltoall":
+        m = w.block_bytes
+        dd = np.arange(s, dtype=np.int64) * m
+        return np.full(s, m, np.int64), dd, dd, s * m, s * m
+    if w.collective == "allgather":
+        m = w.block_bytes
+        return np.full(s, m, np.int64), np.zeros(s, np.int64), np.arange(s, dtype=np.int64) * m, m, s * m
+    lens = np.asarray(w.lens, np.int64)
+    dd = packed_displacements(lens)
+    stride = (int(lens.sum()) + 15) // 16 * 16
+    return lens, dd, dd, stride, stride
+
+
+def send_buffer_np(w: Workload, send_stride: int) -> np.ndarray:
+    """Host copy of the seeded send buffers of a workload (uint8 [P, send_stride])."""
+    return payload_np(w.kind, w.seed, 0, 0, w.P * send_stride).reshape(w.P, send_stride).copy()
+
+
 CONFIG_NAMES = ("cfg1", "cfg2_alltoall", "cfg2_allgather", "cfg3_m4", "cfg3_m64", "cfg3_m512",
                 "cfg3_m4096", "cfg4", "cfg5")

@@ -1,0 +1,246 @@
+"""GPU parity: the CUDA library, called through its C-ABI binding, against the CPU oracle,
+bit for bit, on the same seeded inputs."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1606_07676_b200 import binding as iso
+from paper_1606_07676_b200 import workloads as wl
+from schedule_sim import POISON, layout, make_request, oracle_result, send_buffer_np
+
+pytestmark = pytest.mark.gpu
+
+COMB0, COMB1, COMB2, COMBD = ((iso.ISO_ALG_COMBINING, g) for g in (0, 1, 2, 8))
+DIRECT = (iso.ISO_ALG_DIRECT, 1)
+TORUS = (iso.ISO_ALG_TORUS, 1)
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("these tests need a CUDA device")
+    iso.load_library()          # no fallback: a missing library is an error
+    torch.cuda.set_device(0)
+    return torch
+
+
+class Run:
+    """A workload bound to device buffers; `result(alg, fusion)` runs it and returns the
+    receive buffers as a numpy array."""
+
+    def __init__(self, torch, w, stream=None):
+        self.torch, self.w = torch, w
+        lens, sd, rd, ss, rs = layout(w)
+        self.ss, self.rs = ss, rs
+        self.send_host = send_buffer_np(w, ss)
+        self.send = torch.from_numpy(self.send_host).cuda()
+        self.recv = torch.empty((w.P, rs), dtype=torch.uint8, device="cuda")
+        self.comm, self.req = make_request(w, self.send, self.recv)
+        self.stream = stream
+        st = iso.Iso_request_get_stats(self.req)
+        assert (st["send_stride"], st["recv_stride"]) == (ss, rs)
+
+    def result(self, alg, fusion, bulk=None):
+        iso.Iso_request_set_algorithm(self.req, alg, fusion)
+        if bulk is not None:
+            iso.Iso_request_set_bulk_threshold(self.req, bulk)
+        self.recv.fill_(POISON)
+        self.torch.cuda.synchronize()
+        iso.Iso_Start(self.req, self.stream)
+        iso.Iso_wait(self.req)
+        return self.recv.cpu().numpy()
+
+    def close(self):
+        iso.Iso_request_free(self.req)
+        iso.Iso_comm_free(self.comm)
+
+
+def check(torch, w, algs, bulk=None):
+    run = Run(torch, w)
+    try:
+        want = oracle_result(w, run.send_host)
+        for alg, fusion in algs:
+            got = run.result(alg, fusion, bulk)
+            bad = np.argwhere(got != want)
+            assert bad.size == 0, "alg %d fusion %d: first mismatch at (rank, byte) %s" % (alg, fusion, bad[0])
+    finally:
+        run.close()
+
+
+# ------------------------------------------------------------------- the five configs
+def test_cfg1(torch_cuda):
+    check(torch_cuda, wl.config("cfg1"), [COMB0, COMB1, COMB2, DIRECT, TORUS])
+
+
+def test_cfg2_alltoall(torch_cuda):
+    check(torch_cuda, wl.config("cfg2_alltoall"), [COMB0, COMB1, COMB2, COMBD, DIRECT, TORUS])
+
+
+def test_cfg2_allgather(torch_cuda):
+    check(torch_cuda, wl.config("cfg2_allgather"), [COMB0, COMB1, COMB2, COMBD, DIRECT])
+
+
+@pytest.mark.parametrize("m", [4, 64, 512])
+def test_cfg3(torch_cuda, m):
+    check(torch_cuda, wl.config("cfg3_m%d" % m), [COMB0, COMB1, COMBD, DIRECT, TORUS])
+
+
+def test_cfg3_512_bulk_kernel(torch_cuda):
+    # 512-byte blocks through the bulk-copy kernel as well (threshold lowered)
+    check(torch_cuda, wl.config("cfg3_m512"), [COMB1, DIRECT], bulk=512)
+
+
+def test_cfg4(torch_cuda):
+    check(torch_cuda, wl.config("cfg4"), [COMB0, COMB1, COMB2, DIRECT])
+
+
+def test_cfg5(torch_cuda):
+    w = wl.config("cfg5")
+    check(torch_cuda, w, [COMB0, COMB1, COMB2, DIRECT])
+    check(torch_cuda, w, [COMB1], bulk=0)
+
+
+def test_cfg3_4096_sampled(torch_cuda):
+    """Full size (3 x 6.4 GB on the device): outputs of sampled ranks, block by block."""
+    torch = torch_cuda
+    w = wl.config("cfg3_m4096")
+    m, s, P = 4096, w.s, w.P
+    stride = s * m
+    send = wl.payload_torch(w.kind, w.seed, 0, P * stride, "cuda")
+    recv = torch.empty(P * stride, dtype=torch.uint8, device="cuda")
+    comm, req = make_request(w, send, recv)
+    rng = np.random.default_rng(5)
+    ranks = sorted({0, 1, 255, 256, 257, 511, P - 1, P - 256, P - 257, *rng.integers(0, P, 24).tolist()})
+    try:
+        for alg, fusion in (COMB1, DIRECT):
+            iso.Iso_request_set_algorithm(req, alg, fusion)
+            recv.fill_(POISON)
+            iso.Iso_Start(req)
+            iso.Iso_wait(req)
+            st = iso.Iso_request_get_stats(req)
+            assert st["bulk_bytes"] == st["bytes_moved"]       # 4 KB blocks use the bulk kernel
+            for r in ranks:
+                got = recv[r * stride:(r + 1) * stride].cpu().numpy().reshape(s, m)
+                for i in range(s):
+                    q = oracle.source_rank(w.dims, r, w.offsets[i])
+                    want = wl.payload_np(w.kind, w.seed, 0, q * stride + i * m, m)
+                    assert np.array_equal(got[i], want), (alg, r, i)
+            # a property that holds at any size: the result is a permutation of the send
+            # blocks, so per-slot byte sums over all processes are preserved
+            a = send.view(P, s, m)[:, 3].to(torch.int64).sum().item()
+            b = recv.view(P, s, m)[:, 3].to(torch.int64).sum().item()
+            assert a == b
+    finally:
+        iso.Iso_request_free(req)
+        iso.Iso_comm_free(comm)
+        del send, recv
+        torch.cuda.empty_cache()
+
+
+# --------------------------------------------------------------------- edge cases
+def _tiny_cases():
+    rng = np.random.default_rng(99)
+    cases = []
+    for dims in [(1,), (2,), (7,), (3, 5), (2, 2, 3), (5, 1, 4), (3, 3, 3, 2)]:
+        d = len(dims)
+        for s in (1, 5, 11):
+            offs = rng.integers(-6, 7, size=(s, d)).astype(np.int32)
+            if s >= 5:
+                offs[1] = 0
+                offs[4] = offs[2]
+            cases.append(wl.Workload("t", "alltoall", dims, offs, int(rng.choice([1, 2, 4, 8, 12, 16, 48])), seed=len(cases)))
+            cases.append(wl.Workload("t", "allgather", dims, offs, int(rng.choice([1, 4, 16, 80])), seed=len(cases)))
+            lens = rng.choice([0, 1, 3, 4, 16, 52, 64, 100, 1024, 1040], size=s).astype(np.int64)
+            cases.append(wl.Workload("t", "alltoallv", dims, offs, 0, lens=lens, seed=len(cases)))
+    return cases
+
+
+def test_tiny_tori_and_odd_sizes(torch_cuda):
+    for w in _tiny_cases():
+        algs = [COMB0, COMB1, COMB2, DIRECT] + ([TORUS] if w.collective != "allgather" else [])
+        check(torch_cuda, w, algs)
+
+
+def test_ragged_tail_and_many_tiles(torch_cuda):
+    # P is not a multiple of any tile size; several CTAs and a partial last one
+    w = wl.Workload("ragged", "alltoall", (37, 53), wl.moore(2, 2), 48, seed=7)
+    check(torch_cuda, w, [COMB0, COMB1, DIRECT, TORUS])
+    w = wl.Workload("ragged", "alltoallv", (37, 53), wl.moore(2, 1), 0,
+                    lens=np.array([1024, 4, 2064, 16, 1040, 8, 3072, 64]), seed=8)
+    check(torch_cuda, w, [COMB0, COMB1, DIRECT])
+    check(torch_cuda, w, [COMB1, DIRECT], bulk=256)
+
+
+def test_paper_neighbourhoods(torch_cuda):
+    for offs, dims in [(wl.positive_octant(3, 3), (12, 10, 9)), (wl.shells(3, (3, 7)), (16, 15, 17)),
+                       (wl.moore(4, 1), (6, 5, 4, 7))]:
+        for coll in ("alltoall", "allgather"):
+            w = wl.Workload("nbh", coll, dims, offs, 16, seed=3)
+            check(torch_cuda, w, [COMB1, DIRECT] + ([TORUS] if coll == "alltoall" and len(offs) < 200 else []))
+
+
+def test_allgatherv_and_unaligned_receive_layout(torch_cuda):
+    torch = torch_cuda
+    dims, offs = (6, 7), wl.moore(2, 1)
+    P, s, m = 42, 8, 20
+    rd = np.array([3 + 29 * i for i in range(s)], dtype=np.int64)      # gaps, odd displacements
+    send_host = wl.payload_np("uint8", 1, 0, 0, P * 32).reshape(P, 32).copy()   # stride = 20 rounded up to 32
+    send = torch.from_numpy(send_host).cuda()
+    comm = iso.Iso_neighborhood_create(dims, offs)
+    recv = torch.full((P, 240), POISON, dtype=torch.uint8, device="cuda")
+    req = iso.Iso_neighbor_allgatherv_init(send, m, 1, recv, [m] * s, rd, 1, comm)
+    st = iso.Iso_request_get_stats(req)
+    assert (st["send_stride"], st["recv_stride"]) == (32, 240)
+    for alg, fusion in (COMB1, DIRECT):
+        iso.Iso_request_set_algorithm(req, alg, fusion)
+        recv.fill_(POISON)
+        iso.Iso_Start(req)
+        iso.Iso_wait(req)
+        got = recv.cpu().numpy()
+        blocks = oracle.allgather(dims, offs, m, np.ascontiguousarray(send_host[:, :m])).reshape(P, s, m)
+        want = np.full((P, 240), POISON, np.uint8)
+        for i in range(s):
+            want[:, rd[i]:rd[i] + m] = blocks[:, i]
+        assert np.array_equal(got, want)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+def test_mesh_direct(torch_cuda):
+    torch = torch_cuda
+    w = wl.Workload("mesh", "alltoall", (9, 11), wl.moore(2, 2), 16, seed=4)
+    run = Run(torch, w)
+    iso.Iso_comm_set_periodic(run.comm, [0, 0])
+    got = run.result(iso.ISO_ALG_DIRECT, 1).reshape(w.P, w.s, 16)
+    full = oracle_result(w, run.send_host).reshape(w.P, w.s, 16)
+    for r in range(w.P):
+        R = (r // 11, r % 11)
+        for i, C in enumerate(w.offsets):
+            inside = 0 <= R[0] - C[0] < 9 and 0 <= R[1] - C[1] < 11
+            want = full[r, i] if inside else np.full(16, POISON, np.uint8)
+            assert np.array_equal(got[r, i], want), (r, i)
+    run.close()
+
+
+def test_persistent_request_streams_and_host_buffers(torch_cuda):
+    torch = torch_cuda
+    w = wl.Workload("p", "alltoall", (16, 16, 8), wl.moore(3, 1), 64, kind="fp32", seed=12)
+    side = torch.cuda.Stream()
+    run = Run(torch, w, stream=side)
+    want = oracle_result(w, run.send_host)
+    for _ in range(3):                       # init once, start many times
+        assert np.array_equal(run.result(*COMB1), want)
+    # new contents in the same buffers
+    send2 = wl.payload_np(w.kind, 77, 0, 0, w.P * run.ss).reshape(w.P, run.ss).copy()
+    run.send.copy_(torch.from_numpy(send2))
+    torch.cuda.synchronize()
+    assert np.array_equal(run.result(*COMB1), oracle_result(w, send2))
+    # host buffers through the library's own copies
+    hs = torch.from_numpy(run.send_host).pin_memory()
+    hr = torch.empty((w.P, run.rs), dtype=torch.uint8).pin_memory()
+    hr.fill_(0)
+    iso.Iso_Start_host(run.req, hs, hr, side)
+    iso.Iso_wait(run.req)
+    assert np.array_equal(hr.numpy(), want)
+    run.close()

@@ -1,0 +1,299 @@
+"""Host-side tests of the C-ABI library: symbols, argument checking, and the schedule
+builder, whose exported parts are executed with numpy and compared with the CPU oracle.
+No GPU is needed: requests are created without buffers."""
+import ctypes
+import itertools
+import re
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import counters
+from paper_1606_07676_b200 import binding as iso
+from paper_1606_07676_b200 import workloads as wl
+from schedule_sim import POISON, layout, make_request, oracle_result, send_buffer_np, simulate
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+ALGS = [(iso.ISO_ALG_COMBINING, 0), (iso.ISO_ALG_COMBINING, 1), (iso.ISO_ALG_COMBINING, 2),
+        (iso.ISO_ALG_COMBINING, 8), (iso.ISO_ALG_DIRECT, 1), (iso.ISO_ALG_TORUS, 1)]
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "iso.h")).read()
+    declared = set(re.findall(r"\b(Iso_[A-Za-z_]+)\s*\(", header))
+    declared -= {"Iso_comm", "Iso_request"}
+    lib = iso.load_library()
+    assert declared == set(iso.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+    iso.Iso_selftest()
+
+
+def test_struct_layouts_match_header():
+    assert ctypes.sizeof(iso.Iso_stats) == 11 * 4 + 4 + 7 * 8
+    assert ctypes.sizeof(iso.Iso_part) == 8 * 4 + 3 * 8 + 8 * 4
+
+
+def _tiny_workloads():
+    rng = np.random.default_rng(2016)
+    out = []
+    for dims in [(1,), (2,), (5,), (3, 4), (2, 2, 3), (4, 1, 3), (3, 3, 3), (2, 3, 2, 2)]:
+        d = len(dims)
+        for s in (1, 4, 9):
+            offs = rng.integers(-4, 5, size=(s, d)).astype(np.int32)
+            if s >= 4:
+                offs[1] = 0              # message to oneself
+                offs[3] = offs[2]        # repeated neighbour
+            out.append(wl.Workload("tiny", "alltoall", dims, offs, int(rng.choice([1, 4, 8, 16, 24])), seed=int(rng.integers(1 << 30))))
+            out.append(wl.Workload("tiny", "allgather", dims, offs, int(rng.choice([2, 4, 16, 40])), seed=int(rng.integers(1 << 30))))
+            lens = rng.choice([0, 1, 4, 12, 16, 52, 64, 100], size=s)
+            out.append(wl.Workload("tiny", "alltoallv", dims, offs, 0, lens=lens.astype(np.int64), seed=int(rng.integers(1 << 30))))
+    return out
+
+
+@pytest.mark.parametrize("alg,fusion", ALGS)
+def test_schedules_reproduce_the_oracle_on_tiny_tori(alg, fusion):
+    n = 0
+    for w in _tiny_workloads():
+        if alg == iso.ISO_ALG_TORUS and w.collective == "allgather":
+            continue
+        comm, req = make_request(w)
+        try:
+            iso.Iso_request_set_algorithm(req, alg, fusion)
+            st = iso.Iso_request_get_stats(req)
+            lens, sd, rd, ss, rs = layout(w)
+            assert (st["send_stride"], st["recv_stride"]) == (ss, rs)
+            send = send_buffer_np(w, ss)
+            got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send)
+            want = oracle_result(w, send)
+            assert np.array_equal(got, want), (w.dims, w.collective, w.offsets.tolist())
+            n += 1
+        finally:
+            iso.Iso_request_free(req)
+            iso.Iso_comm_free(comm)
+    assert n > 40
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg3_m4"])
+@pytest.mark.parametrize("alg,fusion", ALGS)
+def test_schedules_on_paper_shaped_configs(name, alg, fusion):
+    w = wl.config(name)
+    if name == "cfg3_m4":
+        w = wl.Workload(name, "alltoall", (16, 12), w.offsets, 4, kind="uint8")
+    comm, req = make_request(w)
+    iso.Iso_request_set_algorithm(req, alg, fusion)
+    st = iso.Iso_request_get_stats(req)
+    send = send_buffer_np(w, st["send_stride"])
+    got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send)
+    assert np.array_equal(got, oracle_result(w, send))
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+@pytest.mark.parametrize("coll", ["alltoall", "allgather"])
+@pytest.mark.parametrize("nbh", ["moore3", "octant3", "shells", "fig1"])
+def test_paper_neighbourhoods_small_torus(coll, nbh):
+    offs = {"moore3": wl.moore(3, 1), "octant3": wl.positive_octant(3, 3), "shells": wl.shells(2, (1, 3)),
+            "fig1": np.array([(0, 0, 0), (0, 0, 1), (1, 0, 0), (1, 1, 0), (1, 1, 1), (3, 2, 0), (3, 3, 2),
+                              (4, 0, 1), (4, 0, 2), (4, 1, 1)], np.int32)}[nbh]
+    dims = (5, 4, 6) if offs.shape[1] == 3 else (9, 8)
+    w = wl.Workload(nbh, coll, dims, offs, 8)
+    comm, req = make_request(w)
+    for alg, fusion in ALGS:
+        if alg == iso.ISO_ALG_TORUS and coll == "allgather":
+            continue
+        iso.Iso_request_set_algorithm(req, alg, fusion)
+        st = iso.Iso_request_get_stats(req)
+        send = send_buffer_np(w, st["send_stride"])
+        got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send)
+        assert np.array_equal(got, oracle_result(w, send)), (alg, fusion)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+# ------------------------------------------------------------- statistics vs the paper
+@pytest.mark.parametrize("name", ["cfg1", "cfg2_alltoall", "cfg3_m64", "cfg4", "cfg5"])
+def test_alltoall_statistics_follow_section_v(name):
+    w = wl.config(name)
+    comm, req = make_request(w)
+    st = iso.Iso_request_get_stats(req)
+    d = w.d
+    assert st["rounds"] == counters.direct_rounds(w.offsets, d, w.dims)
+    assert st["parts"] == counters.direct_volume(w.offsets, d, w.dims)
+    assert st["max_rounds_per_dim"] == max(counters.direct_rounds_per_dim(w.offsets, d, w.dims))
+    assert st["rounds"] <= st["max_rounds_per_dim"] * d            # "at most N d rounds"
+    assert st["phases"] <= d
+    lens = layout(w)[0]
+    hops = counters.direct_hops(w.offsets, d, w.dims)
+    assert st["bytes_min"] == 2 * w.P * int(lens.sum())
+    assert st["bytes_moved"] == 2 * w.P * int(sum(int(l) * max(h, 1) for l, h in zip(lens, hops)))
+    # hop-by-hop schedule of Algorithm 1
+    iso.Iso_request_set_algorithm(req, iso.ISO_ALG_TORUS, 1)
+    st = iso.Iso_request_get_stats(req)
+    assert st["rounds"] == counters.torus_rounds(w.offsets, d, w.dims)
+    assert st["parts"] == counters.torus_volume(w.offsets, d, w.dims)
+    # straightforward schedule
+    iso.Iso_request_set_algorithm(req, iso.ISO_ALG_DIRECT, 1)
+    st = iso.Iso_request_get_stats(req)
+    assert st["rounds"] == w.s and st["bytes_moved"] == st["bytes_min"] and st["launches"] >= 1
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+def test_hand_worked_schedule_4x4():
+    # Moore r=1 on a 4x4 torus: rounds (0,+1)={5,6,7}, (0,-1)={0,1,2}, (1,+1)={2,4,7}, (1,-1)={0,3,5};
+    # hops = [2,1,2,1,1,2,1,2]; the first hop of a two-hop block lands in the intermediate
+    # buffer, the last hop of every block in the receive buffer (Algorithm 1's parity rule)
+    w = wl.Workload("hand", "alltoall", (4, 4), wl.moore(2, 1), 4)
+    comm, req = make_request(w)
+    iso.Iso_request_set_algorithm(req, iso.ISO_ALG_COMBINING, 0)
+    parts = iso.Iso_request_get_parts(req)
+    rounds = {}
+    for p in parts:
+        rounds.setdefault(p["round"], []).append(p)
+    assert sorted(rounds) == [0, 1, 2, 3]
+    assert [sorted(q["slot"] for q in rounds[k]) for k in range(4)] == [[5, 6, 7], [0, 1, 2], [2, 4, 7], [0, 3, 5]]
+    assert [rounds[k][0]["shift"][:2] for k in range(4)] == [[1, 0], [3, 0], [0, 1], [0, 3]]
+    hops = [sum(1 for p in parts if p["slot"] == i) for i in range(8)]
+    assert hops == [2, 1, 2, 1, 1, 2, 1, 2]
+    first = {}
+    for p in parts:
+        first.setdefault(p["slot"], p)
+    for i in range(8):
+        assert first[i]["src_buf"] == iso.ISO_BUF_SEND
+        assert first[i]["dst_buf"] == (iso.ISO_BUF_INTER if hops[i] == 2 else iso.ISO_BUF_RECV)
+    last = {p["slot"]: p for p in parts}
+    assert all(p["dst_buf"] == iso.ISO_BUF_RECV for p in last.values())
+    st = iso.Iso_request_get_stats(req)
+    assert (st["rounds"], st["parts"]) == (4, 12)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+def test_allgather_statistics_follow_the_trie():
+    for offs, dims in [(wl.moore(3, 1), (32, 32, 32)), (wl.positive_octant(3, 3), (16, 16, 16)),
+                       (np.array([(0, 0, 0), (0, 0, 1), (1, 0, 0), (1, 1, 0), (1, 1, 1), (3, 2, 0), (3, 3, 2),
+                                  (4, 0, 1), (4, 0, 2), (4, 1, 1)], np.int32), (8, 8, 8))]:
+        w = wl.Workload("ag", "allgather", dims, offs, 64)
+        comm, req = make_request(w)
+        st = iso.Iso_request_get_stats(req)
+        assert st["parts"] == counters.allgather_direct_volume(offs, 3, dims)
+        assert st["rounds"] == counters.direct_rounds(offs, 3, dims)
+        assert st["bytes_moved"] == 2 * w.P * 64 * (st["parts"] + st["local_copies"])
+        iso.Iso_request_free(req)
+        iso.Iso_comm_free(comm)
+    # Moore neighbourhoods need no intermediate storage: every padded prefix is a neighbour
+    w = wl.config("cfg2_allgather")
+    comm, req = make_request(w)
+    st = iso.Iso_request_get_stats(req)
+    assert (st["parts"], st["rounds"], st["inter_stride"]) == (26, 6, 0)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+def test_fused_levels_interpolate_between_combining_and_direct():
+    w = wl.config("cfg4")
+    comm, req = make_request(w)
+    moved = []
+    for g in (1, 2, 3, 5):
+        iso.Iso_request_set_algorithm(req, iso.ISO_ALG_COMBINING, g)
+        st = iso.Iso_request_get_stats(req)
+        moved.append(st["bytes_moved"])
+        assert st["phases"] == -(-5 // g)
+    assert moved == sorted(moved, reverse=True)
+    assert moved[-1] == st["bytes_min"]
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+def test_alignment_classes_and_bulk_selection():
+    # 4-byte aligned packed displacements: long blocks are split into a 16-byte aligned
+    # body (bulk kernel from 1 KB) and narrow head / tail pieces
+    w = wl.Workload("v", "alltoallv", (4, 4), wl.moore(2, 1), 0, lens=np.array([4, 1024, 16, 2048, 64, 4, 256, 1024]))
+    comm, req = make_request(w)
+    parts = iso.Iso_request_get_parts(req)
+    assert any(p["kernel"] == 1 for p in parts)
+    for p in parts:
+        assert p["src_off"] % p["width"] == 0 or p["kernel"] == 1
+        if p["kernel"] == 1:
+            assert p["src_off"] % 16 == 0 and p["dst_off"] % 16 == 0 and p["len"] % 16 == 0 and p["len"] >= 1024
+    st = iso.Iso_request_get_stats(req)
+    send = send_buffer_np(w, st["send_stride"])
+    assert np.array_equal(simulate(parts, w.dims, st, send), oracle_result(w, send))
+    iso.Iso_request_set_bulk_threshold(req, 0)
+    assert all(p["kernel"] == 0 for p in iso.Iso_request_get_parts(req))
+    assert iso.Iso_request_get_stats(req)["bulk_bytes"] == 0
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+def test_mesh_direct():
+    w = wl.Workload("mesh", "alltoall", (4, 5), wl.moore(2, 2), 4)
+    comm, req = make_request(w)
+    iso.Iso_comm_set_periodic(comm, [0, 1])
+    iso.Iso_request_set_algorithm(req, iso.ISO_ALG_DIRECT, 1)
+    st = iso.Iso_request_get_stats(req)
+    send = send_buffer_np(w, st["send_stride"])
+    got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send, periodic=[0, 1])
+    full = oracle_result(w, send).reshape(w.P, w.s, 4)
+    want = np.full_like(full, POISON)
+    for r in range(w.P):
+        r0 = r // 5
+        for i, C in enumerate(w.offsets):
+            if 0 <= r0 - C[0] < 4:
+                want[r, i] = full[r, i]
+    assert np.array_equal(got.reshape(w.P, w.s, 4), want)
+    with pytest.raises(iso.IsoError):
+        iso.Iso_request_set_algorithm(req, iso.ISO_ALG_COMBINING, 1)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+# ------------------------------------------------------------------------- error paths
+def _code(fn, *a):
+    with pytest.raises(iso.IsoError) as e:
+        fn(*a)
+    return e.value.code
+
+
+def test_argument_errors():
+    assert _code(iso.Iso_neighborhood_create, [0, 4], [[1, 0]]) == iso.ISO_ERR_DIMS
+    assert _code(iso.Iso_neighborhood_create, [2] * 9, [[0] * 9]) == iso.ISO_ERR_DIMS
+    assert _code(iso.Iso_neighborhood_create, [1 << 16, 1 << 16], [[1, 0]]) == iso.ISO_ERR_DIMS
+    comm = iso.Iso_neighborhood_create([4, 4], wl.moore(2, 1))
+    assert _code(iso.Iso_neighbor_alltoall_init, None, 2, 4, None, 4, 4, comm) == iso.ISO_ERR_COUNT
+    assert _code(iso.Iso_neighbor_alltoall_init, None, -1, 4, None, -1, 4, comm) == iso.ISO_ERR_ARG
+    assert _code(iso.Iso_neighbor_alltoall_init, 4096, 2, 4, None, 2, 4, comm) == iso.ISO_ERR_ARG
+    ok = [4] * 8
+    dd = [4 * i for i in range(8)]
+    assert _code(iso.Iso_neighbor_alltoallv_init, None, ok, dd, 1, None, ok, [0] * 8, 1, comm) == iso.ISO_ERR_OVERLAP
+    assert _code(iso.Iso_neighbor_alltoallv_init, None, ok, dd, 1, None, [8] * 8, dd, 1, comm) == iso.ISO_ERR_COUNT
+    assert _code(iso.Iso_neighbor_alltoallv_init, None, ok, [-4] + dd[1:], 1, None, ok, dd, 1, comm) == iso.ISO_ERR_ARG
+    # overlapping user buffers (addresses only; nothing is dereferenced at init)
+    assert _code(iso.Iso_neighbor_alltoall_init, 1 << 20, 4, 1, (1 << 20) + 64, 4, 1, comm) == iso.ISO_ERR_OVERLAP
+    req = iso.Iso_neighbor_alltoall_init(None, 4, 1, None, 1, 4, comm)     # 4 x 1 byte == 1 x 4 bytes
+    assert _code(iso.Iso_request_set_algorithm, req, 7, 1) == iso.ISO_ERR_ARG
+    assert _code(iso.Iso_request_set_algorithm, req, 0, -1) == iso.ISO_ERR_ARG
+    assert _code(iso.Iso_Start, req) == iso.ISO_ERR_STATE                   # no buffers bound
+    iso.Iso_wait(req)                                                       # nothing started: fine
+    iso.Iso_comm_free(comm)                                                 # the request keeps the comm alive
+    assert iso.Iso_request_get_stats(req)["s"] == 8
+    iso.Iso_request_free(req)
+    assert "overlap" in iso.Iso_error_string(iso.ISO_ERR_OVERLAP)
+
+
+def test_empty_neighbourhood_and_zero_sized_blocks():
+    comm = iso.Iso_neighborhood_create([3, 3], np.zeros((0, 2), np.int32))
+    req = iso.Iso_neighbor_alltoall_init(None, 4, 4, None, 4, 4, comm)
+    st = iso.Iso_request_get_stats(req)
+    assert (st["s"], st["parts"], st["launches"], st["bytes_moved"]) == (0, 0, 0, 0)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+    comm = iso.Iso_neighborhood_create([3, 3], wl.moore(2, 1))
+    req = iso.Iso_neighbor_alltoall_init(None, 0, 4, None, 0, 4, comm)
+    assert iso.Iso_request_get_stats(req)["launches"] == 0
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
