@@ -327,7 +327,7 @@ def run_ours(args):
 
         # ---- roofline of the dominant kernel ------------------------------------------
         launches = max(1, st["launches"])
-        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_vec<16,4>"
+        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_rows<16,4>"
         line["roofline"] = {
             "bound": "hbm", "kernel": kernel, "achieved": per_gpu, "peak": peak, "unit": "GB/s",
             "frac": per_gpu / peak, "peak_kind": "%s copy bandwidth" % peak_kind,

@@ -134,6 +134,10 @@ int materialise(Request &r)
         ISO_CUDA(cudaMalloc((void **)&r.d_inter, (size_t)inter_bytes));
         r.d_inter_bytes = inter_bytes;
     }
+    int device = 0, sms = 0;
+    ISO_CUDA(cudaGetDevice(&device));
+    ISO_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    r.sm_count = sms > 0 ? sms : r.sm_count;
     int rc = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
     if (rc != ISO_SUCCESS) return rc;
 
@@ -217,6 +221,8 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
     a.uniform_units = L.uniform_units;
     a.lookup_shift = (uint32_t)L.lookup_shift;
     a.width = (uint32_t)L.width;
+    a.chunk_units = L.chunk_units;
+    a.rows_per_pass = L.rows_per_pass;
     a.tile_procs = L.tile_procs;
     a.n_used = L.n_used;
     a.mesh_mask = 0;
@@ -229,6 +235,7 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
         a.used_dim[k] = j;
         a.used_size[k] = (uint32_t)c.dims[j];
         a.used_rstride[k] = c.rank_stride[j];
+        a.used_wrap[k] = (uint32_t)(c.dims[j] * c.rank_stride[j]);
         if (!c.periodic[j]) a.mesh_mask |= 1 << k;
     }
     return a;
@@ -243,11 +250,11 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream)
         iso_gather_bulk<<<grid, block, L.smem, stream>>>(a);
     } else {
         switch (L.width) {
-        case 16: iso_gather_vec<16, 4><<<grid, block, L.smem, stream>>>(a); break;
-        case 8: iso_gather_vec<8, 4><<<grid, block, L.smem, stream>>>(a); break;
-        case 4: iso_gather_vec<4, 4><<<grid, block, L.smem, stream>>>(a); break;
-        case 2: iso_gather_vec<2, 4><<<grid, block, L.smem, stream>>>(a); break;
-        default: iso_gather_vec<1, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 16: iso_gather_rows<16, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 8: iso_gather_rows<8, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 4: iso_gather_rows<4, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 2: iso_gather_rows<2, 4><<<grid, block, L.smem, stream>>>(a); break;
+        default: iso_gather_rows<1, 4><<<grid, block, L.smem, stream>>>(a); break;
         }
     }
     ISO_CUDA(cudaGetLastError());

@@ -62,6 +62,8 @@ struct LaunchPlan {
     uint32_t uniform_units = 0;  // >0: every part has this many units
     int lookup_shift = 0;
     std::vector<uint16_t> lookup;  // unit >> lookup_shift -> index of the part holding that unit
+    uint32_t chunk_units = 1;    // vector kernel: unit positions per row slot
+    uint32_t rows_per_pass = 1;  // vector kernel: rows a CTA handles at the same time
     int tile_procs = 1;
     int threads = 256;
     int64_t grid = 0;
@@ -95,6 +97,7 @@ struct Request {
     int *h_err = nullptr;
     void *last_stream = nullptr;
     bool started = false;
+    int sm_count = 148;  // replaced by the device's count when the request is materialised
 };
 
 // Builds r.parts, r.inter_stride and the schedule statistics from r.comm, r.kind, r.alg,

@@ -49,6 +49,8 @@ struct LaunchDev {
     uint32_t uniform_units;
     uint32_t lookup_shift;
     uint32_t width;          // bytes per unit / chunk
+    uint32_t chunk_units;    // vector kernel: unit positions owned by one row slot of a CTA
+    uint32_t rows_per_pass;  // vector kernel: rows a CTA works on at the same time
     int tile_procs;
     int n_used;
     int mesh_mask;           // bit k set: used dimension k is not periodic
@@ -57,6 +59,7 @@ struct LaunchDev {
     int used_dim[ISO_MAX_DIMS];
     uint32_t used_size[ISO_MAX_DIMS];       // p_j of the used dimensions
     long long used_rstride[ISO_MAX_DIMS];   // ranks per step along the used dimensions
+    uint32_t used_wrap[ISO_MAX_DIMS];       // p_j * rank stride: added when a shift wraps around
 };
 
 __device__ __forceinline__ uint32_t fastdiv(const FastDivDev &f, uint32_t n)
@@ -130,41 +133,94 @@ template <> struct VecOf<4> { using type = uint32_t; };
 template <> struct VecOf<2> { using type = uint16_t; };
 template <> struct VecOf<1> { using type = uint8_t; };
 
-// Vector gather: one W-byte load and store per unit, UNROLL independent units per thread
-// in flight before the first store.
+// Vector gather.  Thread t of a CTA owns one unit position (row slot g = t / chunk_units,
+// unit u = t % chunk_units) for the whole kernel: it resolves the part, the offsets and the
+// coordinate shifts of that unit once, then walks down the CTA's rows (processes) with
+// UNROLL independent W-byte loads in flight before the first store.  The per-row work is a
+// wrap test per shifted dimension and two address computations.  CTA b handles the rows
+// [P*b/grid, P*(b+1)/grid), so a grid sized to the machine stays balanced to one row.
 template <int W, int UNROLL>
-__global__ void __launch_bounds__(256) iso_gather_vec(const __grid_constant__ LaunchDev L)
+__global__ void __launch_bounds__(256) iso_gather_rows(const __grid_constant__ LaunchDev L)
 {
     using V = typename VecOf<W>::type;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    uint32_t *s_coord = reinterpret_cast<uint32_t *>(smem_raw);
+    uint32_t *s_coord = reinterpret_cast<uint32_t *>(smem_raw);  // [n_used][tile_procs]
 
-    const long long r0 = (long long)blockIdx.x * L.tile_procs;
-    const long long left = L.P - r0;
-    const int np = (int)(left < L.tile_procs ? left : L.tile_procs);
-    tile_coordinates(L, r0, np, s_coord);
-    __syncthreads();
+    const long long row_lo = (L.P * (long long)blockIdx.x) / (long long)gridDim.x;
+    const long long row_hi = (L.P * (long long)(blockIdx.x + 1)) / (long long)gridDim.x;
+    const uint32_t CU = L.chunk_units, G = L.rows_per_pass, U = L.units_per_proc;
+    const uint32_t g = threadIdx.x / CU;
+    const uint32_t ul = threadIdx.x - g * CU;
+    const int TP = L.tile_procs;
 
-    const uint32_t total = (uint32_t)np * L.units_per_proc;
-    const uint32_t step = blockDim.x * UNROLL;
-    for (uint32_t base = threadIdx.x; base < total; base += step) {
-        V val[UNROLL];
-        V *dst[UNROLL];
+    for (long long base = row_lo; base < row_hi; base += TP) {
+        const long long left = row_hi - base;
+        const int np = (int)(left < TP ? left : TP);
+        __syncthreads();
+        tile_coordinates(L, base, np, s_coord);
+        __syncthreads();
+        if (g >= G) continue;
+        for (uint32_t u = ul; u < U; u += CU) {
+            // ---- resolve this unit once ------------------------------------------------
+            uint32_t t;
+            if (L.uniform_units) {
+                t = fastdiv(L.div_uniform, u);
+            } else {
+                t = L.lookup[u >> L.lookup_shift];
+                while (t + 1 < L.nparts && __ldg(&L.parts[t + 1].first_unit) <= u) ++t;
+            }
+            const PartDev *p = L.parts + t;
+            const long long within = (long long)(u - __ldg(&p->first_unit)) * W;
+            const int sb = __ldg(&p->src_buf), db = __ldg(&p->dst_buf);
+            const long long stride_s = L.buf_stride[sb], stride_d = L.buf_stride[db];
+            const unsigned char *A = L.buf[sb] + __ldg(&p->rank_delta) * stride_s + __ldg(&p->src_off) + within;
+            unsigned char *B = L.buf[db] + __ldg(&p->dst_off) + within;
+            int c[ISO_MAX_DIMS];
 #pragma unroll
-        for (int k = 0; k < UNROLL; ++k) {
-            const uint32_t id = base + k * blockDim.x;
-            dst[k] = nullptr;
-            if (id < total) {
-                UnitAddr a = decode_unit(L, r0, id, s_coord);
-                if (a.valid) {
-                    dst[k] = reinterpret_cast<V *>(a.dst);
-                    val[k] = *reinterpret_cast<const V *>(a.src);
+            for (int e = 0; e < ISO_MAX_DIMS; ++e) c[e] = 0;
+            const int nnz = __ldg(&p->nnz);
+            for (int z = 0; z < nnz; ++z) {
+                const int dk = __ldg(&p->dim[z]);
+                const int cv = __ldg(&p->c[z]);
+#pragma unroll
+                for (int e = 0; e < ISO_MAX_DIMS; ++e)
+                    if (e == dk) c[e] = cv;
+            }
+            // ---- walk the rows ----------------------------------------------------------
+            for (int q0 = (int)g; q0 < np; q0 += (int)G * UNROLL) {
+                V val[UNROLL];
+                V *dst[UNROLL];
+#pragma unroll
+                for (int k = 0; k < UNROLL; ++k) {
+                    const int q = q0 + k * (int)G;
+                    dst[k] = nullptr;
+                    if (q < np) {
+                        uint32_t wrap = 0;
+                        bool valid = true;
+#pragma unroll
+                        for (int e = 0; e < ISO_MAX_DIMS; ++e) {
+                            if (e < L.n_used) {
+                                const int x = (int)s_coord[e * TP + q];
+                                if ((L.mesh_mask >> e) & 1) {
+                                    const int y = x - c[e];
+                                    valid = valid && y >= 0 && y < (int)L.used_size[e];
+                                } else if (x < c[e]) {
+                                    wrap += L.used_wrap[e];
+                                }
+                            }
+                        }
+                        if (valid) {
+                            const long long r = base + q;
+                            val[k] = *reinterpret_cast<const V *>(A + (r + wrap) * stride_s);
+                            dst[k] = reinterpret_cast<V *>(B + r * stride_d);
+                        }
+                    }
                 }
+#pragma unroll
+                for (int k = 0; k < UNROLL; ++k)
+                    if (dst[k]) *dst[k] = val[k];
             }
         }
-#pragma unroll
-        for (int k = 0; k < UNROLL; ++k)
-            if (dst[k]) *dst[k] = val[k];
     }
 }
 

@@ -623,28 +623,39 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         }
                     }
                     // geometry
-                    const int64_t bytes_per_proc = (int64_t)units * (kernel == KERNEL_BULK ? unit : width);
+                    (void)width;
                     int64_t tp;
+                    int64_t grid;
                     if (kernel == KERNEL_VEC) {
-                        L.threads = 256;
-                        tp = std::max<int64_t>(1, 32768 / std::max<int64_t>(1, bytes_per_proc));
-                        tp = std::min<int64_t>(tp, 512);
-                        tp = std::min<int64_t>(tp, std::max<int64_t>(1, c.P / (148 * 8)));
+                        // a row slot covers up to 256 unit positions; short rows share a CTA
+                        L.chunk_units = (uint32_t)std::min<uint64_t>(units, 256);
+                        L.rows_per_pass = std::max<uint32_t>(1, 256 / L.chunk_units);
+                        L.threads = (int)((L.chunk_units * L.rows_per_pass + 31) / 32 * 32);
+                        int per_sm = 4;
+                        if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
+                            int v = std::atoi(env);
+                            if (v >= 1 && v <= 8) per_sm = v;
+                        }
+                        // persistent grid: CTA b owns rows [P*b/grid, P*(b+1)/grid)
+                        grid = std::min<int64_t>((c.P + L.rows_per_pass - 1) / L.rows_per_pass,
+                                                 (int64_t)r.sm_count * per_sm);
+                        grid = std::max<int64_t>(grid, 1);
+                        tp = std::min<int64_t>(512, (c.P + grid - 1) / grid);
                     } else {
                         int threads = (int)(196608 / (2 * unit)) / 32 * 32;
                         L.threads = std::max(32, std::min(256, threads));
                         tp = std::max<int64_t>(1, (8 * (int64_t)L.threads + (int64_t)units - 1) / (int64_t)units);
                         tp = std::min<int64_t>(tp, 512);
                         tp = std::min<int64_t>(tp, std::max<int64_t>(1, c.P / (148 * 2)));
-                    }
-                    while (tp > 1 && (uint64_t)tp * units > 0x7fffffffull) tp /= 2;
-                    const char *env_tp = std::getenv(kernel == KERNEL_VEC ? "ISO_VEC_TILE" : "ISO_BULK_TILE");
-                    if (env_tp) {
-                        int64_t v = std::atoll(env_tp);
-                        if (v >= 1 && v <= 512 && (uint64_t)v * units <= 0x7fffffffull) tp = v;
+                        while (tp > 1 && (uint64_t)tp * units > 0x7fffffffull) tp /= 2;
+                        if (const char *env_tp = std::getenv("ISO_BULK_TILE")) {
+                            int64_t v = std::atoll(env_tp);
+                            if (v >= 1 && v <= 512 && (uint64_t)v * units <= 0x7fffffffull) tp = v;
+                        }
+                        grid = (c.P + tp - 1) / tp;
                     }
                     L.tile_procs = (int)tp;
-                    L.grid = (c.P + tp - 1) / tp;
+                    L.grid = grid;
                     if (L.grid > 0x7fffffff) return ISO_ERR_DIMS;
                     L.smem = (size_t)L.n_used * (size_t)tp * sizeof(uint32_t);
                     if (kernel == KERNEL_BULK)
