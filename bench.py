@@ -197,24 +197,80 @@ class Bound:
         self.iso.Iso_comm_free(self.comm)
 
 
+class Flush:
+    """Empties the L2 of anything useful: overwrites a buffer larger than the cache, then reads
+    a second one so that the cache is left full of clean, unrelated lines (a cache full of
+    dirty lines would charge their write-back to whatever runs next)."""
+
+    def __init__(self, torch):
+        self.a = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device="cuda")
+        self.b = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device="cuda")
+        self.sink = torch.zeros(1, dtype=torch.int64, device="cuda")
+
+    def __call__(self):
+        self.a.add_(1)
+        self.sink += self.b.sum()
+
+
 def time_steps(torch, fn, steps, warmup, flush):
-    """Per-step device times (ms) of `fn`, CUDA events on the current stream; between steps
-    the L2 is flushed by overwriting a buffer larger than it (outside the timed spans)."""
-    for _ in range(warmup):
+    """Per-step device times (ms) of `fn(k)`: one CUDA event pair per step on the current
+    stream, the L2 flushed between steps outside the timed spans."""
+    for k in range(warmup):
         if flush is not None:
-            flush.add_(1)
-        fn()
+            flush()
+        fn(k)
     torch.cuda.synchronize()
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     for k in range(steps):
         if flush is not None:
-            flush.add_(1)
+            flush()
         starts[k].record()
-        fn()
+        fn(k)
         ends[k].record()
     torch.cuda.synchronize()
     return [s.elapsed_time(e) for s, e in zip(starts, ends)]
+
+
+def time_run(torch, fn, steps, warmup):
+    """Device time (ms) per step of `steps` back-to-back calls fn(0..steps-1), one CUDA event
+    pair around the whole run on the current stream."""
+    for k in range(warmup):
+        fn(k)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for k in range(steps):
+        fn(k)
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / steps
+
+
+class Replicas:
+    """Independent instances of one workload (different seeds, own buffers and requests),
+    enough of them that a round-robin over the instances touches far more memory than the
+    L2 holds before an instance comes round again."""
+
+    def __init__(self, torch, iso, wl, name, min_bytes=4 * 126 * (1 << 20), max_replicas=16):
+        first = Bound(torch, iso, wl, name)
+        st = iso.Iso_request_get_stats(first.req)
+        foot = st["P"] * (st["send_stride"] + st["recv_stride"] + st["inter_stride"])
+        n = max(1, min(max_replicas, -(-min_bytes // max(1, foot))))
+        self.items = [first] + [Bound(torch, iso, wl, name, seed=first.w.seed + 1000 * k) for k in range(1, n)]
+        self.footprint = foot
+        self.iso, self.torch = iso, torch
+
+    def set(self, alg, fusion):
+        return [b.set(alg, fusion) for b in self.items][0]
+
+    def start(self, k):
+        b = self.items[k % len(self.items)]
+        self.iso.Iso_Start(b.req, self.torch.cuda.current_stream())
+
+    def close(self):
+        for b in self.items:
+            b.close()
 
 
 def cpu_baseline(w, seconds=10.0):
@@ -248,27 +304,22 @@ def run_ours(args):
     iso.load_library()
 
     peak, peak_kind = measured_peak()
-    flush = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.int32, device="cuda")
-    b = Bound(torch, iso, wl, args.workload)
-    stream = torch.cuda.current_stream()
-
-    def start():
-        iso.Iso_Start(b.req, stream)
+    reps = Replicas(torch, iso, wl, args.workload)
+    b = reps.items[0]
 
     # ---- headline: message-combining schedule, one launch per dimension ----------------
-    st = b.set(iso.ISO_ALG_COMBINING, args.fusion)
+    st = reps.set(iso.ISO_ALG_COMBINING, args.fusion)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(local) if rank == 0 else None
     t0 = time.time()
-    times = time_steps(torch, start, args.steps, args.warmup, flush)
+    ms = time_run(torch, reps.start, args.steps, args.warmup)
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     t1 = time.time()
     clocks = sampler.stop(t0, t1) if sampler else None
-    ms = sum(times) / len(times)
     if dist is not None:
         t = torch.tensor([ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -278,56 +329,66 @@ def run_ours(args):
     per_gpu = moved / (ms * 1e-3) / 1e9
 
     detail = {"combining": {"fusion_level": args.fusion, "rounds": st["rounds"], "launches": st["launches"],
-                            "bytes_moved": moved, "bytes_min": minimum, "ms_cold": ms,
-                            "ms_cold_median": tukey_median(times), "gbs_moved": per_gpu,
-                            "gbs_payload": minimum / (ms * 1e-3) / 1e9}}
+                            "bytes_moved": moved, "bytes_min": minimum, "ms": ms, "gbs_moved": per_gpu,
+                            "gbs_payload": minimum / (ms * 1e-3) / 1e9, "replicas": len(reps.items),
+                            "footprint_bytes_per_replica": reps.footprint}}
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.workload, "collective": b.w.collective, "dims": list(b.w.dims), "s": b.w.s,
-                   "P": b.w.P, "block_bytes": b.w.block_bytes or None, "schedule": "combining (Section V), fusion level %d" % args.fusion,
+                   "P": b.w.P, "block_bytes": b.w.block_bytes or None,
+                   "schedule": "combining (Section V), fusion level %d" % args.fusion,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": "flushed between steps (512 MiB overwrite, outside the timed spans)",
+                   "l2": "inputs larger than L2: steps rotate over %d independent instances of the workload "
+                         "(%.0f MB each, %.0f MB in all), timed back to back between one event pair"
+                         % (len(reps.items), reps.footprint / 1e6, reps.footprint * len(reps.items) / 1e6),
                    "bytes": "value = bytes read + written by the schedule / device time"},
         "gpu_launches": st["launches"] * args.steps,
         "frac_of_nominal_8TBs": per_gpu / NOMINAL_HBM_GBS,
     }
 
-    if rank == 0 and world == 1:
-        # warm (back to back, no flush) timing of the same schedule
-        warm = time_steps(torch, start, args.steps, args.warmup, None)
-        detail["combining"]["ms_warm"] = tukey_median(warm)
+    if rank == 0 and world == 1 and args.headline_only:
+        line["e2e"] = None
+        line["roofline"] = {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s",
+                            "frac": per_gpu / peak, "traffic": args.traffic, "peak_kind": "%s copy bandwidth" % peak_kind}
+    elif rank == 0 and world == 1:
+        flush = Flush(torch)
+        one = lambda k: reps.start(0)
+        # the same schedule on ONE instance: per-step events with an L2 flush in between
+        # (includes the event and launch latency of a lone step), and back to back (warm)
+        cold = time_steps(torch, one, min(args.steps, 50), 3, flush)
+        detail["combining"]["ms_single_flushed_median"] = tukey_median(cold)
+        detail["combining"]["ms_single_warm"] = time_run(torch, one, args.steps, 3)
         # per-round launches (the paper's schedule, one launch per round) and the direct kernel
         for key, alg, fusion in (("combining_per_round", iso.ISO_ALG_COMBINING, 0), ("direct", iso.ISO_ALG_DIRECT, 1)):
-            s2 = b.set(alg, fusion)
-            tt = time_steps(torch, start, args.steps, args.warmup, flush)
-            m2 = sum(tt) / len(tt)
-            detail[key] = {"launches": s2["launches"], "bytes_moved": s2["bytes_moved"], "ms_cold": m2,
+            s2 = reps.set(alg, fusion)
+            m2 = time_run(torch, reps.start, args.steps, args.warmup)
+            detail[key] = {"launches": s2["launches"], "bytes_moved": s2["bytes_moved"], "ms": m2,
                            "gbs_moved": s2["bytes_moved"] / (m2 * 1e-3) / 1e9,
                            "gbs_payload": s2["bytes_min"] / (m2 * 1e-3) / 1e9,
                            "frac_of_peak_moved": s2["bytes_moved"] / (m2 * 1e-3) / 1e9 / peak}
-        st = b.set(iso.ISO_ALG_COMBINING, args.fusion)
+        st = reps.set(iso.ISO_ALG_COMBINING, args.fusion)
 
         # ---- end to end: host buffers in, host buffers out, through the C-ABI -----------
         hs = torch.empty(b.w.P * b.ss, dtype=torch.uint8).pin_memory()
         hs.copy_(b.send.cpu())
         hr = torch.empty(b.w.P * b.rs, dtype=torch.uint8).pin_memory()
+        stream = torch.cuda.current_stream()
 
-        def start_host():
+        def start_host(k):
             iso.Iso_Start_host(b.req, hs, hr, stream)
 
         e2e_steps = max(3, min(args.steps, 20))
-        te = time_steps(torch, start_host, e2e_steps, 3, None)
-        me = sum(te) / len(te)
+        me = time_run(torch, start_host, e2e_steps, 3)
         line["e2e"] = {"value": moved / (me * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": me,
                        "h2d_bytes_per_step": int(hs.numel()), "d2h_bytes_per_step": int(hr.numel()),
                        "payload_gbs": minimum / (me * 1e-3) / 1e9}
 
         # ---- roofline of the dominant kernel ------------------------------------------
         launches = max(1, st["launches"])
-        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_rows<16,4>"
+        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_rows<16,8>"
         line["roofline"] = {
             "bound": "hbm", "kernel": kernel, "achieved": per_gpu, "peak": peak, "unit": "GB/s",
             "frac": per_gpu / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
@@ -337,17 +398,18 @@ def run_ours(args):
                     "launch gaps are inside the step time",
         }
         line["cpu_baseline"] = cpu_baseline(b.w, args.cpu_seconds)
-
-        if args.sweep:
-            detail["sweep"] = sweep(torch, iso, wl, flush, peak, args)
     elif rank == 0:
         line["e2e"] = None
         line["roofline"] = {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s",
                             "frac": per_gpu / peak, "traffic": None, "peak_kind": "%s copy bandwidth" % peak_kind}
 
+    reps.close()
+    del reps, b
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and args.sweep and not args.headline_only:
+        detail["sweep"] = sweep(torch, iso, wl, peak, args)
     line["clocks"] = clocks
     line["detail"] = detail
-    b.close()
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
@@ -355,29 +417,27 @@ def run_ours(args):
     return 0
 
 
-def sweep(torch, iso, wl, flush, peak, args):
-    """Every named workload, combining (fusion level 1) and direct: for the results table."""
+def sweep(torch, iso, wl, peak, args):
+    """Every named workload, combining (one launch per dimension, and per round) and direct:
+    the results table.  Same protocol as the headline (rotation over instances, back to back)."""
     out = {}
-    names = [n for n in wl.CONFIG_NAMES]
-    for name in names:
-        b = Bound(torch, iso, wl, name)
-        stream = torch.cuda.current_stream()
+    for name in wl.CONFIG_NAMES:
+        reps = Replicas(torch, iso, wl, name)
         row = {}
         for key, alg, fusion in (("combining", iso.ISO_ALG_COMBINING, 1), ("combining_per_round", iso.ISO_ALG_COMBINING, 0),
                                  ("direct", iso.ISO_ALG_DIRECT, 1)):
-            st = b.set(alg, fusion)
-            steps = 20 if st["bytes_moved"] < (4 << 30) else 5
-            tt = time_steps(torch, lambda: iso.Iso_Start(b.req, stream), steps, 3, flush)
-            tw = time_steps(torch, lambda: iso.Iso_Start(b.req, stream), steps, 3, None)
-            ms, msw = tukey_median(tt), tukey_median(tw)
+            st = reps.set(alg, fusion)
+            steps = 40 if st["bytes_moved"] < (4 << 30) else 6
+            ms = time_run(torch, reps.start, steps, 4)
             row[key] = {"rounds": st["rounds"], "launches": st["launches"], "bytes_moved": st["bytes_moved"],
-                        "bytes_min": st["bytes_min"], "bulk_bytes": st["bulk_bytes"], "ms_cold": ms, "ms_warm": msw,
+                        "bytes_min": st["bytes_min"], "bulk_bytes": st["bulk_bytes"], "ms": ms,
+                        "replicas": len(reps.items),
                         "gbs_moved": st["bytes_moved"] / ms / 1e6, "gbs_payload": st["bytes_min"] / ms / 1e6,
                         "frac_moved_of_peak": st["bytes_moved"] / ms / 1e6 / peak,
                         "frac_moved_of_8TBs": st["bytes_moved"] / ms / 1e6 / NOMINAL_HBM_GBS}
         out[name] = row
-        b.close()
-        del b
+        reps.close()
+        del reps
         torch.cuda.empty_cache()
     return out
 
@@ -392,6 +452,8 @@ def main():
     ap.add_argument("--fusion", type=int, default=1)
     ap.add_argument("--sweep", action="store_true", help="also time every named workload")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--headline-only", action="store_true",
+                    help="time the headline schedule only (short runs under a profiler)")
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture, if one is current")
     args = ap.parse_args()

@@ -73,6 +73,16 @@ enum {
     ISO_ALG_TORUS = 2      /* Section III, Algorithm 1: hop-by-hop between immediate neighbours */
 };
 
+/* Where the message-combining all-to-all keeps a block between two hops. */
+enum {
+    ISO_LAYOUT_PACKED = 0,      /* every non-final hop has its own place in the intermediate buffer,
+                                   places ordered by (writing phase, reading phase, neighbour) so that
+                                   a phase touches few contiguous regions; receive buffer written by
+                                   final hops only.  Intermediate buffer: sum_i (hops_i - 1) blocks */
+    ISO_LAYOUT_ALTERNATING = 1  /* Algorithm 1: the block alternates between its slot of the receive
+                                   buffer and its slot of an intermediate buffer "of the same size" */
+};
+
 enum { ISO_KIND_ALLTOALL = 0, ISO_KIND_ALLGATHER = 1, ISO_KIND_ALLTOALLV = 2 };
 enum { ISO_BUF_SEND = 0, ISO_BUF_RECV = 1, ISO_BUF_INTER = 2 };
 
@@ -194,6 +204,10 @@ int Iso_neighbor_allgatherv_init(const void *sendbuf, int sendcount, Iso_datatyp
  * are replaced by the next Iso_Start.  Errors: ISO_ERR_ARG.
  */
 int Iso_request_set_algorithm(Iso_request request, int alg, int fusion_level);
+
+/* Chooses the intermediate-storage layout (ISO_LAYOUT_*) of ISO_ALG_COMBINING all-to-all
+ * schedules; the hop-by-hop schedule always alternates as in Algorithm 1.  Default: packed. */
+int Iso_request_set_layout(Iso_request request, int layout);
 
 /* Parts of at least `bytes` bytes whose addresses and length are multiples of 16 are moved
  * by the bulk-copy kernel (asynchronous bulk copies staged through shared memory), the rest

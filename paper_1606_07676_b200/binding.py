@@ -17,6 +17,7 @@ ISO_MAX_DIMS = 8
 ISO_ALG_COMBINING, ISO_ALG_DIRECT, ISO_ALG_TORUS = 0, 1, 2
 ISO_KIND_ALLTOALL, ISO_KIND_ALLGATHER, ISO_KIND_ALLTOALLV = 0, 1, 2
 ISO_BUF_SEND, ISO_BUF_RECV, ISO_BUF_INTER = 0, 1, 2
+ISO_LAYOUT_PACKED, ISO_LAYOUT_ALTERNATING = 0, 1
 ISO_BYTE, ISO_INT32, ISO_FLOAT, ISO_DOUBLE = 1, 4, 4, 8
 (ISO_SUCCESS, ISO_ERR_ARG, ISO_ERR_DIMS, ISO_ERR_COUNT, ISO_ERR_ALIGN, ISO_ERR_NOMEM, ISO_ERR_CUDA,
  ISO_ERR_OVERLAP, ISO_ERR_STATE, ISO_ERR_TIMEOUT) = range(10)
@@ -28,7 +29,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), LIB_NAME)
 EXPORTS = (
     "Iso_neighborhood_create", "Iso_comm_free", "Iso_comm_set_periodic",
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
-    "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_bulk_threshold",
+    "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_bulk_threshold",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
     "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
@@ -88,6 +89,7 @@ def load_library() -> ctypes.CDLL:
         "Iso_neighbor_alltoallv_init": [vp, vp, vp, ci, vp, vp, vp, ci, vp, pp],
         "Iso_neighbor_allgatherv_init": [vp, ci, ci, vp, vp, vp, ci, vp, pp],
         "Iso_request_set_algorithm": [vp, ci, ci],
+        "Iso_request_set_layout": [vp, ci],
         "Iso_request_set_bulk_threshold": [vp, i64],
         "Iso_Start": [vp, vp],
         "Iso_Start_host": [vp, vp, vp, vp],
@@ -222,6 +224,10 @@ def Iso_neighbor_allgatherv_init(sendbuf, sendcount: int, sendtype: int, recvbuf
 
 def Iso_request_set_algorithm(request: int, alg: int, fusion_level: int = 1) -> None:
     _check(load_library().Iso_request_set_algorithm(request, alg, fusion_level), "Iso_request_set_algorithm")
+
+
+def Iso_request_set_layout(request: int, layout: int) -> None:
+    _check(load_library().Iso_request_set_layout(request, layout), "Iso_request_set_layout")
 
 
 def Iso_request_set_bulk_threshold(request: int, nbytes: int) -> None:

@@ -147,6 +147,8 @@ int materialise(Request &r)
         bytes += L.parts.size() * sizeof(PartDev);
         L.lookup_off = bytes;
         bytes += (L.lookup.size() * sizeof(uint16_t) + 15) / 16 * 16;
+        L.units_off = bytes;
+        if (L.kernel == KERNEL_VEC) bytes += (size_t)L.units_per_proc * sizeof(UnitDev);
     }
     std::vector<unsigned char> blob(bytes ? bytes : 16, 0);
     for (const LaunchPlan &L : r.launches) {
@@ -179,6 +181,23 @@ int materialise(Request &r)
         }
         if (!L.lookup.empty())
             std::memcpy(blob.data() + L.lookup_off, L.lookup.data(), L.lookup.size() * sizeof(uint16_t));
+        if (L.kernel == KERNEL_VEC) {
+            // one descriptor per unit position
+            const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
+            UnitDev *ud = reinterpret_cast<UnitDev *>(blob.data() + L.units_off);
+            for (size_t t = 0; t < L.parts.size(); ++t) {
+                const LoweredPart &lp = L.parts[t];
+                for (uint32_t k = 0; k < lp.units; ++k) {
+                    UnitDev u{};
+                    u.src_term = pd[t].rank_delta * stride[lp.p.src_buf] + lp.p.src_off + (int64_t)k * L.width;
+                    u.dst_term = lp.p.dst_off + (int64_t)k * L.width;
+                    for (int z = 0; z < pd[t].nnz; ++z) u.c[pd[t].dim[z]] = pd[t].c[z];
+                    u.src_buf = pd[t].src_buf;
+                    u.dst_buf = pd[t].dst_buf;
+                    ud[lp.first_unit + k] = u;
+                }
+            }
+        }
     }
     if (r.d_blob) cudaFree(r.d_blob);
     r.d_blob = nullptr;
@@ -195,7 +214,14 @@ int materialise(Request &r)
     // opt in to large dynamic shared memory once per kernel
     static bool attrs_set = false;
     if (!attrs_set) {
+        if (const char *env = std::getenv("ISO_L2_FETCH")) {
+            // experiment knob: granularity of L2 fills from device memory (a per-context limit)
+            ISO_CUDA(cudaDeviceSetLimit(cudaLimitMaxL2FetchGranularity, (size_t)std::atoi(env)));
+        }
         ISO_CUDA(cudaFuncSetAttribute(iso_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<16, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<8, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<4, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
         attrs_set = true;
     }
     r.dirty = false;
@@ -208,6 +234,7 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
     LaunchDev a{};
     a.parts = reinterpret_cast<const PartDev *>(static_cast<unsigned char *>(r.d_blob) + L.parts_off);
     a.lookup = reinterpret_cast<const uint16_t *>(static_cast<unsigned char *>(r.d_blob) + L.lookup_off);
+    a.units = reinterpret_cast<const UnitDev *>(static_cast<unsigned char *>(r.d_blob) + L.units_off);
     a.buf[ISO_BUF_SEND] = const_cast<unsigned char *>(r.send);
     a.buf[ISO_BUF_RECV] = r.recv;
     a.buf[ISO_BUF_INTER] = r.d_inter;
@@ -236,28 +263,50 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
         a.used_size[k] = (uint32_t)c.dims[j];
         a.used_rstride[k] = c.rank_stride[j];
         a.used_wrap[k] = (uint32_t)(c.dims[j] * c.rank_stride[j]);
+        f = make_fastdiv((uint32_t)c.rank_stride[j]);
+        a.div_rstride[k] = FastDivDev{f.m, f.s1, f.s2, f.div};
+        f = make_fastdiv((uint32_t)c.dims[j]);
+        a.div_size[k] = FastDivDev{f.m, f.s1, f.s2, f.div};
         if (!c.periodic[j]) a.mesh_mask |= 1 << k;
     }
     return a;
 }
 
-int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream)
+template <typename Kernel>
+cudaError_t launch_kernel(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, cudaStream_t stream, bool dependent)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)L.grid);
+    cfg.blockDim = dim3((unsigned)L.threads);
+    cfg.dynamicSmemBytes = L.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    // programmatic dependent launch: the kernel may start while its predecessor in the stream
+    // drains; it orders itself behind it with griddepcontrol.wait before touching data
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
+int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool dependent)
 {
     if (L.grid == 0 || L.units_per_proc == 0) return ISO_SUCCESS;
     LaunchDev a = make_launch_args(r, L);
-    dim3 grid((unsigned)L.grid), block((unsigned)L.threads);
+    cudaError_t e;
     if (L.kernel == KERNEL_BULK) {
-        iso_gather_bulk<<<grid, block, L.smem, stream>>>(a);
+        e = launch_kernel(iso_gather_bulk, L, a, stream, dependent);
     } else {
         switch (L.width) {
-        case 16: iso_gather_rows<16, 4><<<grid, block, L.smem, stream>>>(a); break;
-        case 8: iso_gather_rows<8, 4><<<grid, block, L.smem, stream>>>(a); break;
-        case 4: iso_gather_rows<4, 4><<<grid, block, L.smem, stream>>>(a); break;
-        case 2: iso_gather_rows<2, 4><<<grid, block, L.smem, stream>>>(a); break;
-        default: iso_gather_rows<1, 4><<<grid, block, L.smem, stream>>>(a); break;
+        case 16: e = launch_kernel(iso_gather_rows<16, kVecDepth>, L, a, stream, dependent); break;
+        case 8: e = launch_kernel(iso_gather_rows<8, kVecDepth>, L, a, stream, dependent); break;
+        case 4: e = launch_kernel(iso_gather_rows<4, kVecDepth>, L, a, stream, dependent); break;
+        case 2: e = launch_kernel(iso_gather_rows_reg<2, 4>, L, a, stream, dependent); break;
+        default: e = launch_kernel(iso_gather_rows_reg<1, 4>, L, a, stream, dependent); break;
         }
     }
-    ISO_CUDA(cudaGetLastError());
+    ISO_CUDA(e);
     return ISO_SUCCESS;
 }
 
@@ -431,6 +480,13 @@ int Iso_request_set_algorithm(Iso_request request, int alg, int fusion_level)
     return rc;
 }
 
+int Iso_request_set_layout(Iso_request request, int layout)
+{
+    if (check_handle(request) || (layout != ISO_LAYOUT_PACKED && layout != ISO_LAYOUT_ALTERNATING)) return ISO_ERR_ARG;
+    request->layout = layout;
+    return Iso_request_set_algorithm(request, request->alg, request->fusion);
+}
+
 int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
 {
     if (check_handle(request) || bytes < 0) return ISO_ERR_ARG;
@@ -458,8 +514,9 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         if (rc != ISO_SUCCESS) return rc;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    static const bool use_pdl = !(std::getenv("ISO_NO_PDL") && std::atoi(std::getenv("ISO_NO_PDL")) != 0);
     for (const LaunchPlan &L : r.launches) {
-        int rc = launch_one(r, L, stream);
+        int rc = launch_one(r, L, stream, use_pdl);
         if (rc != ISO_SUCCESS) return rc;
     }
     r.last_stream = cuda_stream;

@@ -52,6 +52,8 @@ struct LoweredPart {
 };
 
 enum { KERNEL_VEC = 0, KERNEL_BULK = 1 };
+constexpr int kMaxVecUnits = 4096;  // unit positions per process in one vector launch
+constexpr int kVecDepth = 8;        // cp.async ring slots per thread in the vector kernel
 
 struct LaunchPlan {
     int kernel = KERNEL_VEC;
@@ -71,7 +73,7 @@ struct LaunchPlan {
     int n_used = 0;
     int used_dim[ISO_MAX_DIMS] = {0};
     // byte offsets of this launch's tables inside the request's device blob
-    size_t parts_off = 0, lookup_off = 0;
+    size_t parts_off = 0, lookup_off = 0, units_off = 0;
 };
 
 struct Request {
@@ -80,6 +82,7 @@ struct Request {
     int alg = ISO_ALG_COMBINING;
     int fusion = 1;
     int64_t bulk_threshold = 1024;
+    int layout = ISO_LAYOUT_PACKED;
     const unsigned char *send = nullptr;
     unsigned char *recv = nullptr;
     int s = 0;

@@ -37,8 +37,18 @@ struct alignas(16) PartDev {
     uint32_t pad1;
 };
 
+// Everything the vector kernel needs to know about one unit position of a process's payload.
+struct alignas(16) UnitDev {
+    long long src_term;  // rank_delta * source stride + source offset of the unit (bytes)
+    long long dst_term;  // destination offset of the unit (bytes)
+    int32_t c[ISO_MAX_DIMS];  // coordinate shift along each used dimension (0: none)
+    uint8_t src_buf, dst_buf;
+    uint8_t pad[14];
+};
+
 struct LaunchDev {
     const PartDev *parts;
+    const UnitDev *units;    // vector kernel: one entry per unit position
     const uint16_t *lookup;  // unit >> lookup_shift -> part (unused when uniform_units > 0)
     unsigned char *buf[3];   // send, recv, inter
     long long buf_stride[3];
@@ -60,6 +70,8 @@ struct LaunchDev {
     uint32_t used_size[ISO_MAX_DIMS];       // p_j of the used dimensions
     long long used_rstride[ISO_MAX_DIMS];   // ranks per step along the used dimensions
     uint32_t used_wrap[ISO_MAX_DIMS];       // p_j * rank stride: added when a shift wraps around
+    FastDivDev div_rstride[ISO_MAX_DIMS];   // division by the rank stride of a used dimension
+    FastDivDev div_size[ISO_MAX_DIMS];      // division by the size of a used dimension
 };
 
 __device__ __forceinline__ uint32_t fastdiv(const FastDivDev &f, uint32_t n)
@@ -71,12 +83,12 @@ __device__ __forceinline__ uint32_t fastdiv(const FastDivDev &f, uint32_t n)
 // Coordinates (along the dimensions this launch shifts in) of the tile's processes.
 __device__ __forceinline__ void tile_coordinates(const LaunchDev &L, long long r0, int np, uint32_t *s_coord)
 {
-    for (int x = threadIdx.x; x < np * L.n_used; x += blockDim.x) {
-        int k = x / np, q = x - k * np;
-        unsigned long long r = (unsigned long long)(r0 + q);
-        s_coord[k * L.tile_procs + q] =
-            (uint32_t)((r / (unsigned long long)L.used_rstride[k]) % L.used_size[k]);
-    }
+    // ranks are below 2^31, so the exact 32-bit division applies
+    for (int k = 0; k < L.n_used; ++k)
+        for (int q = threadIdx.x; q < np; q += blockDim.x) {
+            const uint32_t x = fastdiv(L.div_rstride[k], (uint32_t)(r0 + q));
+            s_coord[k * L.tile_procs + q] = x - fastdiv(L.div_size[k], x) * L.used_size[k];
+        }
 }
 
 struct UnitAddr {
@@ -133,25 +145,106 @@ template <> struct VecOf<4> { using type = uint32_t; };
 template <> struct VecOf<2> { using type = uint16_t; };
 template <> struct VecOf<1> { using type = uint8_t; };
 
+// Programmatic dependent launch: `grid_dependency_wait` blocks until the preceding kernel
+// in the stream has completed and its writes are visible; everything before it (tables,
+// coordinates) overlaps with that kernel's tail.  Both are no-ops for ordinary launches.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <int W> __device__ __forceinline__ void cp_async(void *smem_dst, const void *gsrc);
+template <> __device__ __forceinline__ void cp_async<16>(void *smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+template <> __device__ __forceinline__ void cp_async<8>(void *smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+template <> __device__ __forceinline__ void cp_async<4>(void *smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// What a thread keeps about the unit position it owns.
+struct UnitRegs {
+    const unsigned char *A;  // source base: buffer + src_term
+    unsigned char *B;        // destination base: buffer + dst_term
+    long long stride_s, stride_d;
+    int c[ISO_MAX_DIMS];
+};
+
+__device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
+{
+    const uint4 *raw = reinterpret_cast<const uint4 *>(L.units + u);
+    const uint4 a = __ldg(raw), b = __ldg(raw + 1), c = __ldg(raw + 2), d = __ldg(raw + 3);
+    UnitRegs R;
+    const long long src_term = (long long)(((unsigned long long)a.y << 32) | a.x);
+    const long long dst_term = (long long)(((unsigned long long)a.w << 32) | a.z);
+    const int sb = d.x & 0xff, db = (d.x >> 8) & 0xff;
+    R.A = L.buf[sb] + src_term;
+    R.B = L.buf[db] + dst_term;
+    R.stride_s = L.buf_stride[sb];
+    R.stride_d = L.buf_stride[db];
+    R.c[0] = (int)b.x; R.c[1] = (int)b.y; R.c[2] = (int)b.z; R.c[3] = (int)b.w;
+    R.c[4] = (int)c.x; R.c[5] = (int)c.y; R.c[6] = (int)c.z; R.c[7] = (int)c.w;
+    return R;
+}
+
+// Source address of the unit for tile-local row q (rank base + q); false if the source lies
+// outside a non-periodic dimension.
+__device__ __forceinline__ bool row_source(const LaunchDev &L, const UnitRegs &R, const uint32_t *s_coord, int TP,
+                                           long long base, int q, const unsigned char *&src)
+{
+    uint32_t wrap = 0;
+    bool valid = true;
+#pragma unroll
+    for (int e = 0; e < ISO_MAX_DIMS; ++e) {
+        if (e < L.n_used) {
+            const int x = (int)s_coord[e * TP + q];
+            if ((L.mesh_mask >> e) & 1) {
+                const int y = x - R.c[e];
+                valid = valid && y >= 0 && y < (int)L.used_size[e];
+            } else if (x < R.c[e]) {
+                wrap += L.used_wrap[e];
+            }
+        }
+    }
+    src = R.A + (base + q + wrap) * R.stride_s;
+    return valid;
+}
+
 // Vector gather.  Thread t of a CTA owns one unit position (row slot g = t / chunk_units,
-// unit u = t % chunk_units) for the whole kernel: it resolves the part, the offsets and the
-// coordinate shifts of that unit once, then walks down the CTA's rows (processes) with
-// UNROLL independent W-byte loads in flight before the first store.  The per-row work is a
-// wrap test per shifted dimension and two address computations.  CTA b handles the rows
-// [P*b/grid, P*(b+1)/grid), so a grid sized to the machine stays balanced to one row.
-template <int W, int UNROLL>
+// unit u = t % chunk_units): it loads that unit's descriptor once and then walks down the
+// CTA's rows (processes).  CTA b handles the rows [P*b/grid, P*(b+1)/grid), so a grid sized
+// to the machine stays balanced to one row.  Per row the work is a wrap test per shifted
+// dimension and two address computations.
+//
+// Data path for W in {16, 8, 4}: cp.async from global memory into a thread-private ring of
+// DEPTH slots in shared memory, so that DEPTH loads per thread are in flight without
+// holding registers; a slot is read back and stored to its destination as soon as the
+// oldest group has landed, and refilled with the load of DEPTH rows ahead.
+template <int W, int DEPTH>
 __global__ void __launch_bounds__(256) iso_gather_rows(const __grid_constant__ LaunchDev L)
 {
     using V = typename VecOf<W>::type;
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int TP = L.tile_procs;
     uint32_t *s_coord = reinterpret_cast<uint32_t *>(smem_raw);  // [n_used][tile_procs]
+    const uint32_t coord_bytes = ((uint32_t)L.n_used * (uint32_t)TP * 4u + 15u) & ~15u;
+    V *ring = reinterpret_cast<V *>(smem_raw + coord_bytes) + threadIdx.x;  // slot k at ring[k * blockDim.x]
 
     const long long row_lo = (L.P * (long long)blockIdx.x) / (long long)gridDim.x;
     const long long row_hi = (L.P * (long long)(blockIdx.x + 1)) / (long long)gridDim.x;
     const uint32_t CU = L.chunk_units, G = L.rows_per_pass, U = L.units_per_proc;
     const uint32_t g = threadIdx.x / CU;
     const uint32_t ul = threadIdx.x - g * CU;
-    const int TP = L.tile_procs;
+    const bool mesh = L.mesh_mask != 0;
+    bool first = true;
 
     for (long long base = row_lo; base < row_hi; base += TP) {
         const long long left = row_hi - base;
@@ -159,34 +252,87 @@ __global__ void __launch_bounds__(256) iso_gather_rows(const __grid_constant__ L
         __syncthreads();
         tile_coordinates(L, base, np, s_coord);
         __syncthreads();
+        if (first) {
+            grid_dependency_wait();
+            grid_launch_dependents();
+            first = false;
+        }
+        if (g >= G || (int)g >= np) continue;
+        const int nrows = (np - (int)g + (int)G - 1) / (int)G;  // rows g, g+G, ...
+        for (uint32_t u = ul; u < U; u += CU) {
+            const UnitRegs R = load_unit(L, u);
+            uint32_t valid_bits = 0;
+#pragma unroll
+            for (int i = 0; i < DEPTH; ++i) {
+                if (i < nrows) {
+                    const unsigned char *src;
+                    if (row_source(L, R, s_coord, TP, base, (int)g + i * (int)G, src)) {
+                        cp_async<W>(ring + i * blockDim.x, src);
+                        valid_bits |= 1u << i;
+                    }
+                }
+                cp_async_commit();
+            }
+            int slot = 0;
+            for (int i = 0; i < nrows; ++i) {
+                cp_async_wait<DEPTH - 1>();
+                const int q = (int)g + i * (int)G;
+                if (!mesh || ((valid_bits >> slot) & 1u)) {
+                    const V v = ring[slot * blockDim.x];
+                    *reinterpret_cast<V *>(R.B + (base + q) * R.stride_d) = v;
+                }
+                valid_bits &= ~(1u << slot);
+                const int ahead = i + DEPTH;
+                if (ahead < nrows) {
+                    const unsigned char *src;
+                    if (row_source(L, R, s_coord, TP, base, (int)g + ahead * (int)G, src)) {
+                        cp_async<W>(ring + slot * blockDim.x, src);
+                        valid_bits |= 1u << slot;
+                    }
+                }
+                cp_async_commit();
+                slot = slot + 1 == DEPTH ? 0 : slot + 1;
+            }
+            cp_async_wait<0>();
+        }
+    }
+    if (first) {
+        grid_dependency_wait();
+        grid_launch_dependents();
+    }
+}
+
+// Same ownership scheme with the data held in registers, for 1- and 2-byte units (cp.async
+// moves at least 4 bytes): UNROLL independent loads in flight before the first store.
+template <int W, int UNROLL>
+__global__ void __launch_bounds__(256) iso_gather_rows_reg(const __grid_constant__ LaunchDev L)
+{
+    using V = typename VecOf<W>::type;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int TP = L.tile_procs;
+    uint32_t *s_coord = reinterpret_cast<uint32_t *>(smem_raw);
+
+    const long long row_lo = (L.P * (long long)blockIdx.x) / (long long)gridDim.x;
+    const long long row_hi = (L.P * (long long)(blockIdx.x + 1)) / (long long)gridDim.x;
+    const uint32_t CU = L.chunk_units, G = L.rows_per_pass, U = L.units_per_proc;
+    const uint32_t g = threadIdx.x / CU;
+    const uint32_t ul = threadIdx.x - g * CU;
+    bool first = true;
+
+    for (long long base = row_lo; base < row_hi; base += TP) {
+        const long long left = row_hi - base;
+        const int np = (int)(left < TP ? left : TP);
+        __syncthreads();
+        tile_coordinates(L, base, np, s_coord);
+        __syncthreads();
+        if (first) {
+            grid_dependency_wait();
+            grid_launch_dependents();
+            first = false;
+        }
         if (g >= G) continue;
         for (uint32_t u = ul; u < U; u += CU) {
-            // ---- resolve this unit once ------------------------------------------------
-            uint32_t t;
-            if (L.uniform_units) {
-                t = fastdiv(L.div_uniform, u);
-            } else {
-                t = L.lookup[u >> L.lookup_shift];
-                while (t + 1 < L.nparts && __ldg(&L.parts[t + 1].first_unit) <= u) ++t;
-            }
-            const PartDev *p = L.parts + t;
-            const long long within = (long long)(u - __ldg(&p->first_unit)) * W;
-            const int sb = __ldg(&p->src_buf), db = __ldg(&p->dst_buf);
-            const long long stride_s = L.buf_stride[sb], stride_d = L.buf_stride[db];
-            const unsigned char *A = L.buf[sb] + __ldg(&p->rank_delta) * stride_s + __ldg(&p->src_off) + within;
-            unsigned char *B = L.buf[db] + __ldg(&p->dst_off) + within;
-            int c[ISO_MAX_DIMS];
-#pragma unroll
-            for (int e = 0; e < ISO_MAX_DIMS; ++e) c[e] = 0;
-            const int nnz = __ldg(&p->nnz);
-            for (int z = 0; z < nnz; ++z) {
-                const int dk = __ldg(&p->dim[z]);
-                const int cv = __ldg(&p->c[z]);
-#pragma unroll
-                for (int e = 0; e < ISO_MAX_DIMS; ++e)
-                    if (e == dk) c[e] = cv;
-            }
-            // ---- walk the rows ----------------------------------------------------------
+            const UnitRegs R = load_unit(L, u);
             for (int q0 = (int)g; q0 < np; q0 += (int)G * UNROLL) {
                 V val[UNROLL];
                 V *dst[UNROLL];
@@ -195,24 +341,10 @@ __global__ void __launch_bounds__(256) iso_gather_rows(const __grid_constant__ L
                     const int q = q0 + k * (int)G;
                     dst[k] = nullptr;
                     if (q < np) {
-                        uint32_t wrap = 0;
-                        bool valid = true;
-#pragma unroll
-                        for (int e = 0; e < ISO_MAX_DIMS; ++e) {
-                            if (e < L.n_used) {
-                                const int x = (int)s_coord[e * TP + q];
-                                if ((L.mesh_mask >> e) & 1) {
-                                    const int y = x - c[e];
-                                    valid = valid && y >= 0 && y < (int)L.used_size[e];
-                                } else if (x < c[e]) {
-                                    wrap += L.used_wrap[e];
-                                }
-                            }
-                        }
-                        if (valid) {
-                            const long long r = base + q;
-                            val[k] = *reinterpret_cast<const V *>(A + (r + wrap) * stride_s);
-                            dst[k] = reinterpret_cast<V *>(B + r * stride_d);
+                        const unsigned char *src;
+                        if (row_source(L, R, s_coord, TP, base, q, src)) {
+                            val[k] = *reinterpret_cast<const V *>(src);
+                            dst[k] = reinterpret_cast<V *>(R.B + (base + q) * R.stride_d);
                         }
                     }
                 }
@@ -221,6 +353,10 @@ __global__ void __launch_bounds__(256) iso_gather_rows(const __grid_constant__ L
                     if (dst[k]) *dst[k] = val[k];
             }
         }
+    }
+    if (first) {
+        grid_dependency_wait();
+        grid_launch_dependents();
     }
 }
 
@@ -306,6 +442,8 @@ __global__ void __launch_bounds__(256) iso_gather_bulk(const __grid_constant__ L
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
     __syncthreads();
+    grid_dependency_wait();
+    grid_launch_dependents();
 
     const uint32_t total = (uint32_t)np * L.units_per_proc;
     const uint32_t n = threadIdx.x < total ? (total - threadIdx.x + blockDim.x - 1) / blockDim.x : 0;

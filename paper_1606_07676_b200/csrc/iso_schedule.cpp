@@ -192,6 +192,59 @@ void emit_hop(Request &r, int phase, int round, int slot, const int *shift, int 
     cur_buf[slot] = p.dst_buf;
 }
 
+// Packed intermediate storage.  Algorithm 1 lets a block alternate between the receive
+// buffer and one intermediate buffer, each block staying at "its" slot; on a GPU that leaves
+// every phase reading and writing isolated blocks scattered over three buffers.  Here every
+// non-final hop of a block gets a place of its own in the intermediate buffer, and places are
+// ordered by (phase that writes, phase that reads, slot): a phase then writes one contiguous
+// region per process and reads a few contiguous regions, and the receive buffer is written
+// only by final hops.  The hops, their order and the bytes moved are unchanged; the
+// intermediate buffer grows from one place per multi-hop block to (hops - 1) places.
+void pack_intermediates(Request &r, int s)
+{
+    std::vector<std::vector<size_t>> chain(s);  // indices of a slot's hops, in execution order
+    for (size_t k = 0; k < r.parts.size(); ++k) chain[r.parts[k].slot].push_back(k);
+    struct Place { int write_phase, read_phase, slot, hop; };
+    std::vector<Place> places;
+    for (int i = 0; i < s; ++i)
+        for (size_t j = 0; j + 1 < chain[i].size(); ++j)
+            places.push_back(Place{r.parts[chain[i][j]].phase, r.parts[chain[i][j + 1]].phase, i, (int)j});
+    std::sort(places.begin(), places.end(), [](const Place &a, const Place &b) {
+        if (a.write_phase != b.write_phase) return a.write_phase < b.write_phase;
+        if (a.read_phase != b.read_phase) return a.read_phase < b.read_phase;
+        return a.slot < b.slot;
+    });
+    int64_t cur = 0;
+    for (const Place &pl : places) {
+        const int64_t len = r.len[pl.slot];
+        const bool co_aligned = ((r.sdispl[pl.slot] ^ r.rdispl[pl.slot]) & 15) == 0;
+        const int64_t mis = (len >= 16 && co_aligned) ? (r.rdispl[pl.slot] & 15) : 0;
+        const int64_t a = len >= 16 ? 16 : (len >= 8 ? 8 : (len >= 4 ? 4 : 1));
+        cur = round_up(cur, a) + mis;
+        Part &w = r.parts[chain[pl.slot][pl.hop]], &rd = r.parts[chain[pl.slot][pl.hop + 1]];
+        w.dst_buf = ISO_BUF_INTER;
+        w.dst_off = cur;
+        rd.src_buf = ISO_BUF_INTER;
+        rd.src_off = cur;
+        cur += len;
+    }
+    for (int i = 0; i < s; ++i) {
+        if (chain[i].empty()) continue;
+        Part &first = r.parts[chain[i].front()], &last = r.parts[chain[i].back()];
+        first.src_buf = ISO_BUF_SEND;
+        first.src_off = r.sdispl[i];
+        last.dst_buf = ISO_BUF_RECV;
+        last.dst_off = r.rdispl[i];
+    }
+    r.inter_stride = round_up(cur, 16);
+    // inside a phase, take the parts in the order of their source addresses
+    std::stable_sort(r.parts.begin(), r.parts.end(), [](const Part &a, const Part &b) {
+        if (a.phase != b.phase) return a.phase < b.phase;
+        if (a.src_buf != b.src_buf) return a.src_buf < b.src_buf;
+        return a.src_off < b.src_off;
+    });
+}
+
 // Section V all-to-all: dimensions (or groups of consecutive dimensions) one after the
 // other; inside a group one round per distinct non-zero projected coordinate vector.
 int build_combining_alltoall(Request &r, const Geometry &g)
@@ -239,6 +292,7 @@ int build_combining_alltoall(Request &r, const Geometry &g)
             ++phase;
         }
     }
+    if (r.layout == ISO_LAYOUT_PACKED) pack_intermediates(r, g.s);
     // blocks for the process itself: one local copy, together with the first phase
     for (Part &p : locals_parts) p.phase = 0;
     r.parts.insert(r.parts.begin(), locals_parts.begin(), locals_parts.end());
@@ -566,11 +620,42 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
         for (int kernel = 0; kernel < 2; ++kernel) {
             for (int width = 16; width >= 1; width >>= 1) {
                 std::vector<Piece> cls;
+                std::vector<std::pair<size_t, size_t>> ranges;
                 for (const Piece &q : pieces)
                     if (q.kernel == kernel && q.width == width) cls.push_back(q);
-                const size_t max_parts = 60000;
-                for (size_t lo = 0; lo < cls.size(); lo += max_parts) {
-                    size_t hi = std::min(cls.size(), lo + max_parts);
+                // a vector launch holds at most kMaxVecUnits unit positions per process (each
+                // gets a descriptor): cut longer lists, splitting a piece at a unit boundary
+                if (kernel == KERNEL_VEC) {
+                    const int64_t cap = kMaxVecUnits;
+                    std::vector<Piece> cut;
+                    std::vector<size_t> bounds(1, 0);
+                    int64_t used_units = 0;
+                    for (Piece q : cls) {
+                        while (q.p.len > 0) {
+                            int64_t n = q.p.len / width;
+                            int64_t room = cap - used_units;
+                            if (room == 0) { bounds.push_back(cut.size()); used_units = 0; room = cap; }
+                            int64_t take = std::min(n, room);
+                            Piece head = q;
+                            head.p.len = take * width;
+                            cut.push_back(head);
+                            used_units += take;
+                            q.p.src_off += take * width;
+                            q.p.dst_off += take * width;
+                            q.p.len -= take * width;
+                        }
+                    }
+                    bounds.push_back(cut.size());
+                    cls.swap(cut);
+                    for (size_t b = 0; b + 1 < bounds.size(); ++b)
+                        if (bounds[b] < bounds[b + 1]) ranges.push_back({bounds[b], bounds[b + 1]});
+                } else {
+                    const size_t max_parts = 60000;
+                    for (size_t lo = 0; lo < cls.size(); lo += max_parts)
+                        ranges.push_back({lo, std::min(cls.size(), lo + max_parts)});
+                }
+                for (const auto &range : ranges) {
+                    const size_t lo = range.first, hi = range.second;
                     LaunchPlan L;
                     L.kernel = kernel;
                     L.phase = r.parts[begin].phase;
@@ -658,6 +743,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     L.grid = grid;
                     if (L.grid > 0x7fffffff) return ISO_ERR_DIMS;
                     L.smem = (size_t)L.n_used * (size_t)tp * sizeof(uint32_t);
+                    if (kernel == KERNEL_VEC && width >= 4)
+                        L.smem = (L.smem + 15) / 16 * 16 + (size_t)kVecDepth * L.threads * width;
                     if (kernel == KERNEL_BULK)
                         L.smem = (L.smem + 15) / 16 * 16 + (size_t)L.threads * 2 * (size_t)unit + (size_t)L.threads * 2 * 8;
                     r.launches.push_back(std::move(L));

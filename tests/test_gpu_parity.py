@@ -11,6 +11,7 @@ from schedule_sim import POISON, layout, make_request, oracle_result, send_buffe
 pytestmark = pytest.mark.gpu
 
 COMB0, COMB1, COMB2, COMBD = ((iso.ISO_ALG_COMBINING, g) for g in (0, 1, 2, 8))
+ALT0, ALT1 = ((iso.ISO_ALG_COMBINING, 100 + g) for g in (0, 1))   # Algorithm 1's alternating layout
 DIRECT = (iso.ISO_ALG_DIRECT, 1)
 TORUS = (iso.ISO_ALG_TORUS, 1)
 
@@ -42,6 +43,11 @@ class Run:
         assert (st["send_stride"], st["recv_stride"]) == (ss, rs)
 
     def result(self, alg, fusion, bulk=None):
+        if fusion >= 100:
+            iso.Iso_request_set_layout(self.req, iso.ISO_LAYOUT_ALTERNATING)
+            fusion -= 100
+        else:
+            iso.Iso_request_set_layout(self.req, iso.ISO_LAYOUT_PACKED)
         iso.Iso_request_set_algorithm(self.req, alg, fusion)
         if bulk is not None:
             iso.Iso_request_set_bulk_threshold(self.req, bulk)
@@ -70,11 +76,11 @@ def check(torch, w, algs, bulk=None):
 
 # ------------------------------------------------------------------- the five configs
 def test_cfg1(torch_cuda):
-    check(torch_cuda, wl.config("cfg1"), [COMB0, COMB1, COMB2, DIRECT, TORUS])
+    check(torch_cuda, wl.config("cfg1"), [COMB0, COMB1, COMB2, ALT0, ALT1, DIRECT, TORUS])
 
 
 def test_cfg2_alltoall(torch_cuda):
-    check(torch_cuda, wl.config("cfg2_alltoall"), [COMB0, COMB1, COMB2, COMBD, DIRECT, TORUS])
+    check(torch_cuda, wl.config("cfg2_alltoall"), [COMB0, COMB1, COMB2, COMBD, ALT0, ALT1, DIRECT, TORUS])
 
 
 def test_cfg2_allgather(torch_cuda):
@@ -83,7 +89,7 @@ def test_cfg2_allgather(torch_cuda):
 
 @pytest.mark.parametrize("m", [4, 64, 512])
 def test_cfg3(torch_cuda, m):
-    check(torch_cuda, wl.config("cfg3_m%d" % m), [COMB0, COMB1, COMBD, DIRECT, TORUS])
+    check(torch_cuda, wl.config("cfg3_m%d" % m), [COMB0, COMB1, COMBD, ALT1, DIRECT, TORUS])
 
 
 def test_cfg3_512_bulk_kernel(torch_cuda):
@@ -92,12 +98,12 @@ def test_cfg3_512_bulk_kernel(torch_cuda):
 
 
 def test_cfg4(torch_cuda):
-    check(torch_cuda, wl.config("cfg4"), [COMB0, COMB1, COMB2, DIRECT])
+    check(torch_cuda, wl.config("cfg4"), [COMB0, COMB1, COMB2, ALT1, DIRECT])
 
 
 def test_cfg5(torch_cuda):
     w = wl.config("cfg5")
-    check(torch_cuda, w, [COMB0, COMB1, COMB2, DIRECT])
+    check(torch_cuda, w, [COMB0, COMB1, COMB2, ALT1, DIRECT])
     check(torch_cuda, w, [COMB1], bulk=0)
 
 
@@ -158,7 +164,7 @@ def _tiny_cases():
 
 def test_tiny_tori_and_odd_sizes(torch_cuda):
     for w in _tiny_cases():
-        algs = [COMB0, COMB1, COMB2, DIRECT] + ([TORUS] if w.collective != "allgather" else [])
+        algs = [COMB0, COMB1, COMB2, ALT1, DIRECT] + ([TORUS] if w.collective != "allgather" else [])
         check(torch_cuda, w, algs)
 
 

@@ -18,7 +18,18 @@ from schedule_sim import POISON, layout, make_request, oracle_result, send_buffe
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 ALGS = [(iso.ISO_ALG_COMBINING, 0), (iso.ISO_ALG_COMBINING, 1), (iso.ISO_ALG_COMBINING, 2),
-        (iso.ISO_ALG_COMBINING, 8), (iso.ISO_ALG_DIRECT, 1), (iso.ISO_ALG_TORUS, 1)]
+        (iso.ISO_ALG_COMBINING, 8), (iso.ISO_ALG_DIRECT, 1), (iso.ISO_ALG_TORUS, 1),
+        (iso.ISO_ALG_COMBINING, 100), (iso.ISO_ALG_COMBINING, 101)]
+
+
+def set_alg(req, alg, fusion):
+    """fusion >= 100 selects the alternating buffer layout of Algorithm 1 with fusion - 100."""
+    if fusion >= 100:
+        iso.Iso_request_set_layout(req, iso.ISO_LAYOUT_ALTERNATING)
+        fusion -= 100
+    else:
+        iso.Iso_request_set_layout(req, iso.ISO_LAYOUT_PACKED)
+    iso.Iso_request_set_algorithm(req, alg, fusion)
 
 
 def test_library_exports_every_declared_symbol():
@@ -62,7 +73,7 @@ def test_schedules_reproduce_the_oracle_on_tiny_tori(alg, fusion):
             continue
         comm, req = make_request(w)
         try:
-            iso.Iso_request_set_algorithm(req, alg, fusion)
+            set_alg(req, alg, fusion)
             st = iso.Iso_request_get_stats(req)
             lens, sd, rd, ss, rs = layout(w)
             assert (st["send_stride"], st["recv_stride"]) == (ss, rs)
@@ -84,7 +95,7 @@ def test_schedules_on_paper_shaped_configs(name, alg, fusion):
     if name == "cfg3_m4":
         w = wl.Workload(name, "alltoall", (16, 12), w.offsets, 4, kind="uint8")
     comm, req = make_request(w)
-    iso.Iso_request_set_algorithm(req, alg, fusion)
+    set_alg(req, alg, fusion)
     st = iso.Iso_request_get_stats(req)
     send = send_buffer_np(w, st["send_stride"])
     got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send)
@@ -105,7 +116,7 @@ def test_paper_neighbourhoods_small_torus(coll, nbh):
     for alg, fusion in ALGS:
         if alg == iso.ISO_ALG_TORUS and coll == "allgather":
             continue
-        iso.Iso_request_set_algorithm(req, alg, fusion)
+        set_alg(req, alg, fusion)
         st = iso.Iso_request_get_stats(req)
         send = send_buffer_np(w, st["send_stride"])
         got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send)
@@ -149,6 +160,7 @@ def test_hand_worked_schedule_4x4():
     # buffer, the last hop of every block in the receive buffer (Algorithm 1's parity rule)
     w = wl.Workload("hand", "alltoall", (4, 4), wl.moore(2, 1), 4)
     comm, req = make_request(w)
+    iso.Iso_request_set_layout(req, iso.ISO_LAYOUT_ALTERNATING)
     iso.Iso_request_set_algorithm(req, iso.ISO_ALG_COMBINING, 0)
     parts = iso.Iso_request_get_parts(req)
     rounds = {}
@@ -169,6 +181,42 @@ def test_hand_worked_schedule_4x4():
     assert all(p["dst_buf"] == iso.ISO_BUF_RECV for p in last.values())
     st = iso.Iso_request_get_stats(req)
     assert (st["rounds"], st["parts"]) == (4, 12)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
+def test_buffer_layouts_of_a_three_hop_block():
+    # 27-point stencil: the corner blocks make three hops.  Algorithm 1 sends them
+    # send -> recv -> inter -> recv (receive buffer when an odd number of hops remains);
+    # the packed layout keeps both intermediate copies in the library's buffer, writes the
+    # receive buffer only with final hops, and lays places out so that each phase writes one
+    # contiguous region of the intermediate buffer
+    w = wl.Workload("s27", "alltoall", (4, 4, 4), wl.moore(3, 1), 64)
+    comm, req = make_request(w)
+    corner = [i for i, v in enumerate(w.offsets) if all(v)]
+    assert len(corner) == 8
+    iso.Iso_request_set_layout(req, iso.ISO_LAYOUT_ALTERNATING)
+    parts = iso.Iso_request_get_parts(req)
+    for i in corner:
+        chain = [(p["src_buf"], p["dst_buf"]) for p in parts if p["slot"] == i]
+        assert chain == [(iso.ISO_BUF_SEND, iso.ISO_BUF_RECV), (iso.ISO_BUF_RECV, iso.ISO_BUF_INTER),
+                         (iso.ISO_BUF_INTER, iso.ISO_BUF_RECV)]
+    assert iso.Iso_request_get_stats(req)["inter_stride"] == 20 * 64        # one place per multi-hop block
+    moved = iso.Iso_request_get_stats(req)["bytes_moved"]
+    iso.Iso_request_set_layout(req, iso.ISO_LAYOUT_PACKED)
+    parts = iso.Iso_request_get_parts(req)
+    st = iso.Iso_request_get_stats(req)
+    assert st["bytes_moved"] == moved and st["inter_stride"] == (12 * 1 + 8 * 2) * 64
+    for i in corner:
+        chain = [(p["src_buf"], p["dst_buf"]) for p in parts if p["slot"] == i]
+        assert chain == [(iso.ISO_BUF_SEND, iso.ISO_BUF_INTER), (iso.ISO_BUF_INTER, iso.ISO_BUF_INTER),
+                         (iso.ISO_BUF_INTER, iso.ISO_BUF_RECV)]
+    for ph in range(3):
+        written = sorted((p["dst_off"], p["len"]) for p in parts if p["phase"] == ph and p["dst_buf"] == iso.ISO_BUF_INTER)
+        for (a, n), (b, _) in zip(written, written[1:]):
+            assert a + n == b, "phase %d does not write one contiguous region" % ph
+        last = [p for p in parts if p["phase"] == ph and p["dst_buf"] == iso.ISO_BUF_RECV]
+        assert all(sum(1 for q in parts if q["slot"] == p["slot"] and q["phase"] > ph) == 0 for p in last)
     iso.Iso_request_free(req)
     iso.Iso_comm_free(comm)
 
