@@ -218,7 +218,9 @@ int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes);
  * Non-periodic dimensions (Section VII: "our schedules can easily be extended to
  * non-periodic tori").  periodic[j] = 0 makes dimension j a mesh: a block whose source
  * R - C^i falls outside the mesh is not delivered and the receive slot keeps its previous
- * contents.  Only ISO_ALG_DIRECT supports meshes.  Default: all dimensions periodic.
+ * contents.  Only ISO_ALG_DIRECT supports meshes, and requests created from a neighbourhood
+ * with a mesh dimension start with that schedule.  Call it before creating requests.
+ * Default: all dimensions periodic.
  */
 int Iso_comm_set_periodic(Iso_comm isocomm, const int periodic[]);
 

@@ -110,6 +110,8 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
     r->comm = comm;
     comm->refcount++;
     r->kind = kind;
+    for (int j = 0; j < comm->d; ++j)
+        if (!comm->periodic[j]) r->alg = ISO_ALG_DIRECT;  // meshes: only the direct schedule
     r->send = static_cast<const unsigned char *>(sendbuf);
     r->recv = static_cast<unsigned char *>(recvbuf);
     r->s = comm->s;
@@ -214,10 +216,6 @@ int materialise(Request &r)
     // opt in to large dynamic shared memory once per kernel
     static bool attrs_set = false;
     if (!attrs_set) {
-        if (const char *env = std::getenv("ISO_L2_FETCH")) {
-            // experiment knob: granularity of L2 fills from device memory (a per-context limit)
-            ISO_CUDA(cudaDeviceSetLimit(cudaLimitMaxL2FetchGranularity, (size_t)std::atoi(env)));
-        }
         ISO_CUDA(cudaFuncSetAttribute(iso_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<16, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
         ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<8, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
@@ -484,6 +482,7 @@ int Iso_request_set_layout(Iso_request request, int layout)
 {
     if (check_handle(request) || (layout != ISO_LAYOUT_PACKED && layout != ISO_LAYOUT_ALTERNATING)) return ISO_ERR_ARG;
     request->layout = layout;
+    if (request->alg != ISO_ALG_COMBINING) return ISO_SUCCESS;  // takes effect with the next combining schedule
     return Iso_request_set_algorithm(request, request->alg, request->fusion);
 }
 

@@ -68,9 +68,11 @@ def oracle_result(w, send, r0=0, r1=None, fill=POISON):
     return oracle.alltoallv(w.dims, w.offsets, lens, sd, rd, ss, rs, send, r0, r1, fill=fill)
 
 
-def make_request(w, sendbuf=None, recvbuf=None):
+def make_request(w, sendbuf=None, recvbuf=None, periodic=None):
     """Creates (comm, request) for workload `w` through the C-ABI binding."""
     comm = iso.Iso_neighborhood_create(w.dims, w.offsets)
+    if periodic is not None:
+        iso.Iso_comm_set_periodic(comm, periodic)
     if w.collective == "alltoall":
         req = iso.Iso_neighbor_alltoall_init(sendbuf, w.block_bytes, iso.ISO_BYTE, recvbuf, w.block_bytes,
                                              iso.ISO_BYTE, comm)

@@ -30,14 +30,15 @@ class Run:
     """A workload bound to device buffers; `result(alg, fusion)` runs it and returns the
     receive buffers as a numpy array."""
 
-    def __init__(self, torch, w, stream=None):
+    def __init__(self, torch, w, stream=None, periodic=None):
         self.torch, self.w = torch, w
+        self.periodic = periodic
         lens, sd, rd, ss, rs = layout(w)
         self.ss, self.rs = ss, rs
         self.send_host = send_buffer_np(w, ss)
         self.send = torch.from_numpy(self.send_host).cuda()
         self.recv = torch.empty((w.P, rs), dtype=torch.uint8, device="cuda")
-        self.comm, self.req = make_request(w, self.send, self.recv)
+        self.comm, self.req = make_request(w, self.send, self.recv, periodic)
         self.stream = stream
         st = iso.Iso_request_get_stats(self.req)
         assert (st["send_stride"], st["recv_stride"]) == (ss, rs)
@@ -216,8 +217,8 @@ def test_allgatherv_and_unaligned_receive_layout(torch_cuda):
 def test_mesh_direct(torch_cuda):
     torch = torch_cuda
     w = wl.Workload("mesh", "alltoall", (9, 11), wl.moore(2, 2), 16, seed=4)
-    run = Run(torch, w)
-    iso.Iso_comm_set_periodic(run.comm, [0, 0])
+    run = Run(torch, w, periodic=[0, 0])
+    assert iso.Iso_request_get_stats(run.req)["algorithm"] == iso.ISO_ALG_DIRECT
     got = run.result(iso.ISO_ALG_DIRECT, 1).reshape(w.P, w.s, 16)
     full = oracle_result(w, run.send_host).reshape(w.P, w.s, 16)
     for r in range(w.P):

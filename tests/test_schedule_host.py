@@ -280,9 +280,8 @@ def test_alignment_classes_and_bulk_selection():
 
 def test_mesh_direct():
     w = wl.Workload("mesh", "alltoall", (4, 5), wl.moore(2, 2), 4)
-    comm, req = make_request(w)
-    iso.Iso_comm_set_periodic(comm, [0, 1])
-    iso.Iso_request_set_algorithm(req, iso.ISO_ALG_DIRECT, 1)
+    comm, req = make_request(w, periodic=[0, 1])
+    assert iso.Iso_request_get_stats(req)["algorithm"] == iso.ISO_ALG_DIRECT
     st = iso.Iso_request_get_stats(req)
     send = send_buffer_np(w, st["send_stride"])
     got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send, periodic=[0, 1])
