@@ -62,7 +62,9 @@ enum {
     ISO_ERR_CUDA = 6,    /* a CUDA call failed; see Iso_last_cuda_error */
     ISO_ERR_OVERLAP = 7, /* receive blocks overlap each other, or send and receive buffers overlap */
     ISO_ERR_STATE = 8,   /* call not valid in this state (e.g. request bound to no buffers) */
-    ISO_ERR_TIMEOUT = 9  /* a bounded wait inside a kernel expired; the result is incomplete */
+    ISO_ERR_TIMEOUT = 9, /* a bounded wait inside a kernel expired; the result is incomplete */
+    ISO_ERR_TOO_LARGE = 10 /* Iso_neighbor_alltoall_static: tables + intermediate buffer exceed
+                              ISO_STATIC_SCRATCH_BYTES */
 };
 
 /* Schedules. */
@@ -251,6 +253,45 @@ int Iso_request_get_stats(Iso_request request, Iso_stats *out);
 /* Copies up to `capacity` executed parts (in execution order) to `out` and stores the
  * total number in `*count`.  Needs no device; meant for validation of schedules. */
 int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int *count);
+
+/*
+ * Regular message-combining all-to-all that allocates no device memory.  (The paper has no
+ * counterpart: its library may allocate freely inside the init call.)
+ *
+ * For callers that cannot allocate where they need the collective: programs whose device
+ * memory was budgeted and handed out at start-up, plug-ins living inside another
+ * framework's memory pool, hot paths where a cudaMalloc - which synchronises the device -
+ * is not acceptable.  Iso_neighbor_alltoall_init / Iso_Start keep their unit tables and
+ * their intermediate buffer in memory obtained with cudaMalloc; this call keeps both in a
+ * fixed scratch array of ISO_STATIC_SCRATCH_BYTES bytes that is part of the library image
+ * (every device that loads the library holds one copy until the process exits) and calls
+ * no cudaMalloc, cudaFree, cudaMallocHost or other allocating CUDA routine.  The schedule
+ * itself is computed on the host with ordinary heap memory that is released before return.
+ *
+ * Same arguments as Iso_neighborhood_create + Iso_neighbor_alltoall_init (send and receive
+ * blocks of count * type bytes, both buffers DEVICE pointers owned by the caller, layout
+ * as described at the top of this file) plus the stream; the schedule is ISO_ALG_COMBINING,
+ * one launch per dimension, packed layout, vector kernel only.  The call copies the tables
+ * into the scratch area and enqueues the kernels on `cuda_stream`; it does not wait.
+ *
+ * Limits and rules:
+ *  - P * (intermediate bytes per process) + the unit tables must fit the scratch array,
+ *    else ISO_ERR_TOO_LARGE and nothing is enqueued;
+ *  - the first call on a device looks up the device address of the scratch array
+ *    (cudaGetSymbolAddress, with that device current); make that first call outside any
+ *    stream capture;
+ *  - all calls on one device share the scratch array and it keeps the previous call's
+ *    contents; nothing in it has to start at zero, because every byte a kernel reads from
+ *    it was written earlier in the same call (tables by the copy, intermediate places by
+ *    an earlier phase).  Two calls whose work overlaps on the GPU (different streams, or
+ *    different host threads) race on it: keep calls on one device in one stream order.
+ * Errors: ISO_ERR_ARG, ISO_ERR_DIMS, ISO_ERR_COUNT, ISO_ERR_OVERLAP, ISO_ERR_TOO_LARGE,
+ * ISO_ERR_CUDA.
+ */
+#define ISO_STATIC_SCRATCH_BYTES (8u << 20)
+int Iso_neighbor_alltoall_static(int d, const int dims[], int s, const int relative_coordinates[],
+                                 const void *sendbuf, void *recvbuf, int count, Iso_datatype type,
+                                 void *cuda_stream);
 
 /* Frees the request, its device memory and its reference on the neighbourhood; waits for
  * work in flight first.  `*request` is set to NULL. */

@@ -20,7 +20,8 @@ ISO_BUF_SEND, ISO_BUF_RECV, ISO_BUF_INTER = 0, 1, 2
 ISO_LAYOUT_PACKED, ISO_LAYOUT_ALTERNATING = 0, 1
 ISO_BYTE, ISO_INT32, ISO_FLOAT, ISO_DOUBLE = 1, 4, 4, 8
 (ISO_SUCCESS, ISO_ERR_ARG, ISO_ERR_DIMS, ISO_ERR_COUNT, ISO_ERR_ALIGN, ISO_ERR_NOMEM, ISO_ERR_CUDA,
- ISO_ERR_OVERLAP, ISO_ERR_STATE, ISO_ERR_TIMEOUT) = range(10)
+ ISO_ERR_OVERLAP, ISO_ERR_STATE, ISO_ERR_TIMEOUT, ISO_ERR_TOO_LARGE) = range(11)
+ISO_STATIC_SCRATCH_BYTES = 8 << 20
 
 LIB_NAME = "libiso_b200.so"
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), LIB_NAME)
@@ -31,7 +32,7 @@ EXPORTS = (
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
     "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_bulk_threshold",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
-    "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
+    "Iso_neighbor_alltoall_static", "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
 
 
@@ -96,6 +97,7 @@ def load_library() -> ctypes.CDLL:
         "Iso_wait": [vp],
         "Iso_request_get_stats": [vp, ctypes.POINTER(Iso_stats)],
         "Iso_request_get_parts": [vp, ctypes.POINTER(Iso_part), ci, ctypes.POINTER(ci)],
+        "Iso_neighbor_alltoall_static": [ci, vp, ci, vp, vp, vp, ci, ci, vp],
         "Iso_request_free": [pp],
         "Iso_last_cuda_error": [],
         "Iso_selftest": [],
@@ -260,6 +262,20 @@ def Iso_request_get_parts(request: int) -> list:
     arr = (Iso_part * max(1, n.value))()
     _check(lib.Iso_request_get_parts(request, arr, n.value, ctypes.byref(n)), "Iso_request_get_parts")
     return [arr[k].as_dict() for k in range(n.value)]
+
+
+def Iso_neighbor_alltoall_static(dims, relative_coordinates, sendbuf, recvbuf, count: int, datatype: int,
+                                 stream=None) -> None:
+    """All-to-all through the entry point that allocates no device memory: tables and
+    intermediate buffer live in the library's fixed scratch array (see include/iso.h)."""
+    dims = _i32(dims)
+    coords = _i32(relative_coordinates)
+    d = int(dims.size)
+    if d == 0 or coords.size % d:
+        raise ValueError("relative_coordinates must hold s*d integers")
+    _check(load_library().Iso_neighbor_alltoall_static(d, dims.ctypes.data, coords.size // d, coords.ctypes.data,
+                                                       _addr(sendbuf), _addr(recvbuf), count, datatype,
+                                                       _stream(stream)), "Iso_neighbor_alltoall_static")
 
 
 def Iso_request_free(request: int) -> None:

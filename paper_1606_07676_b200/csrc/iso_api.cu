@@ -618,6 +618,7 @@ const char *Iso_error_string(int code)
     case ISO_ERR_OVERLAP: return "buffers or blocks overlap";
     case ISO_ERR_STATE: return "call not valid in this state";
     case ISO_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case ISO_ERR_TOO_LARGE: return "problem does not fit the static scratch area";
     default: return "unknown error code";
     }
 }
@@ -645,3 +646,163 @@ int Iso_selftest(void)
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free variant of the message-combining all-to-all.
+//
+// Some programs may not allocate device memory at the point where they need the collective:
+// a solver whose memory budget was fixed and handed out at start-up, a plug-in that runs
+// inside another framework's memory pool, or a service that forbids cudaMalloc on its hot
+// path because the call synchronises the whole device.  The ordinary path (Iso_neighbor_alltoall_init +
+// Iso_Start) allocates its index tables and its intermediate buffer with cudaMalloc.  The
+// entry point below keeps both in a fixed array that is part of the library image
+// instead, so that it never allocates; the price is an upper bound on the problem size and
+// one shared scratch area per device.
+namespace {
+
+// The scratch area: intermediate buffer first, unit tables behind it.  Every device that
+// loads the library holds one copy until the process exits.
+static __device__ __align__(256) unsigned char iso_static_scratch[ISO_STATIC_SCRATCH_BYTES];
+
+// Device address of the scratch area per device ordinal.  The array's name is only a
+// host-side handle; kernels need the address cudaGetSymbolAddress returns on that device.
+constexpr int kMaxDevices = 64;
+unsigned char *g_scratch_addr[kMaxDevices] = {nullptr};
+
+int scratch_for_current_device(unsigned char **out)
+{
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return ISO_ERR_CUDA;
+    if (device < 0 || device >= kMaxDevices) return ISO_ERR_ARG;
+    if (!g_scratch_addr[device]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, iso_static_scratch);
+        if (e != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return ISO_ERR_CUDA;
+        }
+        g_scratch_addr[device] = static_cast<unsigned char *>(p);
+    }
+    *out = g_scratch_addr[device];
+    return ISO_SUCCESS;
+}
+
+int64_t round_up_256(int64_t x) { return (x + 255) / 256 * 256; }
+
+}  // namespace
+
+extern "C" int Iso_neighbor_alltoall_static(int d, const int dims[], int s, const int relative_coordinates[],
+                                            const void *sendbuf, void *recvbuf, int count, Iso_datatype type,
+                                            void *cuda_stream)
+{
+    if (!dims || s < 0 || (s > 0 && !relative_coordinates) || !sendbuf || !recvbuf || count < 0 || type < 1)
+        return ISO_ERR_ARG;
+    if (d < 1 || d > ISO_MAX_DIMS) return ISO_ERR_DIMS;
+
+    // the neighbourhood and the request live on the host stack / heap for this call only
+    Comm comm;
+    comm.d = d;
+    comm.s = s;
+    int64_t P = 1, stride = 1;
+    for (int j = 0; j < d; ++j) {
+        if (dims[j] < 1 || P > (int64_t)0x7fffffff / dims[j]) return ISO_ERR_DIMS;
+        P *= dims[j];
+    }
+    comm.P = P;
+    for (int j = d - 1; j >= 0; --j) {
+        comm.dims[j] = dims[j];
+        comm.periodic[j] = 1;
+        comm.rank_stride[j] = stride;
+        stride *= dims[j];
+    }
+    comm.coords.assign(relative_coordinates, relative_coordinates + (size_t)s * d);
+
+    const int64_t m = (int64_t)count * type;
+    Request r;
+    r.comm = &comm;
+    r.kind = ISO_KIND_ALLTOALL;
+    r.alg = ISO_ALG_COMBINING;
+    r.fusion = 1;
+    r.layout = ISO_LAYOUT_PACKED;
+    r.bulk_threshold = 0;  // vector kernel only: no error flag, nothing that must start at zero
+    r.send = static_cast<const unsigned char *>(sendbuf);
+    r.recv = static_cast<unsigned char *>(recvbuf);
+    r.s = s;
+    r.len.assign(s, m);
+    r.sdispl.resize(s);
+    r.rdispl.resize(s);
+    for (int i = 0; i < s; ++i) r.sdispl[i] = r.rdispl[i] = (int64_t)i * m;
+    r.send_stride = r.recv_stride = (int64_t)s * m;
+    if (s == 0 || m == 0) return ISO_SUCCESS;
+    if (r.send_stride > INT64_MAX / P) return ISO_ERR_COUNT;
+    {
+        const unsigned char *s0 = r.send, *s1 = r.send + P * r.send_stride;
+        const unsigned char *d0 = r.recv, *d1 = r.recv + P * r.recv_stride;
+        if (s0 < d1 && d0 < s1) return ISO_ERR_OVERLAP;
+    }
+    int rc = build_schedule(r);
+    if (rc != ISO_SUCCESS) return rc;
+
+    // does it fit?  (checked before anything touches the device)
+    if (r.inter_stride > (int64_t)ISO_STATIC_SCRATCH_BYTES / P) return ISO_ERR_TOO_LARGE;
+    const int64_t inter_bytes = round_up_256(P * r.inter_stride);
+    unsigned char *scratch = nullptr;
+    rc = scratch_for_current_device(&scratch);
+    if (rc != ISO_SUCCESS) return rc;
+    int device = 0, sms = 0;
+    if (cudaGetDevice(&device) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0)
+        r.sm_count = sms;
+    rc = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)scratch);
+    if (rc != ISO_SUCCESS) return rc;
+    int64_t table_bytes = 0;
+    for (LaunchPlan &L : r.launches) {
+        if (L.kernel != KERNEL_VEC) return ISO_ERR_STATE;
+        L.units_off = (size_t)table_bytes;
+        table_bytes += (int64_t)L.units_per_proc * (int64_t)sizeof(UnitDev);
+    }
+    if (inter_bytes + table_bytes > (int64_t)ISO_STATIC_SCRATCH_BYTES) return ISO_ERR_TOO_LARGE;
+
+    // unit tables, built on the host and copied behind the intermediate buffer
+    std::vector<unsigned char> blob((size_t)table_bytes, 0);
+    const int64_t strides[3] = {r.send_stride, r.recv_stride, r.inter_stride};
+    for (const LaunchPlan &L : r.launches) {
+        int used_index[ISO_MAX_DIMS];
+        for (int j = 0; j < ISO_MAX_DIMS; ++j) used_index[j] = -1;
+        for (int k = 0; k < L.n_used; ++k) used_index[L.used_dim[k]] = k;
+        UnitDev *ud = reinterpret_cast<UnitDev *>(blob.data() + L.units_off);
+        for (const LoweredPart &lp : L.parts) {
+            long long delta = 0;
+            UnitDev u{};
+            for (int j = 0; j < d; ++j) {
+                if (!lp.p.shift[j]) continue;
+                delta -= (long long)lp.p.shift[j] * comm.rank_stride[j];
+                u.c[used_index[j]] = lp.p.shift[j];
+            }
+            u.src_buf = (uint8_t)lp.p.src_buf;
+            u.dst_buf = (uint8_t)lp.p.dst_buf;
+            for (uint32_t k = 0; k < lp.units; ++k) {
+                u.src_term = delta * strides[lp.p.src_buf] + lp.p.src_off + (int64_t)k * L.width;
+                u.dst_term = lp.p.dst_off + (int64_t)k * L.width;
+                ud[lp.first_unit + k] = u;
+            }
+        }
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    unsigned char *tables = scratch + inter_bytes;
+    if (table_bytes > 0 &&
+        cudaMemcpyAsync(tables, blob.data(), (size_t)table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ISO_ERR_CUDA;
+    }
+
+    // the ordinary launch path, pointed at the scratch area (nothing here is owned by `r`)
+    r.d_blob = tables;
+    r.d_inter = scratch;
+    for (const LaunchPlan &L : r.launches) {
+        rc = launch_one(r, L, stream, false);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    return ISO_SUCCESS;
+}
