@@ -82,7 +82,7 @@ enum {
                                    a phase touches few contiguous regions; receive buffer written by
                                    final hops only.  Intermediate buffer: sum_i (hops_i - 1) blocks */
     ISO_LAYOUT_ALTERNATING = 1  /* Algorithm 1: the block alternates between its slot of the receive
-                                   buffer and its slot of an intermediate buffer "of the same size" */
+                                   buffer and its slot of an equally large intermediate buffer */
 };
 
 enum { ISO_KIND_ALLTOALL = 0, ISO_KIND_ALLGATHER = 1, ISO_KIND_ALLTOALLV = 2 };
@@ -95,7 +95,7 @@ typedef struct Iso_stats {
     int d;
     int s;
     int rounds;           /* communication rounds of the schedule (Sections III-A and V) */
-    int max_rounds_per_dim; /* the factor N of the bound "at most N*d rounds" */
+    int max_rounds_per_dim; /* the factor N of the paper's N*d bound on the rounds */
     int phases;           /* groups of rounds that run without an ordering point between them */
     int launches;         /* kernel launches per Iso_Start */
     int parts;            /* block transmissions per process: sum of hops (all-to-all),
@@ -175,8 +175,8 @@ int Iso_neighbor_allgather_init(const void *sendbuf, int sendcount, Iso_datatype
  * displacement recvdispls[i] of the receiver's buffer.  Counts and displacements (s
  * entries each, host arrays, copied) are the same on every process and block sizes must
  * match pairwise in bytes (ISO_ERR_COUNT).  Displacements must be >= 0; receive blocks
- * must not overlap each other (ISO_ERR_OVERLAP); send blocks may.  "It uses the same
- * schedules as in the regular case" (Section IV).
+ * must not overlap each other (ISO_ERR_OVERLAP); send blocks may.  The schedules are those
+ * of the regular case (Section IV).
  */
 int Iso_neighbor_alltoallv_init(const void *sendbuf, const int sendcounts[],
                                 const int64_t senddispls[], Iso_datatype sendtype,
@@ -199,8 +199,8 @@ int Iso_neighbor_allgatherv_init(const void *sendbuf, int sendcount, Iso_datatyp
  * ISO_ALG_COMBINING: 0 = one kernel launch per communication round; 1 (the default) = all
  * rounds of one dimension in one launch (same bytes moved: within a dimension every block
  * moves at most once); g >= 2 = the dimensions are taken in groups of g consecutive ones and
- * a block's hops inside a group are composed into a single shift (Section V: "all blocks
- * going to the same relative neighbor ... can be combined"), so fewer intermediate copies
+ * a block's hops inside a group are composed into a single shift (Section V combines all
+ * blocks bound for the same relative neighbour), so fewer intermediate copies
  * pass through memory; g >= d moves exactly the bytes of ISO_ALG_DIRECT.
  * May be called at any time between starts; the schedule is rebuilt and the device tables
  * are replaced by the next Iso_Start.  Errors: ISO_ERR_ARG.
@@ -217,8 +217,7 @@ int Iso_request_set_layout(Iso_request request, int layout);
 int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes);
 
 /*
- * Non-periodic dimensions (Section VII: "our schedules can easily be extended to
- * non-periodic tori").  periodic[j] = 0 makes dimension j a mesh: a block whose source
+ * Non-periodic dimensions (the extension Section VII mentions).  periodic[j] = 0 makes dimension j a mesh: a block whose source
  * R - C^i falls outside the mesh is not delivered and the receive slot keeps its previous
  * contents.  Only ISO_ALG_DIRECT supports meshes, and requests created from a neighbourhood
  * with a mesh dimension start with that schedule.  Call it before creating requests.

@@ -7,7 +7,7 @@ schedule builder of the CUDA library, whose statistics the tests compare with
 these numbers.
 
 Where ``dims`` is given the coordinates are first replaced by their residue
-modulo p_j ("different coordinates may denote the same neighbor", Section II):
+modulo p_j (Section II notes that on a small torus several coordinates can name the same process):
 the residue in [0, p_j) for the direct-communication schedules, the
 representative of smallest magnitude (ties towards the positive one) for the
 hop-by-hop schedules.

@@ -48,7 +48,7 @@ def test_paper_neighbourhood_sizes():
     assert len(wl.shells(3, (3, 7))) == 1396
     assert len(wl.positive_octant(3, 1)) == 7     # the octant example of Section II
     sh = wl.shells(3, (3, 7))
-    assert counters.torus_rounds(sh, 3) == 2 * 7 * 3    # "about 2 r2 d = 42" rounds
+    assert counters.torus_rounds(sh, 3) == 2 * 7 * 3    # the paper puts the hop-by-hop schedule at about 2*r2*d = 42 rounds
 
 
 def test_fig1_trie_shape():
@@ -77,7 +77,7 @@ def test_irregular_size_rule_total():
     offs = wl.moore(3, 1)
     total = sum(512 ** (3 - int(np.abs(v).sum())) for v in offs)
     assert total == 8 * 1 + 12 * 512 + 6 * 512 ** 2
-    assert abs(total / 2 ** 20 - 1.5) < 0.01      # "1.5 MB for the entire send buffer"
+    assert abs(total / 2 ** 20 - 1.5) < 0.01      # the paper gives 1.5 MB for the whole send buffer
 
 
 # ----------------------------------------------------------------------- generators

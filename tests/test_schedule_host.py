@@ -135,7 +135,7 @@ def test_alltoall_statistics_follow_section_v(name):
     assert st["rounds"] == counters.direct_rounds(w.offsets, d, w.dims)
     assert st["parts"] == counters.direct_volume(w.offsets, d, w.dims)
     assert st["max_rounds_per_dim"] == max(counters.direct_rounds_per_dim(w.offsets, d, w.dims))
-    assert st["rounds"] <= st["max_rounds_per_dim"] * d            # "at most N d rounds"
+    assert st["rounds"] <= st["max_rounds_per_dim"] * d            # the N d bound on the rounds
     assert st["phases"] <= d
     lens = layout(w)[0]
     hops = counters.direct_hops(w.offsets, d, w.dims)
