@@ -217,9 +217,6 @@ int materialise(Request &r)
     static bool attrs_set = false;
     if (!attrs_set) {
         ISO_CUDA(cudaFuncSetAttribute(iso_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<16, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
-        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<8, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
-        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows<4, kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
         attrs_set = true;
     }
     r.dirty = false;
@@ -295,14 +292,27 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
     cudaError_t e;
     if (L.kernel == KERNEL_BULK) {
         e = launch_kernel(iso_gather_bulk, L, a, stream, dependent);
+    } else if (L.width < 4) {
+        e = L.width == 2 ? launch_kernel(iso_gather_rows_reg<2, 4>, L, a, stream, dependent)
+                         : launch_kernel(iso_gather_rows_reg<1, 4>, L, a, stream, dependent);
     } else {
-        switch (L.width) {
-        case 16: e = launch_kernel(iso_gather_rows<16, kVecDepth>, L, a, stream, dependent); break;
-        case 8: e = launch_kernel(iso_gather_rows<8, kVecDepth>, L, a, stream, dependent); break;
-        case 4: e = launch_kernel(iso_gather_rows<4, kVecDepth>, L, a, stream, dependent); break;
-        case 2: e = launch_kernel(iso_gather_rows_reg<2, 4>, L, a, stream, dependent); break;
-        default: e = launch_kernel(iso_gather_rows_reg<1, 4>, L, a, stream, dependent); break;
-        }
+        // kernels specialised on the number of shifted dimensions; meshes take the general one
+        const int nu = L.n_used <= 3 ? L.n_used : ISO_MAX_DIMS;
+#define ISO_ROWS(W, NU, MESH) e = launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH>, L, a, stream, dependent)
+#define ISO_ROWS_W(W)                                             \
+    do {                                                          \
+        if (a.mesh_mask) ISO_ROWS(W, ISO_MAX_DIMS, true);         \
+        else if (nu == 0) ISO_ROWS(W, 0, false);                  \
+        else if (nu == 1) ISO_ROWS(W, 1, false);                  \
+        else if (nu == 2) ISO_ROWS(W, 2, false);                  \
+        else if (nu == 3) ISO_ROWS(W, 3, false);                  \
+        else ISO_ROWS(W, ISO_MAX_DIMS, false);                    \
+    } while (0)
+        if (L.width == 16) ISO_ROWS_W(16);
+        else if (L.width == 8) ISO_ROWS_W(8);
+        else ISO_ROWS_W(4);
+#undef ISO_ROWS_W
+#undef ISO_ROWS
     }
     ISO_CUDA(e);
     return ISO_SUCCESS;

@@ -220,78 +220,107 @@ __device__ __forceinline__ bool row_source(const LaunchDev &L, const UnitRegs &R
 
 // Vector gather.  Thread t of a CTA owns one unit position (row slot g = t / chunk_units,
 // unit u = t % chunk_units): it loads that unit's descriptor once and then walks down the
-// CTA's rows (processes).  CTA b handles the rows [P*b/grid, P*(b+1)/grid), so a grid sized
-// to the machine stays balanced to one row.  Per row the work is a wrap test per shifted
-// dimension and two address computations.
+// CTA's rows (processes) with running source and destination pointers.  CTA b handles the
+// rows [P*b/grid, P*(b+1)/grid), so a grid sized to the machine stays balanced to one row.
+// Per row the work is a wrap test per shifted dimension and two pointer increments.
 //
 // Data path for W in {16, 8, 4}: cp.async from global memory into a thread-private ring of
 // DEPTH slots in shared memory, so that DEPTH loads per thread are in flight without
 // holding registers; a slot is read back and stored to its destination as soon as the
 // oldest group has landed, and refilled with the load of DEPTH rows ahead.
-template <int W, int DEPTH>
-__global__ void __launch_bounds__(256) iso_gather_rows(const __grid_constant__ LaunchDev L)
+//
+// NU is the number of shifted dimensions the kernel is compiled for (the launch's n_used
+// must not exceed it; ISO_MAX_DIMS is the general case), MESH whether some of them are
+// non-periodic (then a row whose source lies outside the mesh is skipped).
+template <int W, int DEPTH, int NU, bool MESH>
+__global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant__ LaunchDev L)
 {
     using V = typename VecOf<W>::type;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int TP = L.tile_procs;
     uint32_t *s_coord = reinterpret_cast<uint32_t *>(smem_raw);  // [n_used][tile_procs]
     const uint32_t coord_bytes = ((uint32_t)L.n_used * (uint32_t)TP * 4u + 15u) & ~15u;
-    V *ring = reinterpret_cast<V *>(smem_raw + coord_bytes) + threadIdx.x;  // slot k at ring[k * blockDim.x]
+    V *const ring = reinterpret_cast<V *>(smem_raw + coord_bytes) + threadIdx.x;  // slot k at ring[k * blockDim.x]
+    V *const ring_end = ring + DEPTH * blockDim.x;
 
     const long long row_lo = (L.P * (long long)blockIdx.x) / (long long)gridDim.x;
     const long long row_hi = (L.P * (long long)(blockIdx.x + 1)) / (long long)gridDim.x;
-    const uint32_t CU = L.chunk_units, G = L.rows_per_pass, U = L.units_per_proc;
-    const uint32_t g = threadIdx.x / CU;
-    const uint32_t ul = threadIdx.x - g * CU;
-    const bool mesh = L.mesh_mask != 0;
+    const uint32_t CU = L.chunk_units, U = L.units_per_proc;
+    const int G = (int)L.rows_per_pass;
+    const int g = (int)(threadIdx.x / CU);
+    const uint32_t ul = threadIdx.x - (uint32_t)g * CU;
     bool first = true;
 
     for (long long base = row_lo; base < row_hi; base += TP) {
         const long long left = row_hi - base;
         const int np = (int)(left < TP ? left : TP);
         __syncthreads();
-        tile_coordinates(L, base, np, s_coord);
+        if (NU > 0) tile_coordinates(L, base, np, s_coord);
         __syncthreads();
         if (first) {
             grid_dependency_wait();
             grid_launch_dependents();
             first = false;
         }
-        if (g >= G || (int)g >= np) continue;
-        const int nrows = (np - (int)g + (int)G - 1) / (int)G;  // rows g, g+G, ...
+        if (g >= G || g >= np) continue;
         for (uint32_t u = ul; u < U; u += CU) {
             const UnitRegs R = load_unit(L, u);
-            uint32_t valid_bits = 0;
+            long long wrap_bytes[NU > 0 ? NU : 1];
+#pragma unroll
+            for (int e = 0; e < NU; ++e) wrap_bytes[e] = (long long)L.used_wrap[e] * R.stride_s;
+            const long long src_step = (long long)G * R.stride_s, dst_step = (long long)G * R.stride_d;
+
+            // source of row q given the pointer that ignores wrap-around; false: outside the mesh
+            auto source = [&](const unsigned char *nowrap, int q, const unsigned char *&src) -> bool {
+                bool valid = true;
+                src = nowrap;
+#pragma unroll
+                for (int e = 0; e < NU; ++e) {
+                    if (NU < ISO_MAX_DIMS || e < L.n_used) {
+                        const int x = (int)s_coord[e * TP + q];
+                        if (MESH && ((L.mesh_mask >> e) & 1)) {
+                            const int y = x - R.c[e];
+                            valid = valid && y >= 0 && y < (int)L.used_size[e];
+                        } else if (x < R.c[e]) {
+                            src += wrap_bytes[e];
+                        }
+                    }
+                }
+                return valid;
+            };
+
+            int q_ld = g;  // next row to load
+            const unsigned char *src_ld = R.A + (base + g) * R.stride_s;
+            unsigned char *dst = R.B + (base + g) * R.stride_d;
 #pragma unroll
             for (int i = 0; i < DEPTH; ++i) {
-                if (i < nrows) {
+                if (q_ld < np) {
                     const unsigned char *src;
-                    if (row_source(L, R, s_coord, TP, base, (int)g + i * (int)G, src)) {
-                        cp_async<W>(ring + i * blockDim.x, src);
-                        valid_bits |= 1u << i;
-                    }
+                    if (source(src_ld, q_ld, src)) cp_async<W>(ring + i * blockDim.x, src);
+                    q_ld += G;
+                    src_ld += src_step;
                 }
                 cp_async_commit();
             }
-            int slot = 0;
-            for (int i = 0; i < nrows; ++i) {
+            V *slot = ring;
+            for (int q = g; q < np; q += G) {
                 cp_async_wait<DEPTH - 1>();
-                const int q = (int)g + i * (int)G;
-                if (!mesh || ((valid_bits >> slot) & 1u)) {
-                    const V v = ring[slot * blockDim.x];
-                    *reinterpret_cast<V *>(R.B + (base + q) * R.stride_d) = v;
+                bool valid = true;
+                if (MESH) {
+                    const unsigned char *ignored;
+                    valid = source(nullptr, q, ignored);
                 }
-                valid_bits &= ~(1u << slot);
-                const int ahead = i + DEPTH;
-                if (ahead < nrows) {
+                if (valid) *reinterpret_cast<V *>(dst) = *slot;
+                dst += dst_step;
+                if (q_ld < np) {
                     const unsigned char *src;
-                    if (row_source(L, R, s_coord, TP, base, (int)g + ahead * (int)G, src)) {
-                        cp_async<W>(ring + slot * blockDim.x, src);
-                        valid_bits |= 1u << slot;
-                    }
+                    if (source(src_ld, q_ld, src)) cp_async<W>(slot, src);
+                    q_ld += G;
+                    src_ld += src_step;
                 }
                 cp_async_commit();
-                slot = slot + 1 == DEPTH ? 0 : slot + 1;
+                slot += blockDim.x;
+                if (slot == ring_end) slot = ring;
             }
             cp_async_wait<0>();
         }
