@@ -186,8 +186,12 @@ class Bound:
         else:
             self.req = iso.Iso_neighbor_alltoallv_init(self.send, self.lens, self.sd, 1, self.recv, self.lens, self.rd, 1, self.comm)
 
+    bulk_threshold = None
+
     def set(self, alg, fusion):
         self.iso.Iso_request_set_algorithm(self.req, alg, fusion)
+        if Bound.bulk_threshold is not None:
+            self.iso.Iso_request_set_bulk_threshold(self.req, Bound.bulk_threshold)
         self.iso.Iso_Start(self.req, self.torch.cuda.current_stream())    # materialise outside the timed region
         self.iso.Iso_wait(self.req)
         return self.iso.Iso_request_get_stats(self.req)
@@ -304,6 +308,7 @@ def run_ours(args):
     iso.load_library()
 
     peak, peak_kind = measured_peak()
+    Bound.bulk_threshold = args.bulk_threshold
     reps = Replicas(torch, iso, wl, args.workload)
     b = reps.items[0]
 
@@ -454,6 +459,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--headline-only", action="store_true",
                     help="time the headline schedule only (short runs under a profiler)")
+    ap.add_argument("--bulk-threshold", type=int, default=None,
+                    help="override the size from which parts go to the bulk-copy kernel (0: never)")
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture, if one is current")
     args = ap.parse_args()

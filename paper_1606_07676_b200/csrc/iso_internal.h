@@ -81,7 +81,7 @@ struct Request {
     int kind = ISO_KIND_ALLTOALL;
     int alg = ISO_ALG_COMBINING;
     int fusion = 1;
-    int64_t bulk_threshold = 1024;
+    int64_t bulk_threshold = 512;
     int layout = ISO_LAYOUT_PACKED;
     const unsigned char *send = nullptr;
     unsigned char *recv = nullptr;

@@ -721,11 +721,11 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                             int v = std::atoi(env);
                             if (v >= 1 && v <= 8) per_sm = v;
                         }
-                        // persistent grid: CTA b owns rows [P*b/grid, P*(b+1)/grid)
+                        // persistent grid: CTA b takes the row groups b, b + grid, ...
                         grid = std::min<int64_t>((c.P + L.rows_per_pass - 1) / L.rows_per_pass,
                                                  (int64_t)r.sm_count * per_sm);
                         grid = std::max<int64_t>(grid, 1);
-                        tp = std::min<int64_t>(512, (c.P + grid - 1) / grid);
+                        tp = 1;
                     } else {
                         int threads = (int)(196608 / (2 * unit)) / 32 * 32;
                         L.threads = std::max(32, std::min(256, threads));
@@ -743,8 +743,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     L.grid = grid;
                     if (L.grid > 0x7fffffff) return ISO_ERR_DIMS;
                     L.smem = (size_t)L.n_used * (size_t)tp * sizeof(uint32_t);
-                    if (kernel == KERNEL_VEC && width >= 4)
-                        L.smem = (L.smem + 15) / 16 * 16 + (size_t)kVecDepth * L.threads * width;
+                    if (kernel == KERNEL_VEC) L.smem = width >= 4 ? (size_t)kVecDepth * L.threads * width : 0;
                     if (kernel == KERNEL_BULK)
                         L.smem = (L.smem + 15) / 16 * 16 + (size_t)L.threads * 2 * (size_t)unit + (size_t)L.threads * 2 * 8;
                     r.launches.push_back(std::move(L));

@@ -93,9 +93,11 @@ def test_cfg3(torch_cuda, m):
     check(torch_cuda, wl.config("cfg3_m%d" % m), [COMB0, COMB1, COMBD, ALT1, DIRECT, TORUS])
 
 
-def test_cfg3_512_bulk_kernel(torch_cuda):
-    # 512-byte blocks through the bulk-copy kernel as well (threshold lowered)
-    check(torch_cuda, wl.config("cfg3_m512"), [COMB1, DIRECT], bulk=512)
+def test_cfg3_512_both_kernels(torch_cuda):
+    # 512-byte blocks go to the bulk-copy kernel by default; here also through the vector
+    # kernel (bulk kernel off) and with the threshold at 1 KB
+    check(torch_cuda, wl.config("cfg3_m512"), [COMB1, DIRECT], bulk=0)
+    check(torch_cuda, wl.config("cfg3_m512"), [COMB1], bulk=1024)
 
 
 def test_cfg4(torch_cuda):

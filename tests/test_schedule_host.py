@@ -267,7 +267,7 @@ def test_alignment_classes_and_bulk_selection():
     for p in parts:
         assert p["src_off"] % p["width"] == 0 or p["kernel"] == 1
         if p["kernel"] == 1:
-            assert p["src_off"] % 16 == 0 and p["dst_off"] % 16 == 0 and p["len"] % 16 == 0 and p["len"] >= 1024
+            assert p["src_off"] % 16 == 0 and p["dst_off"] % 16 == 0 and p["len"] % 16 == 0 and p["len"] >= 512
     st = iso.Iso_request_get_stats(req)
     send = send_buffer_np(w, st["send_stride"])
     assert np.array_equal(simulate(parts, w.dims, st, send), oracle_result(w, send))
