@@ -187,8 +187,10 @@ class Bound:
             self.req = iso.Iso_neighbor_alltoallv_init(self.send, self.lens, self.sd, 1, self.recv, self.lens, self.rd, 1, self.comm)
 
     bulk_threshold = None
+    single_launch = False
 
     def set(self, alg, fusion):
+        self.iso.Iso_request_set_single_launch(self.req, Bound.single_launch)
         self.iso.Iso_request_set_algorithm(self.req, alg, fusion)
         if Bound.bulk_threshold is not None:
             self.iso.Iso_request_set_bulk_threshold(self.req, Bound.bulk_threshold)
@@ -309,6 +311,7 @@ def run_ours(args):
 
     peak, peak_kind = measured_peak()
     Bound.bulk_threshold = args.bulk_threshold
+    Bound.single_launch = args.single_launch
     reps = Replicas(torch, iso, wl, args.workload)
     b = reps.items[0]
 
@@ -350,7 +353,7 @@ def run_ours(args):
                          "(%.0f MB each, %.0f MB in all), timed back to back between one event pair"
                          % (len(reps.items), reps.footprint / 1e6, reps.footprint * len(reps.items) / 1e6),
                    "bytes": "value = bytes read + written by the schedule / device time"},
-        "gpu_launches": st["launches"] * args.steps,
+        "gpu_launches": iso.Iso_request_get_stats(b.req)["launches"] * args.steps,
         "frac_of_nominal_8TBs": per_gpu / NOMINAL_HBM_GBS,
     }
 
@@ -459,6 +462,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--headline-only", action="store_true",
                     help="time the headline schedule only (short runs under a profiler)")
+    ap.add_argument("--single-launch", action="store_true",
+                    help="run all phases in one cooperative launch instead of one launch per phase")
     ap.add_argument("--bulk-threshold", type=int, default=None,
                     help="override the size from which parts go to the bulk-copy kernel (0: never)")
     ap.add_argument("--traffic", type=float, default=None,

@@ -211,6 +211,21 @@ int Iso_request_set_algorithm(Iso_request request, int alg, int fusion_level);
  * schedules; the hop-by-hop schedule always alternates as in Algorithm 1.  Default: packed. */
 int Iso_request_set_layout(Iso_request request, int layout);
 
+/*
+ * One-launch execution.  When every launch of the schedule is a 16-byte vector launch on
+ * periodic dimensions, Iso_Start runs all phases in ONE cooperative kernel launch: the
+ * thread blocks go through the phases together and meet at a grid-wide barrier between
+ * them (the ordering point the paper gets from completing a round's MPI_Sendrecv), which
+ * saves the ramp-up and drain of one kernel per phase.  The barrier wait is bounded; if it
+ * expires the kernel stops and Iso_wait returns ISO_ERR_TIMEOUT.  enable = 0 goes back to
+ * one launch per phase, which is the default: with programmatic dependent launches between
+ * the phases the per-phase kernels were faster for schedules of two or three phases
+ * (40.8 against 48.5 microseconds on the 32^3 torus), the single launch only from about
+ * five phases on (285 against 302 microseconds on the 8^5 torus).  Iso_request_get_stats
+ * reports launches = 1 once the request has been started in this mode.
+ */
+int Iso_request_set_single_launch(Iso_request request, int enable);
+
 /* Parts of at least `bytes` bytes whose addresses and length are multiples of 16 are moved
  * by the bulk-copy kernel (asynchronous bulk copies staged through shared memory), the rest
  * by the vector kernel.  Default 512 (measured crossover: the bulk kernel wins from 512-byte

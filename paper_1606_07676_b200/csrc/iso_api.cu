@@ -40,6 +40,9 @@ void release_device(Request &r)
     if (r.d_blob) cudaFree(r.d_blob);
     if (r.d_inter) cudaFree(r.d_inter);
     if (r.d_err) cudaFree(r.d_err);
+    if (r.d_counter) cudaFree(r.d_counter);
+    r.d_counter = nullptr;
+    r.multi_grid = 0;
     if (r.h_err) cudaFreeHost(r.h_err);
     r.d_blob = nullptr;
     r.d_inter = nullptr;
@@ -123,6 +126,8 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
 
 int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
 
+LaunchDev make_launch_args(const Request &r, const LaunchPlan &L);
+
 // Uploads the lowered schedule and allocates the intermediate buffer.
 int materialise(Request &r)
 {
@@ -152,6 +157,16 @@ int materialise(Request &r)
         L.units_off = bytes;
         if (L.kernel == KERNEL_VEC) bytes += (size_t)L.units_per_proc * sizeof(UnitDev);
     }
+    // one-launch execution: every launch is a 16-byte vector launch on periodic dimensions
+    bool single = r.persistent && r.launches.size() >= 2;
+    for (const LaunchPlan &L : r.launches) {
+        if (L.kernel != KERNEL_VEC || L.width != 16) single = false;
+        for (int k = 0; k < L.n_used; ++k)
+            if (!c.periodic[L.used_dim[k]]) single = false;
+    }
+    bytes = (bytes + 127) / 128 * 128;
+    const size_t launches_off = bytes;
+    if (single) bytes += r.launches.size() * sizeof(LaunchDev);
     std::vector<unsigned char> blob(bytes ? bytes : 16, 0);
     for (const LaunchPlan &L : r.launches) {
         int used_index[ISO_MAX_DIMS];
@@ -204,6 +219,32 @@ int materialise(Request &r)
     if (r.d_blob) cudaFree(r.d_blob);
     r.d_blob = nullptr;
     ISO_CUDA(cudaMalloc(&r.d_blob, blob.size()));
+    r.multi_grid = 0;
+    if (single) {
+        if (!r.d_counter) {
+            ISO_CUDA(cudaMalloc((void **)&r.d_counter, sizeof(unsigned long long)));
+            ISO_CUDA(cudaMemset(r.d_counter, 0, sizeof(unsigned long long)));
+            r.epoch = 0;
+        }
+        // the grid must be resident as a whole: ask how many CTAs fit
+        const size_t smem = (sizeof(LaunchDev) + 127) / 128 * 128 + (size_t)kVecDepth * 256 * 16;
+        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows_multi<kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        int per_sm = 0;
+        ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_multi<kVecDepth>, 256, smem));
+        int want = 4;
+        if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
+            int v = std::atoi(env);
+            if (v >= 1 && v <= 8) want = v;
+        }
+        per_sm = std::min(per_sm, want);
+        if (per_sm >= 1) {
+            r.multi_grid = per_sm * r.sm_count;
+            r.multi_smem = smem;
+            r.multi_launches_off = launches_off;
+            LaunchDev *ld = reinterpret_cast<LaunchDev *>(blob.data() + launches_off);
+            for (size_t k = 0; k < r.launches.size(); ++k) ld[k] = make_launch_args(r, r.launches[k]);
+        }
+    }
     ISO_CUDA(cudaMemcpy(r.d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice));
     if (!r.d_err) {
         ISO_CUDA(cudaMalloc((void **)&r.d_err, sizeof(int)));
@@ -496,6 +537,18 @@ int Iso_request_set_layout(Iso_request request, int layout)
     return Iso_request_set_algorithm(request, request->alg, request->fusion);
 }
 
+int Iso_request_set_single_launch(Iso_request request, int enable)
+{
+    if (check_handle(request)) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    request->persistent = enable != 0;
+    request->dirty = true;
+    return ISO_SUCCESS;
+}
+
 int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
 {
     if (check_handle(request) || bytes < 0) return ISO_ERR_ARG;
@@ -524,6 +577,30 @@ int Iso_Start(Iso_request request, void *cuda_stream)
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     static const bool use_pdl = !(std::getenv("ISO_NO_PDL") && std::atoi(std::getenv("ISO_NO_PDL")) != 0);
+    if (r.multi_grid > 0) {
+        // all phases in one cooperative launch with grid barriers in between
+        MultiDev m{};
+        m.launches = reinterpret_cast<const LaunchDev *>(static_cast<unsigned char *>(r.d_blob) + r.multi_launches_off);
+        m.n = (int)r.launches.size();
+        m.counter = r.d_counter;
+        m.epoch = r.epoch;
+        m.err = r.d_err;
+        r.epoch += (unsigned long long)(m.n - 1) * (unsigned long long)r.multi_grid;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)r.multi_grid);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = r.multi_smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        ISO_CUDA(cudaLaunchKernelEx(&cfg, iso_gather_rows_multi<kVecDepth>, m));
+        r.last_stream = cuda_stream;
+        r.started = true;
+        return ISO_SUCCESS;
+    }
     for (const LaunchPlan &L : r.launches) {
         int rc = launch_one(r, L, stream, use_pdl);
         if (rc != ISO_SUCCESS) return rc;
@@ -562,6 +639,11 @@ int Iso_wait(Iso_request request)
     if (r.h_err && *r.h_err) {
         *r.h_err = 0;
         cudaMemsetAsync(r.d_err, 0, sizeof(int), stream);
+        if (r.d_counter) {
+            // a barrier gave up: start counting afresh
+            cudaMemsetAsync(r.d_counter, 0, sizeof(unsigned long long), stream);
+            r.epoch = 0;
+        }
         return ISO_ERR_TIMEOUT;
     }
     return ISO_SUCCESS;
@@ -571,6 +653,7 @@ int Iso_request_get_stats(Iso_request request, Iso_stats *out)
 {
     if (check_handle(request) || !out) return ISO_ERR_ARG;
     *out = request->stats;
+    if (!request->dirty && request->multi_grid > 0) out->launches = 1;
     return ISO_SUCCESS;
 }
 

@@ -83,6 +83,7 @@ struct Request {
     int fusion = 1;
     int64_t bulk_threshold = 512;
     int layout = ISO_LAYOUT_PACKED;
+    bool persistent = false;  // run all phases in one cooperative launch when the schedule allows
     const unsigned char *send = nullptr;
     unsigned char *recv = nullptr;
     int s = 0;
@@ -97,6 +98,10 @@ struct Request {
     unsigned char *d_inter = nullptr;
     int64_t d_inter_bytes = 0;
     int *d_err = nullptr;
+    unsigned long long *d_counter = nullptr;  // grid-barrier arrivals (one-launch execution)
+    unsigned long long epoch = 0;             // counter value at the next launch
+    int multi_grid = 0;                       // > 0: one-launch execution with this grid
+    size_t multi_smem = 0, multi_launches_off = 0;
     int *h_err = nullptr;
     void *last_stream = nullptr;
     bool started = false;

@@ -214,26 +214,32 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
 // must not exceed it; ISO_MAX_DIMS is the general case), MESH whether some of them are
 // non-periodic (then a row whose source lies outside the mesh is skipped).
 template <int W, int DEPTH, int NU, bool MESH>
-__global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant__ LaunchDev L)
+__device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned char *ring_base, bool dependent_launch)
 {
     using V = typename VecOf<W>::type;
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    V *const ring = reinterpret_cast<V *>(smem_raw) + threadIdx.x;  // slot k at ring[k * blockDim.x]
+    V *const ring = reinterpret_cast<V *>(ring_base) + threadIdx.x;  // slot k at ring[k * blockDim.x]
     V *const ring_end = ring + DEPTH * blockDim.x;
 
     const uint32_t CU = L.chunk_units, U = L.units_per_proc;
     const int G = (int)L.rows_per_pass;
     const int g = (int)(threadIdx.x / CU);
     const uint32_t ul = threadIdx.x - (uint32_t)g * CU;
-    grid_dependency_wait();
-    grid_launch_dependents();
     const long long r0 = (long long)G * blockIdx.x + g;
-    if (g >= G || r0 >= L.P) return;
+    const bool active = g < G && r0 < L.P && ul < U;
+    // the tables are not produced by kernels: fetch the first descriptor before ordering
+    // behind the previous kernel
+    UnitRegs R_first;
+    if (active) R_first = load_unit(L, ul);
+    if (dependent_launch) {
+        grid_dependency_wait();
+        grid_launch_dependents();
+    }
+    if (!active) return;
     const long long rstep = (long long)G * gridDim.x;
     const long long r_end = L.P;
 
     for (uint32_t u = ul; u < U; u += CU) {
-        const UnitRegs R = load_unit(L, u);
+        const UnitRegs R = u == ul ? R_first : load_unit(L, u);
         long long wrap_bytes[NU > 0 ? NU : 1];
 #pragma unroll
         for (int e = 0; e < NU; ++e) wrap_bytes[e] = (long long)L.used_wrap[e] * R.stride_s;
@@ -292,6 +298,80 @@ __global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant_
             if (slot == ring_end) slot = ring;
         }
         cp_async_wait<0>();
+    }
+}
+
+template <int W, int DEPTH, int NU, bool MESH>
+__global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant__ LaunchDev L)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    gather_rows_body<W, DEPTH, NU, MESH>(L, smem_raw, true);
+}
+
+// All phases of a schedule in ONE cooperative launch: the CTAs run phase after phase and
+// meet at a grid-wide barrier in between, which removes the launch ramp and drain of the
+// per-phase kernels.  Every launch of the schedule must be a 16-byte vector launch on
+// periodic dimensions.  The launch descriptors live in device memory and are copied to
+// shared memory phase by phase.
+struct MultiDev {
+    const LaunchDev *launches;
+    int n;
+    unsigned long long *counter;  // arrivals at the grid barrier, never reset
+    unsigned long long epoch;     // value of the counter when this launch began
+    int *err;                     // set to 2 when a barrier wait gives up
+};
+
+constexpr uint32_t kBarrierPolls = 1u << 22;
+
+// Grid-wide barrier for a cooperative launch (all CTAs are resident).  One thread per CTA
+// publishes the CTA's writes, counts itself in and polls the counter a bounded number of
+// times; on expiry it raises the error flag and every thread of the CTA gets `false`.
+__device__ __forceinline__ bool grid_barrier(const MultiDev &M, unsigned long long target, int *s_ok)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(M.counter, 1ULL);
+        bool ok = true;
+        uint32_t polls = 0;
+        for (;;) {
+            unsigned long long seen;
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(M.counter) : "memory");
+            if (seen >= target) break;
+            if (++polls >= kBarrierPolls) {
+                ok = false;
+                break;
+            }
+            __nanosleep(40);
+        }
+        __threadfence();
+        if (!ok) atomicExch(M.err, 2);
+        *s_ok = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return *s_ok != 0;
+}
+
+template <int DEPTH>
+__global__ void __launch_bounds__(256, 4) iso_gather_rows_multi(const __grid_constant__ MultiDev M)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ int s_ok;
+    LaunchDev *sL = reinterpret_cast<LaunchDev *>(smem_raw);
+    unsigned char *ring = smem_raw + ((sizeof(LaunchDev) + 127) / 128) * 128;
+    for (int ph = 0; ph < M.n; ++ph) {
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(M.launches + ph);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(sL);
+        for (uint32_t i = threadIdx.x; i < sizeof(LaunchDev) / 4; i += blockDim.x) dst[i] = __ldg(src + i);
+        __syncthreads();
+        switch (sL->n_used) {
+        case 0: gather_rows_body<16, DEPTH, 0, false>(*sL, ring, false); break;
+        case 1: gather_rows_body<16, DEPTH, 1, false>(*sL, ring, false); break;
+        case 2: gather_rows_body<16, DEPTH, 2, false>(*sL, ring, false); break;
+        case 3: gather_rows_body<16, DEPTH, 3, false>(*sL, ring, false); break;
+        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false>(*sL, ring, false); break;
+        }
+        if (ph + 1 < M.n && !grid_barrier(M, M.epoch + (unsigned long long)(ph + 1) * gridDim.x, &s_ok)) return;
     }
 }
 

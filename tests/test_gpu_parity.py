@@ -43,7 +43,8 @@ class Run:
         st = iso.Iso_request_get_stats(self.req)
         assert (st["send_stride"], st["recv_stride"]) == (ss, rs)
 
-    def result(self, alg, fusion, bulk=None):
+    def result(self, alg, fusion, bulk=None, single=False):
+        iso.Iso_request_set_single_launch(self.req, single)
         if fusion >= 100:
             iso.Iso_request_set_layout(self.req, iso.ISO_LAYOUT_ALTERNATING)
             fusion -= 100
@@ -63,12 +64,12 @@ class Run:
         iso.Iso_comm_free(self.comm)
 
 
-def check(torch, w, algs, bulk=None):
+def check(torch, w, algs, bulk=None, single=False):
     run = Run(torch, w)
     try:
         want = oracle_result(w, run.send_host)
         for alg, fusion in algs:
-            got = run.result(alg, fusion, bulk)
+            got = run.result(alg, fusion, bulk, single)
             bad = np.argwhere(got != want)
             assert bad.size == 0, "alg %d fusion %d: first mismatch at (rank, byte) %s" % (alg, fusion, bad[0])
     finally:
@@ -82,6 +83,21 @@ def test_cfg1(torch_cuda):
 
 def test_cfg2_alltoall(torch_cuda):
     check(torch_cuda, wl.config("cfg2_alltoall"), [COMB0, COMB1, COMB2, COMBD, ALT0, ALT1, DIRECT, TORUS])
+
+
+def test_all_phases_in_one_cooperative_launch(torch_cuda):
+    # opt-in execution mode: one cooperative launch with grid barriers between the phases
+    check(torch_cuda, wl.config("cfg2_alltoall"), [COMB0, COMB1, COMB2, ALT1, TORUS], single=True)
+    check(torch_cuda, wl.config("cfg2_allgather"), [COMB0, COMB1], single=True)
+    check(torch_cuda, wl.config("cfg3_m64"), [COMB0, COMB1, TORUS], single=True)
+    check(torch_cuda, wl.config("cfg4"), [COMB1], single=True)
+    check(torch_cuda, wl.Workload("ragged", "alltoall", (37, 53), wl.moore(2, 2), 48, seed=7), [COMB0, COMB1], single=True)
+    run = Run(torch_cuda, wl.config("cfg2_alltoall"))
+    run.result(*COMB1, single=True)
+    assert iso.Iso_request_get_stats(run.req)["launches"] == 1
+    run.result(*COMB1, single=False)
+    assert iso.Iso_request_get_stats(run.req)["launches"] == 3
+    run.close()
 
 
 def test_cfg2_allgather(torch_cuda):
