@@ -31,6 +31,10 @@ import numpy as np
 
 METRIC = "neighbor-alltoall effective GB/s (device-timed) and % of B200 HBM peak, combining vs direct"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + written) per launch of the dominant kernel, from the ncu capture
+# summarised in profiles/iso_gather_rows_cfg2_alltoall.md; only valid for that kernel build
+# and workload, so it is reported for the default workload and schedule only.
+TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_alltoall": 45.74e6}
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 512 << 20
 
@@ -57,7 +61,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -327,7 +331,10 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
     t1 = time.time()
-    clocks = sampler.stop(t0, t1) if sampler else None
+    clocks = None
+    if sampler is not None and (world > 1 or args.headline_only):
+        clocks = sampler.stop(t0, t1)
+        sampler = None
     if dist is not None:
         t = torch.tensor([ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -378,6 +385,10 @@ def run_ours(args):
                            "gbs_payload": s2["bytes_min"] / (m2 * 1e-3) / 1e9,
                            "frac_of_peak_moved": s2["bytes_moved"] / (m2 * 1e-3) / 1e9 / peak}
         st = reps.set(iso.ISO_ALG_COMBINING, args.fusion)
+        # clocks were sampled over all device-timed legs above (the headline leg alone
+        # lasts only steps x 40 microseconds)
+        clocks = sampler.stop(t0, time.time())
+        sampler = None
 
         # ---- end to end: host buffers in, host buffers out, through the C-ABI -----------
         hs = torch.empty(b.w.P * b.ss, dtype=torch.uint8).pin_memory()
@@ -401,7 +412,11 @@ def run_ours(args):
             "bound": "hbm", "kernel": kernel, "achieved": per_gpu, "peak": peak, "unit": "GB/s",
             "frac": per_gpu / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
             "bytes_per_launch": moved // launches, "avg_launch_ms": ms / launches,
-            "traffic": args.traffic,
+            "traffic": args.traffic if args.traffic is not None else (
+                TRAFFIC_BYTES_PER_LAUNCH.get(args.workload) if args.fusion == 1 and not args.single_launch
+                and args.bulk_threshold is None else None),
+            "traffic_note": "DRAM read+write bytes per launch (ncu, caches flushed before each launch); "
+                            "writes still held in L2 when the kernel ends are not in it",
             "note": "achieved = bytes read+written per launch / (step time / launches per step); "
                     "launch gaps are inside the step time",
         }
@@ -453,7 +468,7 @@ def sweep(torch, iso, wl, peak, args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_alltoall")
