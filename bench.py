@@ -125,6 +125,16 @@ def init_distributed(n_gpus: int):
     return rank, world, local, dist
 
 
+def max_over_ranks(dist, value: float, device) -> float:
+    """The slowest rank's time: what a multi-rank run reports."""
+    if dist is None:
+        return value
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 # ------------------------------------------------------------------------ reference arm
 def oracle_run(w, send):
     """One pass of the CPU oracle over the whole workload (only the CPU-baseline leg and the
@@ -335,10 +345,7 @@ def run_ours(args):
     if sampler is not None and (world > 1 or args.headline_only):
         clocks = sampler.stop(t0, t1)
         sampler = None
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(dist, ms, "cuda")
     moved, minimum = st["bytes_moved"], st["bytes_min"]
     value = world * moved / (ms * 1e-3) / 1e9
     per_gpu = moved / (ms * 1e-3) / 1e9
