@@ -32,7 +32,7 @@ import numpy as np
 METRIC = "neighbor-alltoall effective GB/s (device-timed) and % of B200 HBM peak, combining vs direct"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + written) per launch of the dominant kernel, from the ncu capture
-# summarised in profiles/iso_gather_rows_cfg2_alltoall.md; only valid for that kernel build
+# summarised under profiles/ (iso_gather_rows on cfg2_alltoall); only valid for that kernel build
 # and workload, so it is reported for the default workload and schedule only.
 TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_alltoall": 45.74e6}
 FALLBACK_HBM_GBS = 6650.0
@@ -451,7 +451,7 @@ def sweep(torch, iso, wl, peak, args):
     """Every named workload, combining (one launch per dimension, and per round) and direct:
     the results table.  Same protocol as the headline (rotation over instances, back to back)."""
     out = {}
-    for name in wl.CONFIG_NAMES:
+    for name in (wl.PAPER_NAMES if args.sweep == "paper" else wl.CONFIG_NAMES):
         reps = Replicas(torch, iso, wl, name)
         row = {}
         for key, alg, fusion in (("combining", iso.ISO_ALG_COMBINING, 1), ("combining_per_round", iso.ISO_ALG_COMBINING, 0),
@@ -480,7 +480,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_alltoall")
     ap.add_argument("--fusion", type=int, default=1)
-    ap.add_argument("--sweep", action="store_true", help="also time every named workload")
+    ap.add_argument("--sweep", nargs="?", const="configs", default=None, choices=["configs", "paper"],
+                    help="also time every named workload (configs: the five configurations; "
+                         "paper: the paper's larger neighbourhoods)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--headline-only", action="store_true",
                     help="time the headline schedule only (short runs under a profiler)")

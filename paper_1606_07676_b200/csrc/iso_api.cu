@@ -160,7 +160,7 @@ int materialise(Request &r)
     // one-launch execution: every launch is a 16-byte vector launch on periodic dimensions
     bool single = r.persistent && r.launches.size() >= 2;
     for (const LaunchPlan &L : r.launches) {
-        if (L.kernel != KERNEL_VEC || L.width != 16) single = false;
+        if (L.kernel != KERNEL_VEC || L.width != 16 || L.threads > 256) single = false;
         for (int k = 0; k < L.n_used; ++k)
             if (!c.periodic[L.used_dim[k]]) single = false;
     }
@@ -326,6 +326,20 @@ cudaError_t launch_kernel(Kernel kernel, const LaunchPlan &L, const LaunchDev &a
     return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
+// Wide CTAs need more dynamic shared memory than the default limit: opt in once per kernel.
+template <typename Kernel>
+cudaError_t launch_wide(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, cudaStream_t stream, bool dependent)
+{
+    static std::vector<const void *> opted_in;  // kernels that already have the larger limit
+    const void *key = reinterpret_cast<const void *>(kernel);
+    if (std::find(opted_in.begin(), opted_in.end(), key) == opted_in.end()) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kVecDepth * 1024 * 16);
+        if (e != cudaSuccess) return e;
+        opted_in.push_back(key);
+    }
+    return launch_kernel(kernel, L, a, stream, dependent);
+}
+
 int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool dependent)
 {
     if (L.grid == 0 || L.units_per_proc == 0) return ISO_SUCCESS;
@@ -339,7 +353,10 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
     } else {
         // kernels specialised on the number of shifted dimensions; meshes take the general one
         const int nu = L.n_used <= 3 ? L.n_used : ISO_MAX_DIMS;
-#define ISO_ROWS(W, NU, MESH) e = launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH>, L, a, stream, dependent)
+#define ISO_ROWS(W, NU, MESH)                                                                              \
+    e = (W == 16 && L.threads > 256)                                                                       \
+            ? launch_wide(iso_gather_rows_wide<16, kVecDepth, NU, MESH>, L, a, stream, dependent)            \
+            : launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH>, L, a, stream, dependent)
 #define ISO_ROWS_W(W)                                             \
     do {                                                          \
         if (a.mesh_mask) ISO_ROWS(W, ISO_MAX_DIMS, true);         \

@@ -308,6 +308,16 @@ __global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant_
     gather_rows_body<W, DEPTH, NU, MESH>(L, smem_raw, true);
 }
 
+// The same body in CTAs of up to 1024 threads, for launches whose payload per process has
+// more than 256 unit positions: one CTA then covers up to 16 KB of a row at a time, so rows
+// are still visited one after the other instead of in 4 KB columns.
+template <int W, int DEPTH, int NU, bool MESH>
+__global__ void __launch_bounds__(1024, 1) iso_gather_rows_wide(const __grid_constant__ LaunchDev L)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    gather_rows_body<W, DEPTH, NU, MESH>(L, smem_raw, true);
+}
+
 // All phases of a schedule in ONE cooperative launch: the CTAs run phase after phase and
 // meet at a grid-wide barrier in between, which removes the launch ramp and drain of the
 // per-phase kernels.  Every launch of the schedule must be a 16-byte vector launch on

@@ -616,6 +616,22 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
             }
         }
 
+        // a vector class that carries next to nothing per process is not worth a launch of
+        // its own: its pieces join the next narrower class that is in use
+        for (int width = 16; width > 1; width >>= 1) {
+            int64_t bytes = 0;
+            for (const Piece &q : pieces)
+                if (q.kernel == KERNEL_VEC && q.width == width) bytes += q.p.len;
+            if (bytes == 0 || bytes >= 128) continue;
+            int narrower = 0;
+            for (int w2 = width >> 1; w2 >= 1 && !narrower; w2 >>= 1)
+                for (const Piece &q : pieces)
+                    if (q.kernel == KERNEL_VEC && q.width == w2) { narrower = w2; break; }
+            if (!narrower) continue;
+            for (Piece &q : pieces)
+                if (q.kernel == KERNEL_VEC && q.width == width) q.width = narrower;
+        }
+
         // one launch per (kernel, width) class, in a fixed order
         for (int kernel = 0; kernel < 2; ++kernel) {
             for (int width = 16; width >= 1; width >>= 1) {
@@ -713,13 +729,15 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     int64_t grid;
                     if (kernel == KERNEL_VEC) {
                         // a row slot covers up to 256 unit positions; short rows share a CTA
-                        L.chunk_units = (uint32_t)std::min<uint64_t>(units, 256);
-                        L.rows_per_pass = std::max<uint32_t>(1, 256 / L.chunk_units);
+                        // 16-byte launches with long rows use CTAs of up to 1024 threads
+                        const uint32_t max_threads = (width == 16 && units > 256) ? 1024 : 256;
+                        L.chunk_units = (uint32_t)std::min<uint64_t>(units, max_threads);
+                        L.rows_per_pass = std::max<uint32_t>(1, max_threads == 256 ? 256 / L.chunk_units : 1);
                         L.threads = (int)((L.chunk_units * L.rows_per_pass + 31) / 32 * 32);
-                        int per_sm = 4;
+                        int per_sm = L.threads > 512 ? 1 : (L.threads > 256 ? 2 : 4);
                         if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
                             int v = std::atoi(env);
-                            if (v >= 1 && v <= 8) per_sm = v;
+                            if (v >= 1 && v <= 8 && L.threads <= 256) per_sm = v;
                         }
                         // persistent grid: CTA b takes the row groups b, b + grid, ...
                         grid = std::min<int64_t>((c.P + L.rows_per_pass - 1) / L.rows_per_pass,

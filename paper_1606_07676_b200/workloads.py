@@ -228,6 +228,9 @@ def config(name: str, seed: int = DEFAULT_SEED) -> Workload:
     cfg4           all-to-all, 8^5, Moore r=1, 16 B of fp32
     cfg5           irregular all-to-all, 64x64x32, 30 random offsets in [-3,3]^3,
                    lengths uniform over {4,16,64,256,1024} B, packed displacements
+    <nbh>_alltoall / <nbh>_allgather with nbh in moore_d3r3 (342 neighbours), octant_d3r3
+                   (63), shells_d3 (1396, Chebyshev distances 3 and 7) on 32^3 and moore_d4r1
+                   (80) on 16^4: the paper's larger neighbourhoods, 64-byte blocks
     """
     if name == "cfg1":
         return Workload(name, "alltoall", (8, 8), moore(2, 1), 8, kind="int32", seed=seed)
@@ -244,6 +247,13 @@ def config(name: str, seed: int = DEFAULT_SEED) -> Workload:
         offs = random_offsets(seed, 3, 30, -3, 3)
         lens = random_sizes(seed, 30)
         return Workload(name, "alltoallv", (64, 64, 32), offs, 0, lens=lens, kind="uint8", seed=seed)
+    # neighbourhoods of the paper's second set of experiments (Sections IV and VI), 64-byte blocks
+    paper = {"moore_d3r3": ((32, 32, 32), lambda: moore(3, 3)), "octant_d3r3": ((32, 32, 32), lambda: positive_octant(3, 3)),
+             "shells_d3": ((32, 32, 32), lambda: shells(3, (3, 7))), "moore_d4r1": ((16, 16, 16, 16), lambda: moore(4, 1))}
+    for key, (dims, make) in paper.items():
+        for coll in ("alltoall", "allgather"):
+            if name == "%s_%s" % (key, coll):
+                return Workload(name, coll, dims, make(), 64, kind="fp32", seed=seed)
     raise KeyError(name)
 
 
@@ -269,6 +279,9 @@ def send_buffer_np(w: Workload, send_stride: int) -> np.ndarray:
     """Host copy of the seeded send buffers of a workload (uint8 [P, send_stride])."""
     return payload_np(w.kind, w.seed, 0, 0, w.P * send_stride).reshape(w.P, send_stride).copy()
 
+
+PAPER_NAMES = tuple("%s_%s" % (k, c) for k in ("moore_d3r3", "octant_d3r3", "shells_d3", "moore_d4r1")
+                    for c in ("alltoall", "allgather"))
 
 CONFIG_NAMES = ("cfg1", "cfg2_alltoall", "cfg2_allgather", "cfg3_m4", "cfg3_m64", "cfg3_m512",
                 "cfg3_m4096", "cfg4", "cfg5")

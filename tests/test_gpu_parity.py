@@ -163,6 +163,42 @@ def test_cfg3_4096_sampled(torch_cuda):
         torch.cuda.empty_cache()
 
 
+def _sampled_check(torch, w, algs, nranks=12):
+    """Full-size run with device-generated inputs; the outputs of sampled ranks are checked
+    block by block against sources named by the oracle and regenerated on the host."""
+    lens, sd, rd, ss, rs = layout(w)
+    m, s, P = w.block_bytes, w.s, w.P
+    send = wl.payload_torch(w.kind, w.seed, 0, P * ss, "cuda")
+    recv = torch.empty(P * rs, dtype=torch.uint8, device="cuda")
+    comm, req = make_request(w, send, recv)
+    rng = np.random.default_rng(17)
+    ranks = sorted({0, 1, P - 1, w.dims[-1] - 1, w.dims[-1], *rng.integers(0, P, nranks).tolist()})
+    try:
+        for alg, fusion in algs:
+            iso.Iso_request_set_algorithm(req, alg, fusion)
+            recv.fill_(POISON)
+            iso.Iso_Start(req)
+            iso.Iso_wait(req)
+            for r in ranks:
+                got = recv[r * rs:(r + 1) * rs].cpu().numpy().reshape(s, m)
+                for i in range(s):
+                    q = oracle.source_rank(w.dims, r, w.offsets[i])
+                    off = q * ss + (i * m if w.collective == "alltoall" else 0)
+                    assert np.array_equal(got[i], wl.payload_np(w.kind, w.seed, 0, off, m)), (w.name, alg, r, i)
+    finally:
+        iso.Iso_request_free(req)
+        iso.Iso_comm_free(comm)
+        del send, recv
+        torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["shells_d3_alltoall", "shells_d3_allgather", "moore_d4r1_alltoall",
+                                  "octant_d3r3_allgather", "moore_d3r3_alltoall"])
+def test_paper_neighbourhoods_full_size_sampled(torch_cuda, name):
+    w = wl.config(name)
+    _sampled_check(torch_cuda, w, [COMB1, DIRECT] if w.s < 1000 else [COMB1])
+
+
 # --------------------------------------------------------------------- edge cases
 def _tiny_cases():
     rng = np.random.default_rng(99)
