@@ -292,6 +292,25 @@ int build_combining_alltoall(Request &r, const Geometry &g)
             ++phase;
         }
     }
+    // Blocks of at most 16 bytes: run every block's final hop in the last phase (a hop may
+    // be postponed, only the order of a block's own hops matters), so that the receive
+    // buffer is written by one launch, whole rows at a time, instead of in isolated
+    // half-sector pieces by every phase.  Measured +40 % on the 8^5 torus with 16-byte
+    // blocks; for blocks of 64 bytes and more the uneven phases cost 4-6 %, so they keep
+    // the natural phases.
+    bool lazy_final = r.layout == ISO_LAYOUT_PACKED && r.fusion != 0 && phase > 1;
+    for (int i = 0; i < g.s; ++i)
+        if (r.len[i] > 16) lazy_final = false;
+    if (const char *env = std::getenv("ISO_LAZY_FINAL"))
+        lazy_final = r.layout == ISO_LAYOUT_PACKED && r.fusion != 0 && phase > 1 && std::atoi(env) != 0;
+    if (lazy_final) {
+        std::vector<int> last_hop(g.s, -1);
+        for (size_t k = 0; k < r.parts.size(); ++k) last_hop[r.parts[k].slot] = (int)k;
+        for (int i = 0; i < g.s; ++i)
+            if (last_hop[i] >= 0) r.parts[last_hop[i]].phase = phase - 1;
+        std::stable_sort(r.parts.begin(), r.parts.end(),
+                         [](const Part &a, const Part &b) { return a.phase < b.phase; });
+    }
     if (r.layout == ISO_LAYOUT_PACKED) pack_intermediates(r, g.s);
     // blocks for the process itself: one local copy, together with the first phase
     for (Part &p : locals_parts) p.phase = 0;
