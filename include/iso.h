@@ -253,8 +253,15 @@ int Iso_Start(Iso_request request, void *cuda_stream);
 
 /* Same with HOST buffers holding all P processes' send / receive buffers in the layout
  * above: copies `host_sendbuf` to the request's device send buffer, runs the schedule and
- * copies the device receive buffer to `host_recvbuf`, all on `cuda_stream`.  The copies are
- * asynchronous when the host memory is page-locked.  Complete after Iso_wait. */
+ * copies the device receive buffer to `host_recvbuf`.  When only blocks read from the send
+ * buffer move along dimension 0 (true for the combining and direct schedules on periodic
+ * tori with at least four planes) the work is pipelined over up to eight slabs of
+ * dimension 0: a slab's schedule runs as soon as the slabs it reads from have arrived and
+ * its receive buffers travel back while later slabs are still being uploaded (uploads and
+ * downloads on two internal streams created by the first such call, kernels on
+ * `cuda_stream`, which is made to wait for the downloads).  Otherwise: one upload, the
+ * schedule, one download, all on `cuda_stream`.  The copies are asynchronous when the host
+ * memory is page-locked.  Complete after Iso_wait or a synchronisation of `cuda_stream`. */
 int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_recvbuf,
                    void *cuda_stream);
 

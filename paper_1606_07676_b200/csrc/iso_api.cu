@@ -40,6 +40,12 @@ void release_device(Request &r)
     if (r.d_blob) cudaFree(r.d_blob);
     if (r.d_inter) cudaFree(r.d_inter);
     if (r.d_err) cudaFree(r.d_err);
+    if (r.copy_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.copy_stream));
+    if (r.up_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.up_stream));
+    r.up_stream = nullptr;
+    for (void *e : r.slab_events) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+    r.copy_stream = nullptr;
+    r.slab_events.clear();
     if (r.d_counter) cudaFree(r.d_counter);
     r.d_counter = nullptr;
     r.multi_grid = 0;
@@ -278,6 +284,8 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
     a.buf_stride[ISO_BUF_RECV] = r.recv_stride;
     a.buf_stride[ISO_BUF_INTER] = r.inter_stride;
     a.P = c.P;
+    a.row_lo = 0;
+    a.row_hi = c.P;
     a.err = r.d_err;
     a.nparts = (uint32_t)L.parts.size();
     a.units_per_proc = L.units_per_proc;
@@ -308,11 +316,23 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
     return a;
 }
 
+// Grid for the rows [a.row_lo, a.row_hi): the plan's grid scaled to the share of the rows.
+unsigned grid_for_rows(const LaunchPlan &L, const LaunchDev &a)
+{
+    const long long rows = a.row_hi - a.row_lo;
+    if (rows >= a.P) return (unsigned)L.grid;
+    if (L.kernel == KERNEL_BULK) return (unsigned)((rows + L.tile_procs - 1) / L.tile_procs);
+    const long long groups = (rows + L.rows_per_pass - 1) / L.rows_per_pass;
+    long long g = (L.grid * rows + a.P - 1) / a.P;
+    g = std::max<long long>(1, std::min(g, groups));
+    return (unsigned)g;
+}
+
 template <typename Kernel>
 cudaError_t launch_kernel(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, cudaStream_t stream, bool dependent)
 {
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)L.grid);
+    cfg.gridDim = dim3(grid_for_rows(L, a));
     cfg.blockDim = dim3((unsigned)L.threads);
     cfg.dynamicSmemBytes = L.smem;
     cfg.stream = stream;
@@ -340,10 +360,16 @@ cudaError_t launch_wide(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, 
     return launch_kernel(kernel, L, a, stream, dependent);
 }
 
-int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool dependent)
+int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool dependent, long long row_lo = 0,
+               long long row_hi = -1)
 {
     if (L.grid == 0 || L.units_per_proc == 0) return ISO_SUCCESS;
     LaunchDev a = make_launch_args(r, L);
+    if (row_hi >= 0) {
+        a.row_lo = row_lo;
+        a.row_hi = row_hi;
+        if (row_hi <= row_lo) return ISO_SUCCESS;
+    }
     cudaError_t e;
     if (L.kernel == KERNEL_BULK) {
         e = launch_kernel(iso_gather_bulk, L, a, stream, dependent);
@@ -374,6 +400,52 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
     }
     ISO_CUDA(e);
     return ISO_SUCCESS;
+}
+
+// Slabs of the leading dimension for the pipelined host-buffer path.
+struct SlabPlan {
+    long long row_lo, row_hi;
+    int last_needed;  // index of the last slab whose send buffers this slab's schedule reads
+};
+
+// Fills `slabs` when the schedule can run slab by slab: every part that shifts along
+// dimension 0 must read the send buffer (everything else then stays inside a plane of
+// dimension 0), all dimensions periodic, and at least four planes.  Leaves it empty otherwise.
+void plan_slabs(const Request &r, std::vector<SlabPlan> &slabs)
+{
+    const Comm &c = *r.comm;
+    slabs.clear();
+    const int p0 = c.dims[0];
+    if (c.d < 2 || p0 < 4 || r.launches.empty()) return;
+    for (int j = 0; j < c.d; ++j)
+        if (!c.periodic[j]) return;
+    std::vector<int> shifts;  // distinct shifts along dimension 0 (0 included)
+    shifts.push_back(0);
+    for (const LaunchPlan &L : r.launches)
+        for (const LoweredPart &lp : L.parts) {
+            const int s0 = lp.p.shift[0];
+            if (s0 == 0) continue;
+            if (lp.p.src_buf != ISO_BUF_SEND) return;
+            if (std::find(shifts.begin(), shifts.end(), s0) == shifts.end()) shifts.push_back(s0);
+        }
+    int n = std::min(p0, 8);
+    if (const char *env = std::getenv("ISO_HOST_SLABS")) {
+        int v = std::atoi(env);
+        if (v <= 1) return;
+        n = std::min(p0, v);
+    }
+    const long long plane = c.rank_stride[0];
+    std::vector<int> slab_of(p0);
+    for (int k = 0; k < n; ++k) {
+        const int a = (int)((long long)p0 * k / n), b = (int)((long long)p0 * (k + 1) / n);
+        for (int x = a; x < b; ++x) slab_of[x] = k;
+        slabs.push_back(SlabPlan{a * plane, b * plane, k});
+    }
+    for (int x = 0; x < p0; ++x)
+        for (int s0 : shifts) {
+            const int src = ((x - s0) % p0 + p0) % p0;
+            slabs[slab_of[x]].last_needed = std::max(slabs[slab_of[x]].last_needed, slab_of[src]);
+        }
 }
 
 int check_handle(Iso_request request)
@@ -634,12 +706,79 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
     if (!r.send || !r.recv) return ISO_ERR_STATE;
     const Comm &c = *r.comm;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t sbytes = (size_t)(c.P * r.send_stride), rbytes = (size_t)(c.P * r.recv_stride);
-    if (sbytes)
-        ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send), host_sendbuf, sbytes, cudaMemcpyHostToDevice, stream));
-    int rc = Iso_Start(request, cuda_stream);
-    if (rc != ISO_SUCCESS) return rc;
-    if (rbytes) ISO_CUDA(cudaMemcpyAsync(host_recvbuf, r.recv, rbytes, cudaMemcpyDeviceToHost, stream));
+    if (r.dirty) {
+        if (r.started) {
+            int rc = Iso_wait(request);
+            if (rc != ISO_SUCCESS) return rc;
+        }
+        int rc = materialise(r);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    const unsigned char *hs = static_cast<const unsigned char *>(host_sendbuf);
+    unsigned char *hr = static_cast<unsigned char *>(host_recvbuf);
+    std::vector<SlabPlan> slabs;
+    if (r.multi_grid == 0) plan_slabs(r, slabs);
+    if (slabs.empty()) {
+        // no pipelining possible: copy in, run, copy out
+        const size_t sbytes = (size_t)(c.P * r.send_stride), rbytes = (size_t)(c.P * r.recv_stride);
+        if (sbytes)
+            ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send), hs, sbytes, cudaMemcpyHostToDevice, stream));
+        int rc = Iso_Start(request, cuda_stream);
+        if (rc != ISO_SUCCESS) return rc;
+        if (rbytes) ISO_CUDA(cudaMemcpyAsync(hr, r.recv, rbytes, cudaMemcpyDeviceToHost, stream));
+        return ISO_SUCCESS;
+    }
+
+    // Pipelined over slabs of the leading dimension.  Only blocks read from the send buffer
+    // cross slabs, so a slab's whole schedule can run as soon as the send buffers of the
+    // slabs it reads have arrived, and its receive buffers can travel back while later
+    // slabs are still on their way in.  Three streams: uploads back to back on one, kernels
+    // on the caller's stream, downloads on a third, so that both directions of the link are
+    // busy at the same time and no copy waits behind a kernel.
+    const size_t S = slabs.size();
+    if (!r.copy_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.copy_stream), cudaStreamNonBlocking));
+    if (!r.up_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.up_stream), cudaStreamNonBlocking));
+    cudaStream_t down = static_cast<cudaStream_t>(r.copy_stream), up = static_cast<cudaStream_t>(r.up_stream);
+    while (r.slab_events.size() < 2 * S + 1) {
+        cudaEvent_t e;
+        ISO_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        r.slab_events.push_back(e);
+    }
+    // copies of this call must not overtake earlier work on the caller's stream
+    cudaEvent_t fence = static_cast<cudaEvent_t>(r.slab_events[2 * S]);
+    ISO_CUDA(cudaEventRecord(fence, stream));
+    ISO_CUDA(cudaStreamWaitEvent(up, fence, 0));
+    ISO_CUDA(cudaStreamWaitEvent(down, fence, 0));
+    static const bool use_pdl = !(std::getenv("ISO_NO_PDL") && std::atoi(std::getenv("ISO_NO_PDL")) != 0);
+    std::vector<char> done(S, 0);
+    for (size_t upi = 0; upi < S; ++upi) {
+        const SlabPlan &u = slabs[upi];
+        const size_t off = (size_t)(u.row_lo * r.send_stride), n = (size_t)((u.row_hi - u.row_lo) * r.send_stride);
+        if (n) ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send) + off, hs + off, n, cudaMemcpyHostToDevice, up));
+        cudaEvent_t arrived = static_cast<cudaEvent_t>(r.slab_events[S + upi]);
+        ISO_CUDA(cudaEventRecord(arrived, up));
+        // every slab whose last needed upload this was
+        for (size_t k = 0; k < S; ++k) {
+            if (done[k] || slabs[k].last_needed > (int)upi) continue;
+            const SlabPlan &w = slabs[k];
+            ISO_CUDA(cudaStreamWaitEvent(stream, arrived, 0));
+            for (const LaunchPlan &L : r.launches) {
+                int rc = launch_one(r, L, stream, use_pdl, w.row_lo, w.row_hi);
+                if (rc != ISO_SUCCESS) return rc;
+            }
+            cudaEvent_t ev = static_cast<cudaEvent_t>(r.slab_events[k]);
+            ISO_CUDA(cudaEventRecord(ev, stream));
+            ISO_CUDA(cudaStreamWaitEvent(down, ev, 0));
+            const size_t roff = (size_t)(w.row_lo * r.recv_stride), rn = (size_t)((w.row_hi - w.row_lo) * r.recv_stride);
+            if (rn) ISO_CUDA(cudaMemcpyAsync(hr + roff, r.recv + roff, rn, cudaMemcpyDeviceToHost, down));
+            done[k] = 1;
+        }
+    }
+    // join: the caller's stream is complete only when the downloads are
+    ISO_CUDA(cudaEventRecord(fence, down));
+    ISO_CUDA(cudaStreamWaitEvent(stream, fence, 0));
+    r.last_stream = cuda_stream;
+    r.started = true;
     return ISO_SUCCESS;
 }
 

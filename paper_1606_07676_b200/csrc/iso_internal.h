@@ -105,6 +105,9 @@ struct Request {
     int *h_err = nullptr;
     void *last_stream = nullptr;
     bool started = false;
+    void *copy_stream = nullptr;       // download stream of the pipelined host-buffer path
+    void *up_stream = nullptr;         // its upload stream
+    std::vector<void *> slab_events;   // its events
     int sm_count = 148;  // replaced by the device's count when the request is materialised
 };
 

@@ -53,6 +53,7 @@ struct LaunchDev {
     unsigned char *buf[3];   // send, recv, inter
     long long buf_stride[3];
     long long P;
+    long long row_lo, row_hi;  // the processes this launch works on: ranks [row_lo, row_hi)
     int *err;                // device error flag (bulk kernel time-outs)
     uint32_t nparts;
     uint32_t units_per_proc;
@@ -224,8 +225,8 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
     const int G = (int)L.rows_per_pass;
     const int g = (int)(threadIdx.x / CU);
     const uint32_t ul = threadIdx.x - (uint32_t)g * CU;
-    const long long r0 = (long long)G * blockIdx.x + g;
-    const bool active = g < G && r0 < L.P && ul < U;
+    const long long r0 = L.row_lo + (long long)G * blockIdx.x + g;
+    const bool active = g < G && r0 < L.row_hi && ul < U;
     // the tables are not produced by kernels: fetch the first descriptor before ordering
     // behind the previous kernel
     UnitRegs R_first;
@@ -236,7 +237,7 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
     }
     if (!active) return;
     const long long rstep = (long long)G * gridDim.x;
-    const long long r_end = L.P;
+    const long long r_end = L.row_hi;
 
     for (uint32_t u = ul; u < U; u += CU) {
         const UnitRegs R = u == ul ? R_first : load_unit(L, u);
@@ -397,20 +398,20 @@ __global__ void __launch_bounds__(256) iso_gather_rows_reg(const __grid_constant
     const uint32_t ul = threadIdx.x - (uint32_t)g * CU;
     grid_dependency_wait();
     grid_launch_dependents();
-    const long long r0 = (long long)G * blockIdx.x + g;
-    if (g >= G || r0 >= L.P) return;
+    const long long r0 = L.row_lo + (long long)G * blockIdx.x + g;
+    if (g >= G || r0 >= L.row_hi) return;
     const long long rstep = (long long)G * gridDim.x;
 
     for (uint32_t u = ul; u < U; u += CU) {
         const UnitRegs R = load_unit(L, u);
-        for (long long rb = r0; rb < L.P; rb += rstep * UNROLL) {
+        for (long long rb = r0; rb < L.row_hi; rb += rstep * UNROLL) {
             V val[UNROLL];
             V *dst[UNROLL];
 #pragma unroll
             for (int k = 0; k < UNROLL; ++k) {
                 const long long r = rb + k * rstep;
                 dst[k] = nullptr;
-                if (r < L.P) {
+                if (r < L.row_hi) {
                     long long wrap = 0;
                     bool valid = true;
                     for (int e = 0; e < L.n_used; ++e) {
@@ -507,9 +508,9 @@ __global__ void __launch_bounds__(256) iso_gather_bulk(const __grid_constant__ L
     uint32_t *s_coord =
         reinterpret_cast<uint32_t *>(smem_raw + (size_t)blockDim.x * 2 * chunk + (size_t)blockDim.x * 16);
 
-    const long long r0 = (long long)blockIdx.x * L.tile_procs;
-    const long long left = L.P - r0;
-    const int np = (int)(left < L.tile_procs ? left : L.tile_procs);
+    const long long r0 = L.row_lo + (long long)blockIdx.x * L.tile_procs;
+    const long long left = L.row_hi - r0;
+    const int np = left <= 0 ? 0 : (int)(left < L.tile_procs ? left : L.tile_procs);
     tile_coordinates(L, r0, np, s_coord);
     uint64_t *bar = s_bar + 2 * threadIdx.x;
     unsigned char *stage = s_data + (size_t)threadIdx.x * 2 * chunk;

@@ -305,3 +305,49 @@ def test_persistent_request_streams_and_host_buffers(torch_cuda):
     iso.Iso_wait(run.req)
     assert np.array_equal(hr.numpy(), want)
     run.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2_alltoall", "cfg2_allgather", "cfg3_m64", "cfg5"])
+def test_host_buffers_pipelined_over_slabs(torch_cuda, name):
+    """Iso_Start_host uploads, runs and downloads slab by slab along dimension 0; the result
+    must not depend on that, for every schedule, twice in a row with different contents."""
+    torch = torch_cuda
+    w = wl.config(name)
+    if name == "cfg5":
+        w = wl.Workload("v", "alltoallv", (16, 8, 8), w.offsets, 0, lens=w.lens, seed=5)
+    run = Run(torch, w)
+    hs = torch.from_numpy(run.send_host).pin_memory()
+    hr = torch.empty((w.P, run.rs), dtype=torch.uint8).pin_memory()
+    algs = [COMB1, COMB0, ALT1, DIRECT] + ([TORUS] if w.collective == "alltoall" else [])
+    if w.collective == "allgather":
+        algs = [COMB1, DIRECT]
+    try:
+        for seed_shift, (alg, fusion) in enumerate(algs):
+            contents = wl.send_buffer_np(wl.Workload(w.name, w.collective, w.dims, w.offsets, w.block_bytes, lens=w.lens,
+                                                     kind=w.kind, seed=w.seed + seed_shift), run.ss)
+            hs.copy_(torch.from_numpy(contents))
+            want = oracle_result(w, contents)
+            if fusion >= 100:
+                iso.Iso_request_set_layout(run.req, iso.ISO_LAYOUT_ALTERNATING)
+                fusion -= 100
+            else:
+                iso.Iso_request_set_layout(run.req, iso.ISO_LAYOUT_PACKED)
+            iso.Iso_request_set_algorithm(run.req, alg, fusion)
+            run.recv.fill_(POISON)
+            hr.fill_(0)
+            torch.cuda.synchronize()
+            iso.Iso_Start_host(run.req, hs, hr)
+            iso.Iso_wait(run.req)
+            got = hr.numpy()
+            if w.collective == "alltoallv":
+                # bytes of the stride that no block covers are whatever the device buffer held
+                covered = np.zeros(run.rs, bool)
+                lens, sd, rd, ss, rs = layout(w)
+                for i in range(w.s):
+                    covered[rd[i]:rd[i] + lens[i]] = True
+                assert np.array_equal(got[:, covered], want[:, covered]), (name, alg)
+            else:
+                assert np.array_equal(got, want), (name, alg)
+    finally:
+        run.close()
+
