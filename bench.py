@@ -472,6 +472,34 @@ def sweep(torch, iso, wl, peak, args):
     return out
 
 
+def run_init_times(args):
+    """Host-side set-up times on the grid of the paper's Table II (Moore neighbourhoods, d = 2..5,
+    r = 1..3, 480 processes): neighbourhood creation and all-to-all init (schedule computation and
+    lowering; no device is touched).  Median of 400 calls, milliseconds."""
+    from paper_1606_07676_b200 import binding as iso
+    from paper_1606_07676_b200 import workloads as wl
+    dims_for = {2: (24, 20), 3: (10, 8, 6), 4: (6, 5, 4, 4), 5: (5, 4, 4, 3, 2)}
+    out = {}
+    for d, dims in dims_for.items():
+        for r_ in (1, 2, 3):
+            offs = wl.moore(d, r_)
+            t_create, t_init = [], []
+            for _ in range(args.steps if args.steps < 1000 else 400):
+                t0 = time.perf_counter()
+                comm = iso.Iso_neighborhood_create(dims, offs)
+                t1 = time.perf_counter()
+                req = iso.Iso_neighbor_alltoall_init(None, 1, 4, None, 1, 4, comm)
+                t2 = time.perf_counter()
+                iso.Iso_request_free(req)
+                iso.Iso_comm_free(comm)
+                t_create.append((t1 - t0) * 1e3)
+                t_init.append((t2 - t1) * 1e3)
+            out["d%d_r%d" % (d, r_)] = {"s": int(len(offs)), "create_ms": statistics.median(t_create),
+                                        "alltoall_init_ms": statistics.median(t_init)}
+    print(json.dumps({"init_times": out, "unit": "ms", "note": "host only, median of repeated calls"}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -492,7 +520,11 @@ def main():
                     help="override the size from which parts go to the bulk-copy kernel (0: never)")
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture, if one is current")
+    ap.add_argument("--init-times", action="store_true",
+                    help="print host-side set-up times on the grid of the paper's Table II and exit")
     args = ap.parse_args()
+    if args.init_times:
+        return run_init_times(args)
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         return run_reference(args)
