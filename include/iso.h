@@ -126,7 +126,9 @@ typedef struct Iso_part {
     int64_t src_off;
     int64_t dst_off;
     int64_t len;
-    int shift[ISO_MAX_DIMS]; /* per dimension, reduced to [0, p_j) */
+    int shift[ISO_MAX_DIMS]; /* per dimension, reduced to [0, p_j); signed on non-periodic dimensions */
+    int check[ISO_MAX_DIMS]; /* non-periodic dimensions: process x takes part only if
+                                0 <= x_j - check_j < p_j (0: no condition) */
 } Iso_part;
 
 /*
@@ -233,11 +235,15 @@ int Iso_request_set_single_launch(Iso_request request, int enable);
 int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes);
 
 /*
- * Non-periodic dimensions (the extension Section VII mentions).  periodic[j] = 0 makes dimension j a mesh: a block whose source
- * R - C^i falls outside the mesh is not delivered and the receive slot keeps its previous
- * contents.  Only ISO_ALG_DIRECT supports meshes, and requests created from a neighbourhood
- * with a mesh dimension start with that schedule.  Call it before creating requests.
- * Default: all dimensions periodic.
+ * Non-periodic dimensions (the extension Section VII mentions).  periodic[j] = 0 makes
+ * dimension j a mesh: a block whose source R - C^i falls outside the mesh is not delivered
+ * and the receive slot keeps its previous contents.  Supported by ISO_ALG_DIRECT (all
+ * collectives) and by ISO_ALG_COMBINING for the all-to-all collectives: every hop of a block
+ * is skipped for the processes on whose route the original sender or the final receiver
+ * would lie outside (always with the packed layout: the receive buffer cannot double as
+ * scratch when undelivered slots must keep their contents).  Allgather requests on a mesh
+ * start with the direct schedule.  Call it
+ * before creating requests.  Default: all dimensions periodic.
  */
 int Iso_comm_set_periodic(Iso_comm isocomm, const int periodic[]);
 

@@ -58,11 +58,12 @@ class Iso_part(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
                 ("phase", "round", "slot", "src_buf", "dst_buf", "kernel", "width", "reserved")] + \
                [(n, ctypes.c_int64) for n in ("src_off", "dst_off", "len")] + \
-               [("shift", ctypes.c_int * ISO_MAX_DIMS)]
+               [("shift", ctypes.c_int * ISO_MAX_DIMS), ("check", ctypes.c_int * ISO_MAX_DIMS)]
 
     def as_dict(self) -> dict:
-        d = {n: int(getattr(self, n)) for n, _ in self._fields_ if n not in ("shift", "reserved")}
+        d = {n: int(getattr(self, n)) for n, _ in self._fields_ if n not in ("shift", "check", "reserved")}
         d["shift"] = list(self.shift)
+        d["check"] = list(self.check)
         return d
 
 

@@ -120,7 +120,7 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
     comm->refcount++;
     r->kind = kind;
     for (int j = 0; j < comm->d; ++j)
-        if (!comm->periodic[j]) r->alg = ISO_ALG_DIRECT;  // meshes: only the direct schedule
+        if (!comm->periodic[j] && kind == ISO_KIND_ALLGATHER) r->alg = ISO_ALG_DIRECT;  // mesh allgather: direct only
     r->send = static_cast<const unsigned char *>(sendbuf);
     r->recv = static_cast<unsigned char *>(recvbuf);
     r->s = comm->s;
@@ -192,10 +192,12 @@ int materialise(Request &r)
             long long delta = 0;
             int nnz = 0;
             for (int j = 0; j < c.d; ++j) {
-                if (!lp.p.shift[j]) continue;
+                // periodic dimension: the shift (wrap test); mesh dimension: the check value
+                const int value = c.periodic[j] ? lp.p.shift[j] : lp.p.check[j];
                 delta -= (long long)lp.p.shift[j] * c.rank_stride[j];
+                if (!value) continue;
                 d.dim[nnz] = (uint8_t)used_index[j];
-                d.c[nnz] = lp.p.shift[j];
+                d.c[nnz] = value;
                 ++nnz;
             }
             d.nnz = (uint8_t)nnz;
@@ -832,6 +834,7 @@ int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int 
                 q.dst_off = lp.p.dst_off;
                 q.len = lp.p.len;
                 std::memcpy(q.shift, lp.p.shift, sizeof(q.shift));
+                std::memcpy(q.check, lp.p.check, sizeof(q.check));
                 out[n] = q;
             }
             ++n;

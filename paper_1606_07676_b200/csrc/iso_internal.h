@@ -30,6 +30,7 @@ struct Part {
     int64_t dst_off = 0;
     int64_t len = 0;
     int shift[ISO_MAX_DIMS] = {0};  // residue in [0,p_j) for periodic dimensions, signed for mesh ones
+    int check[ISO_MAX_DIMS] = {0};  // mesh dimensions: process x takes part only if 0 <= x_j - check_j < p_j
 };
 
 // Exact unsigned 32-bit division by an invariant divisor (Granlund & Montgomery 1994,

@@ -135,6 +135,8 @@ int build_direct(Request &r, const Geometry &g)
         p.dst_off = r.rdispl[i];
         p.len = r.len[i];
         std::memcpy(p.shift, v, sizeof(int) * g.d);
+        for (int j = 0; j < g.d; ++j)
+            if (!c.periodic[j]) p.check[j] = v[j];
         r.parts.push_back(p);
         if (zero) ++locals; else ++parts;
     }
@@ -252,25 +254,32 @@ int build_combining_alltoall(Request &r, const Geometry &g)
     const Comm &c = *r.comm;
     const Groups gr = make_groups(g.d, r.fusion);
     std::vector<int> hops(g.s, 0);
-    for (int i = 0; i < g.s; ++i)
+    std::vector<char> live(g.s, 1);  // false: empty block, or no process can ever receive it (mesh)
+    bool mesh = false;
+    for (int j = 0; j < g.d; ++j) mesh |= !c.periodic[j];
+    for (int i = 0; i < g.s; ++i) {
+        if (r.len[i] == 0) live[i] = 0;
+        for (int j = 0; j < g.d; ++j)
+            if (!c.periodic[j] && std::abs((int64_t)g.at(i)[j]) >= c.dims[j]) live[i] = 0;
         for (int k = 0; k < gr.n; ++k)
             if (group_nonzero(g.at(i), gr.begin[k], gr.begin[k + 1])) ++hops[i];
+    }
     std::vector<char> needs(g.s, 0);
-    for (int i = 0; i < g.s; ++i) needs[i] = r.len[i] > 0 && hops[i] >= 2;
+    for (int i = 0; i < g.s; ++i) needs[i] = live[i] && hops[i] >= 2;
     std::vector<int64_t> inter_off = layout_inter(r, needs);
 
     std::vector<int> remaining = hops, cur_buf(g.s, ISO_BUF_SEND);
     int round = 0, phase = 0, nmax = 0, parts = 0, locals = 0;
     std::vector<Part> locals_parts;
     for (int i = 0; i < g.s; ++i)
-        if (r.len[i] > 0 && hops[i] == 0) { add_local_copy(r, i, locals_parts); ++locals; }
+        if (live[i] && hops[i] == 0) { add_local_copy(r, i, locals_parts); ++locals; }
 
     for (int k = 0; k < gr.n; ++k) {
         const int j0 = gr.begin[k], j1 = gr.begin[k + 1];
         // bucket the neighbours by their coordinates in this group
         std::map<std::vector<int>, std::vector<int>, RoundOrder> buckets(RoundOrder{c.dims, j0, j1});
         for (int i = 0; i < g.s; ++i) {
-            if (r.len[i] == 0 || !group_nonzero(g.at(i), j0, j1)) continue;
+            if (!live[i] || !group_nonzero(g.at(i), j0, j1)) continue;
             buckets[std::vector<int>(g.at(i) + j0, g.at(i) + j1)].push_back(i);
         }
         nmax = std::max<int>(nmax, (int)buckets.size());
@@ -292,6 +301,25 @@ int build_combining_alltoall(Request &r, const Geometry &g)
             ++phase;
         }
     }
+    if (mesh) {
+        // Non-periodic dimensions: a block travels only if both its original sender and its
+        // final receiver exist.  Seen from the process x that receives hop h of the block,
+        // the sender is x minus the coordinates already applied and the receiver x plus the
+        // ones still to come, so along a mesh dimension j the hop is performed iff
+        // 0 <= x_j - check_j < p_j with check_j = +c_j (applied, this hop included) or -c_j.
+        std::vector<std::vector<size_t>> chain(g.s);
+        for (size_t k = 0; k < r.parts.size(); ++k) chain[r.parts[k].slot].push_back(k);
+        for (int i = 0; i < g.s; ++i) {
+            bool applied[ISO_MAX_DIMS] = {false};
+            for (size_t k : chain[i]) {
+                Part &p = r.parts[k];
+                for (int j = 0; j < g.d; ++j)
+                    if (p.shift[j]) applied[j] = true;
+                for (int j = 0; j < g.d; ++j)
+                    if (!c.periodic[j]) p.check[j] = applied[j] ? g.at(i)[j] : -g.at(i)[j];
+            }
+        }
+    }
     // Blocks of at most 16 bytes: run every block's final hop in the last phase (a hop may
     // be postponed, only the order of a block's own hops matters), so that the receive
     // buffer is written by one launch, whole rows at a time, instead of in isolated
@@ -311,7 +339,9 @@ int build_combining_alltoall(Request &r, const Geometry &g)
         std::stable_sort(r.parts.begin(), r.parts.end(),
                          [](const Part &a, const Part &b) { return a.phase < b.phase; });
     }
-    if (r.layout == ISO_LAYOUT_PACKED) pack_intermediates(r, g.s);
+    // on a mesh the receive buffer must not serve as scratch (an undelivered slot keeps its
+    // contents), so the packed layout is used whatever was asked for
+    if (r.layout == ISO_LAYOUT_PACKED || mesh) pack_intermediates(r, g.s);
     // blocks for the process itself: one local copy, together with the first phase
     for (Part &p : locals_parts) p.phase = 0;
     r.parts.insert(r.parts.begin(), locals_parts.begin(), locals_parts.end());
@@ -498,7 +528,8 @@ int build_schedule(Request &r)
             int v = c.coords[(size_t)i * c.d + j];
             g.red[(size_t)i * c.d + j] = c.periodic[j] ? reduce_mod(v, c.dims[j]) : v;
         }
-    if (mesh && r.alg != ISO_ALG_DIRECT) return ISO_ERR_ARG;
+    // meshes: the direct schedule, and the combining schedule of the all-to-all
+    if (mesh && !(r.alg == ISO_ALG_DIRECT || (r.alg == ISO_ALG_COMBINING && r.kind != ISO_KIND_ALLGATHER))) return ISO_ERR_ARG;
     const bool gather = r.kind == ISO_KIND_ALLGATHER;
     if (r.alg == ISO_ALG_TORUS && gather) return ISO_ERR_ARG;
     if (r.alg != ISO_ALG_COMBINING && r.alg != ISO_ALG_DIRECT && r.alg != ISO_ALG_TORUS) return ISO_ERR_ARG;
@@ -720,7 +751,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         units += n;
                         if (!L.parts.empty() && L.parts[0].units != lp.units) uniform = false;
                         for (int j = 0; j < c.d; ++j)
-                            if (lp.p.shift[j]) used[j] = true;
+                            if (lp.p.shift[j] || lp.p.check[j]) used[j] = true;
                         L.parts.push_back(lp);
                         if (kernel == KERNEL_BULK) bulk_bytes += lp.p.len;
                     }

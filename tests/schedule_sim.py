@@ -43,8 +43,9 @@ def simulate(parts, dims, stats, send, periodic=None):
                 if periodic[j]:
                     src[:, j] = (src[:, j] - c) % dims[j]
                 else:
+                    y = coords[:, j] - p["check"][j]
+                    valid &= (y >= 0) & (y < dims[j])
                     src[:, j] = src[:, j] - c
-                    valid &= (src[:, j] >= 0) & (src[:, j] < dims[j])
             src[~valid] = 0
             sr = np.ravel_multi_index(tuple(src.T), dims) if P else np.zeros(0, np.int64)
             so, do, n = p["src_off"], p["dst_off"], p["len"]

@@ -268,20 +268,27 @@ def test_allgatherv_and_unaligned_receive_layout(torch_cuda):
     iso.Iso_comm_free(comm)
 
 
-def test_mesh_direct(torch_cuda):
+def test_mesh(torch_cuda):
+    """Non-periodic dimensions: blocks whose source lies outside are not delivered."""
     torch = torch_cuda
-    w = wl.Workload("mesh", "alltoall", (9, 11), wl.moore(2, 2), 16, seed=4)
-    run = Run(torch, w, periodic=[0, 0])
-    assert iso.Iso_request_get_stats(run.req)["algorithm"] == iso.ISO_ALG_DIRECT
-    got = run.result(iso.ISO_ALG_DIRECT, 1).reshape(w.P, w.s, 16)
-    full = oracle_result(w, run.send_host).reshape(w.P, w.s, 16)
-    for r in range(w.P):
-        R = (r // 11, r % 11)
-        for i, C in enumerate(w.offsets):
-            inside = 0 <= R[0] - C[0] < 9 and 0 <= R[1] - C[1] < 11
-            want = full[r, i] if inside else np.full(16, POISON, np.uint8)
-            assert np.array_equal(got[r, i], want), (r, i)
-    run.close()
+    for dims, periodic, offs, m in [((9, 11), [0, 0], wl.moore(2, 2), 16), ((6, 7, 5), [0, 1, 0], wl.moore(3, 1), 64),
+                                    ((12, 9), [1, 0], wl.moore(2, 1), 1024)]:
+        w = wl.Workload("mesh", "alltoall", dims, offs, m, seed=4)
+        run = Run(torch, w, periodic=periodic)
+        full = oracle_result(w, run.send_host).reshape(w.P, w.s, m)
+        want = np.full_like(full, POISON)
+        coords = np.stack(np.unravel_index(np.arange(w.P), dims), axis=1)
+        for i, C in enumerate(offs):
+            inside = np.ones(w.P, bool)
+            for j, per in enumerate(periodic):
+                if not per:
+                    y = coords[:, j] - int(C[j])
+                    inside &= (y >= 0) & (y < dims[j])
+            want[inside, i] = full[inside, i]
+        for alg, fusion in (DIRECT, COMB1, COMB0, COMB2, ALT1):
+            got = run.result(alg, fusion).reshape(w.P, w.s, m)
+            assert np.array_equal(got, want), (dims, alg, fusion)
+        run.close()
 
 
 def test_persistent_request_streams_and_host_buffers(torch_cuda):

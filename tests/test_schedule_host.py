@@ -45,7 +45,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(iso.Iso_stats) == 11 * 4 + 4 + 7 * 8
-    assert ctypes.sizeof(iso.Iso_part) == 8 * 4 + 3 * 8 + 8 * 4
+    assert ctypes.sizeof(iso.Iso_part) == 8 * 4 + 3 * 8 + 8 * 4 + 8 * 4
 
 
 def _tiny_workloads():
@@ -278,21 +278,50 @@ def test_alignment_classes_and_bulk_selection():
     iso.Iso_comm_free(comm)
 
 
-def test_mesh_direct():
-    w = wl.Workload("mesh", "alltoall", (4, 5), wl.moore(2, 2), 4)
-    comm, req = make_request(w, periodic=[0, 1])
+def _mesh_expected(w, send, periodic):
+    """Oracle result with the blocks whose source lies outside a non-periodic dimension left
+    at the poison value (the receive slot keeps its previous contents)."""
+    m = w.block_bytes
+    full = oracle_result(w, send).reshape(w.P, w.s, m)
+    want = np.full_like(full, POISON)
+    coords = np.stack(np.unravel_index(np.arange(w.P), w.dims), axis=1)
+    for i, C in enumerate(w.offsets):
+        inside = np.ones(w.P, bool)
+        for j, per in enumerate(periodic):
+            if not per:
+                y = coords[:, j] - int(C[j])
+                inside &= (y >= 0) & (y < w.dims[j])
+        want[inside, i] = full[inside, i]
+    return want.reshape(w.P, w.s * m)
+
+
+@pytest.mark.parametrize("dims,periodic,nbh", [((4, 5), [0, 1], "moore2"), ((5, 4, 3), [0, 0, 0], "moore1"),
+                                               ((3, 6, 4), [1, 0, 1], "moore1"), ((7, 2), [0, 0], "far")])
+def test_mesh_schedules(dims, periodic, nbh):
+    offs = {"moore2": wl.moore(2, 2), "moore1": wl.moore(len(dims), 1),
+            "far": np.array([[1, 0], [-3, 1], [7, 0], [0, 0], [2, -1], [-1, -1]], np.int32)}[nbh]
+    w = wl.Workload("mesh", "alltoall", dims, offs, 4)
+    comm, req = make_request(w, periodic=periodic)
+    assert iso.Iso_request_get_stats(req)["algorithm"] == iso.ISO_ALG_COMBINING
+    for alg, fusion in [(iso.ISO_ALG_DIRECT, 1), (iso.ISO_ALG_COMBINING, 0), (iso.ISO_ALG_COMBINING, 1),
+                        (iso.ISO_ALG_COMBINING, 2), (iso.ISO_ALG_COMBINING, 101)]:
+        set_alg(req, alg, fusion)
+        st = iso.Iso_request_get_stats(req)
+        send = send_buffer_np(w, st["send_stride"])
+        got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send, periodic=periodic)
+        assert np.array_equal(got, _mesh_expected(w, send, periodic)), (alg, fusion)
+    with pytest.raises(iso.IsoError):
+        iso.Iso_request_set_algorithm(req, iso.ISO_ALG_TORUS, 1)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+    # allgather on a mesh: the direct schedule only
+    wg = wl.Workload("mesh", "allgather", dims, offs, 4)
+    comm, req = make_request(wg, periodic=periodic)
     assert iso.Iso_request_get_stats(req)["algorithm"] == iso.ISO_ALG_DIRECT
     st = iso.Iso_request_get_stats(req)
-    send = send_buffer_np(w, st["send_stride"])
-    got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send, periodic=[0, 1])
-    full = oracle_result(w, send).reshape(w.P, w.s, 4)
-    want = np.full_like(full, POISON)
-    for r in range(w.P):
-        r0 = r // 5
-        for i, C in enumerate(w.offsets):
-            if 0 <= r0 - C[0] < 4:
-                want[r, i] = full[r, i]
-    assert np.array_equal(got.reshape(w.P, w.s, 4), want)
+    send = send_buffer_np(wg, st["send_stride"])
+    got = simulate(iso.Iso_request_get_parts(req), wg.dims, st, send, periodic=periodic)
+    assert np.array_equal(got, _mesh_expected(wg, send, periodic))
     with pytest.raises(iso.IsoError):
         iso.Iso_request_set_algorithm(req, iso.ISO_ALG_COMBINING, 1)
     iso.Iso_request_free(req)
