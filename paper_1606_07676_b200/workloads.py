@@ -247,6 +247,13 @@ def config(name: str, seed: int = DEFAULT_SEED) -> Workload:
         offs = random_offsets(seed, 3, 30, -3, 3)
         lens = random_sizes(seed, 30)
         return Workload(name, "alltoallv", (64, 64, 32), offs, 0, lens=lens, kind="uint8", seed=seed)
+    if name.startswith("stencil_d3_m"):
+        # the paper's irregular experiment (Section IV): block to neighbour i has mhat^(d - ||C^i||_1)
+        # bytes, so corners get 1 byte, edges mhat, faces mhat^2; packed displacements
+        mhat = int(name[len("stencil_d3_m"):])
+        offs = moore(3, 1)
+        lens = np.asarray([mhat ** (3 - int(np.abs(v).sum())) for v in offs], dtype=np.int64)
+        return Workload(name, "alltoallv", (32, 32, 32), offs, 0, lens=lens, kind="uint8", seed=seed)
     # neighbourhoods of the paper's second set of experiments (Sections IV and VI), 64-byte blocks
     paper = {"moore_d3r3": ((32, 32, 32), lambda: moore(3, 3)), "octant_d3r3": ((32, 32, 32), lambda: positive_octant(3, 3)),
              "shells_d3": ((32, 32, 32), lambda: shells(3, (3, 7))), "moore_d4r1": ((16, 16, 16, 16), lambda: moore(4, 1))}
@@ -281,7 +288,7 @@ def send_buffer_np(w: Workload, send_stride: int) -> np.ndarray:
 
 
 PAPER_NAMES = tuple("%s_%s" % (k, c) for k in ("moore_d3r3", "octant_d3r3", "shells_d3", "moore_d4r1")
-                    for c in ("alltoall", "allgather"))
+                    for c in ("alltoall", "allgather")) + ("stencil_d3_m32", "stencil_d3_m512")
 
 CONFIG_NAMES = ("cfg1", "cfg2_alltoall", "cfg2_allgather", "cfg3_m4", "cfg3_m64", "cfg3_m512",
                 "cfg3_m4096", "cfg4", "cfg5")

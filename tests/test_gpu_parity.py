@@ -241,6 +241,16 @@ def test_paper_neighbourhoods(torch_cuda):
             check(torch_cuda, w, [COMB1, DIRECT] + ([TORUS] if coll == "alltoall" and len(offs) < 200 else []))
 
 
+def test_stencil_shaped_irregular_sizes(torch_cuda):
+    # corners 1 byte, edges mhat, faces mhat^2, packed: every displacement is odd, long blocks
+    # are split into a narrow head, an aligned body (bulk kernel) and a narrow tail
+    for mhat in (8, 32):
+        full = wl.config("stencil_d3_m%d" % mhat)
+        w = wl.Workload(full.name, "alltoallv", (9, 8, 10), full.offsets, 0, lens=full.lens, seed=21)
+        check(torch_cuda, w, [COMB0, COMB1, COMB2, ALT1, DIRECT, TORUS])
+        check(torch_cuda, w, [COMB1], bulk=0)
+
+
 def test_allgatherv_and_unaligned_receive_layout(torch_cuda):
     torch = torch_cuda
     dims, offs = (6, 7), wl.moore(2, 1)
