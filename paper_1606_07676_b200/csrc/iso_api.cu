@@ -450,6 +450,19 @@ void plan_slabs(const Request &r, std::vector<SlabPlan> &slabs)
         }
 }
 
+// No exception may cross the C boundary: allocation failures become ISO_ERR_NOMEM.
+template <typename F>
+int guarded(F &&f) noexcept
+{
+    try {
+        return f();
+    } catch (const std::bad_alloc &) {
+        return ISO_ERR_NOMEM;
+    } catch (...) {
+        return ISO_ERR_STATE;
+    }
+}
+
 int check_handle(Iso_request request)
 {
     return request && request->comm ? ISO_SUCCESS : ISO_ERR_ARG;
@@ -461,6 +474,7 @@ extern "C" {
 
 int Iso_neighborhood_create(int d, const int dims[], int s, const int relative_coordinates[], Iso_comm *isocomm)
 {
+    return guarded([&]() -> int {
     if (!isocomm || !dims || s < 0 || (s > 0 && !relative_coordinates)) return ISO_ERR_ARG;
     if (d < 1 || d > ISO_MAX_DIMS) return ISO_ERR_DIMS;
     int64_t P = 1;
@@ -489,6 +503,7 @@ int Iso_neighborhood_create(int d, const int dims[], int s, const int relative_c
     }
     *isocomm = c;
     return ISO_SUCCESS;
+    });
 }
 
 int Iso_comm_set_periodic(Iso_comm isocomm, const int periodic[])
@@ -509,6 +524,7 @@ int Iso_comm_free(Iso_comm *isocomm)
 int Iso_neighbor_alltoall_init(const void *sendbuf, int sendcount, Iso_datatype sendtype, void *recvbuf,
                                int recvcount, Iso_datatype recvtype, Iso_comm isocomm, Iso_request *request)
 {
+    return guarded([&]() -> int {
     if (!isocomm || !request || sendcount < 0 || recvcount < 0 || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
     if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
     const int64_t m = (int64_t)sendcount * sendtype;
@@ -521,11 +537,13 @@ int Iso_neighbor_alltoall_init(const void *sendbuf, int sendcount, Iso_datatype 
     }
     r->send_stride = r->recv_stride = (int64_t)r->s * m;
     return finish_init(r, request);
+    });
 }
 
 int Iso_neighbor_allgather_init(const void *sendbuf, int sendcount, Iso_datatype sendtype, void *recvbuf,
                                 int recvcount, Iso_datatype recvtype, Iso_comm isocomm, Iso_request *request)
 {
+    return guarded([&]() -> int {
     if (!isocomm || !request || sendcount < 0 || recvcount < 0 || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
     if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
     const int64_t m = (int64_t)sendcount * sendtype;
@@ -540,6 +558,7 @@ int Iso_neighbor_allgather_init(const void *sendbuf, int sendcount, Iso_datatype
     r->send_stride = m;
     r->recv_stride = (int64_t)r->s * m;
     return finish_init(r, request);
+    });
 }
 
 int Iso_neighbor_alltoallv_init(const void *sendbuf, const int sendcounts[], const int64_t senddispls[],
@@ -547,6 +566,7 @@ int Iso_neighbor_alltoallv_init(const void *sendbuf, const int sendcounts[], con
                                 const int64_t recvdispls[], Iso_datatype recvtype, Iso_comm isocomm,
                                 Iso_request *request)
 {
+    return guarded([&]() -> int {
     if (!isocomm || !request || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
     if (isocomm->s > 0 && (!sendcounts || !senddispls || !recvcounts || !recvdispls)) return ISO_ERR_ARG;
     if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
@@ -567,12 +587,14 @@ int Iso_neighbor_alltoallv_init(const void *sendbuf, const int sendcounts[], con
     r->send_stride = round_up16(se);
     r->recv_stride = round_up16(re);
     return finish_init(r, request);
+    });
 }
 
 int Iso_neighbor_allgatherv_init(const void *sendbuf, int sendcount, Iso_datatype sendtype, void *recvbuf,
                                  const int recvcounts[], const int64_t recvdispls[], Iso_datatype recvtype,
                                  Iso_comm isocomm, Iso_request *request)
 {
+    return guarded([&]() -> int {
     if (!isocomm || !request || sendcount < 0 || sendtype < 1 || recvtype < 1) return ISO_ERR_ARG;
     if (isocomm->s > 0 && (!recvcounts || !recvdispls)) return ISO_ERR_ARG;
     if ((sendbuf == nullptr) != (recvbuf == nullptr)) return ISO_ERR_ARG;
@@ -593,10 +615,12 @@ int Iso_neighbor_allgatherv_init(const void *sendbuf, int sendcount, Iso_datatyp
     r->send_stride = round_up16(m);
     r->recv_stride = round_up16(re);
     return finish_init(r, request);
+    });
 }
 
 int Iso_request_set_algorithm(Iso_request request, int alg, int fusion_level)
 {
+    return guarded([&]() -> int {
     if (check_handle(request)) return ISO_ERR_ARG;
     if (alg != ISO_ALG_COMBINING && alg != ISO_ALG_DIRECT && alg != ISO_ALG_TORUS) return ISO_ERR_ARG;
     if (fusion_level < 0) return ISO_ERR_ARG;
@@ -618,18 +642,22 @@ int Iso_request_set_algorithm(Iso_request request, int alg, int fusion_level)
     }
     request->dirty = true;
     return rc;
+    });
 }
 
 int Iso_request_set_layout(Iso_request request, int layout)
 {
+    return guarded([&]() -> int {
     if (check_handle(request) || (layout != ISO_LAYOUT_PACKED && layout != ISO_LAYOUT_ALTERNATING)) return ISO_ERR_ARG;
     request->layout = layout;
     if (request->alg != ISO_ALG_COMBINING) return ISO_SUCCESS;  // takes effect with the next combining schedule
     return Iso_request_set_algorithm(request, request->alg, request->fusion);
+    });
 }
 
 int Iso_request_set_single_launch(Iso_request request, int enable)
 {
+    return guarded([&]() -> int {
     if (check_handle(request)) return ISO_ERR_ARG;
     if (request->started) {
         int rc = Iso_wait(request);
@@ -638,10 +666,12 @@ int Iso_request_set_single_launch(Iso_request request, int enable)
     request->persistent = enable != 0;
     request->dirty = true;
     return ISO_SUCCESS;
+    });
 }
 
 int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
 {
+    return guarded([&]() -> int {
     if (check_handle(request) || bytes < 0) return ISO_ERR_ARG;
     if (request->started) {
         int rc = Iso_wait(request);
@@ -651,10 +681,12 @@ int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
     int rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
     request->dirty = true;
     return rc;
+    });
 }
 
 int Iso_Start(Iso_request request, void *cuda_stream)
 {
+    return guarded([&]() -> int {
     if (check_handle(request)) return ISO_ERR_ARG;
     Request &r = *request;
     if (!r.send || !r.recv) return ISO_ERR_STATE;
@@ -699,10 +731,12 @@ int Iso_Start(Iso_request request, void *cuda_stream)
     r.last_stream = cuda_stream;
     r.started = true;
     return ISO_SUCCESS;
+    });
 }
 
 int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_recvbuf, void *cuda_stream)
 {
+    return guarded([&]() -> int {
     if (check_handle(request) || !host_sendbuf || !host_recvbuf) return ISO_ERR_ARG;
     Request &r = *request;
     if (!r.send || !r.recv) return ISO_ERR_STATE;
@@ -782,6 +816,7 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
     r.last_stream = cuda_stream;
     r.started = true;
     return ISO_SUCCESS;
+    });
 }
 
 int Iso_wait(Iso_request request)
@@ -817,6 +852,7 @@ int Iso_request_get_stats(Iso_request request, Iso_stats *out)
 
 int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int *count)
 {
+    return guarded([&]() -> int {
     if (check_handle(request) || !count || capacity < 0 || (capacity > 0 && !out)) return ISO_ERR_ARG;
     int n = 0;
     for (const LaunchPlan &L : request->launches) {
@@ -842,6 +878,7 @@ int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int 
     }
     *count = n;
     return ISO_SUCCESS;
+    });
 }
 
 int Iso_request_free(Iso_request *request)
@@ -948,6 +985,7 @@ extern "C" int Iso_neighbor_alltoall_static(int d, const int dims[], int s, cons
                                             const void *sendbuf, void *recvbuf, int count, Iso_datatype type,
                                             void *cuda_stream)
 {
+    return guarded([&]() -> int {
     if (!dims || s < 0 || (s > 0 && !relative_coordinates) || !sendbuf || !recvbuf || count < 0 || type < 1)
         return ISO_ERR_ARG;
     if (d < 1 || d > ISO_MAX_DIMS) return ISO_ERR_DIMS;
@@ -1057,4 +1095,5 @@ extern "C" int Iso_neighbor_alltoall_static(int d, const int dims[], int s, cons
         if (rc != ISO_SUCCESS) return rc;
     }
     return ISO_SUCCESS;
+    });
 }
