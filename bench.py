@@ -34,7 +34,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + written) per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (iso_gather_rows on cfg2_alltoall); only valid for that kernel build
 # and workload, so it is reported for the default workload and schedule only.
-TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_alltoall": 45.74e6}
+TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_alltoall": 44.89e6}
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 512 << 20
 
