@@ -241,6 +241,40 @@ def test_paper_neighbourhoods(torch_cuda):
             check(torch_cuda, w, [COMB1, DIRECT] + ([TORUS] if coll == "alltoall" and len(offs) < 200 else []))
 
 
+def test_alltoallv_with_different_send_and_receive_layouts(torch_cuda):
+    """Receive displacements are a permutation of the send displacements with gaps, so source
+    and destination of a block are misaligned against each other."""
+    torch = torch_cuda
+    rng = np.random.default_rng(31)
+    dims, offs = (7, 6, 5), wl.moore(3, 1)
+    P, s = 210, 26
+    lens = rng.choice([0, 4, 16, 20, 64, 260, 1024, 1500], size=s).astype(np.int64)
+    sd = wl.packed_displacements(lens)
+    rd = np.zeros(s, np.int64)
+    cur = 8
+    for i in rng.permutation(s):
+        rd[i] = cur
+        cur += lens[i] + int(rng.choice([0, 4, 12]))
+    ss = (int(lens.sum()) + 15) // 16 * 16
+    rs = (int((rd + lens).max()) + 15) // 16 * 16
+    send_h = wl.payload_np("uint8", 9, 0, 0, P * ss).reshape(P, ss).copy()
+    send = torch.from_numpy(send_h).cuda()
+    recv = torch.empty((P, rs), dtype=torch.uint8, device="cuda")
+    comm = iso.Iso_neighborhood_create(dims, offs)
+    req = iso.Iso_neighbor_alltoallv_init(send, lens, sd, 1, recv, lens, rd, 1, comm)
+    st = iso.Iso_request_get_stats(req)
+    assert (st["send_stride"], st["recv_stride"]) == (ss, rs)
+    want = oracle.alltoallv(dims, offs, lens, sd, rd, ss, rs, send_h, fill=POISON)
+    for alg, fusion in (COMB1, COMB0, COMB2, DIRECT, TORUS):
+        iso.Iso_request_set_algorithm(req, alg, fusion)
+        recv.fill_(POISON)
+        iso.Iso_Start(req)
+        iso.Iso_wait(req)
+        assert np.array_equal(recv.cpu().numpy(), want), (alg, fusion)
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
 def test_stencil_shaped_irregular_sizes(torch_cuda):
     # corners 1 byte, edges mhat, faces mhat^2, packed: every displacement is odd, long blocks
     # are split into a narrow head, an aligned body (bulk kernel) and a narrow tail
