@@ -61,11 +61,13 @@ struct Geometry {
 // coordinates first); keys of fused dimension groups are compared coordinate by coordinate.
 struct RoundOrder {
     const int *dims;
+    const int *periodic;  // on a mesh dimension the coordinates are signed and taken as they are
     int j0, j1;
     bool operator()(const std::vector<int> &a, const std::vector<int> &b) const
     {
         for (int j = j0; j < j1; ++j) {
-            int sa = symmetric_rep(a[j - j0], dims[j]), sb = symmetric_rep(b[j - j0], dims[j]);
+            int sa = periodic[j] ? symmetric_rep(a[j - j0], dims[j]) : a[j - j0];
+            int sb = periodic[j] ? symmetric_rep(b[j - j0], dims[j]) : b[j - j0];
             if (sa == sb) continue;
             bool na = sa < 0, nb = sb < 0;
             if (na != nb) return nb;  // non-negative first
@@ -277,7 +279,7 @@ int build_combining_alltoall(Request &r, const Geometry &g)
     for (int k = 0; k < gr.n; ++k) {
         const int j0 = gr.begin[k], j1 = gr.begin[k + 1];
         // bucket the neighbours by their coordinates in this group
-        std::map<std::vector<int>, std::vector<int>, RoundOrder> buckets(RoundOrder{c.dims, j0, j1});
+        std::map<std::vector<int>, std::vector<int>, RoundOrder> buckets(RoundOrder{c.dims, c.periodic, j0, j1});
         for (int i = 0; i < g.s; ++i) {
             if (!live[i] || !group_nonzero(g.at(i), j0, j1)) continue;
             buckets[std::vector<int>(g.at(i) + j0, g.at(i) + j1)].push_back(i);
@@ -430,7 +432,7 @@ int build_combining_allgather(Request &r, const Geometry &g)
     for (int k = 0; k < gr.n && m > 0; ++k) {
         const int j0 = gr.begin[k], j1 = gr.begin[k + 1];
         // rounds of this group: distinct non-zero coordinate keys
-        std::map<std::vector<int>, int, RoundOrder> round_of(RoundOrder{c.dims, j0, j1});
+        std::map<std::vector<int>, int, RoundOrder> round_of(RoundOrder{c.dims, c.periodic, j0, j1});
         for (int i = 0; i < g.s; ++i)
             if (group_nonzero(g.at(i), j0, j1)) round_of[std::vector<int>(g.at(i) + j0, g.at(i) + j1)] = 0;
         nmax = std::max<int>(nmax, (int)round_of.size());
