@@ -228,6 +228,19 @@ int Iso_request_set_layout(Iso_request request, int layout);
  */
 int Iso_request_set_single_launch(Iso_request request, int enable);
 
+/*
+ * Slab execution.  When only blocks read from the send buffer move along dimension 0 (the
+ * combining and direct schedules on periodic tori) the torus can be processed in slabs of
+ * consecutive planes of dimension 0, all phases of one slab before the next slab: a slab's
+ * intermediate blocks are then read back while still in the L2 cache, and the intermediate
+ * buffer only holds one slab and is reused, so its lines are overwritten in cache instead of
+ * being written to device memory.  `slabs` = 0 (default) lets the library choose (vector
+ * launches only, and only when a slab's launch still lasts about 12 microseconds), 1 turns
+ * it off, n >= 2 asks for n slabs (at most the size of dimension 0; ignored when the
+ * schedule does not allow it or in single-launch mode).  The result never depends on it.
+ */
+int Iso_request_set_slabs(Iso_request request, int slabs);
+
 /* Parts of at least `bytes` bytes whose addresses and length are multiples of 16 are moved
  * by the bulk-copy kernel (asynchronous bulk copies staged through shared memory), the rest
  * by the vector kernel.  Default 512 (measured crossover: the bulk kernel wins from 512-byte

@@ -84,6 +84,7 @@ struct Request {
     int fusion = 1;
     int64_t bulk_threshold = 512;
     int layout = ISO_LAYOUT_PACKED;
+    int slab_request = 0;     // slabs of dimension 0 Iso_Start runs one after the other (0: automatic, 1: none)
     bool persistent = false;  // run all phases in one cooperative launch when the schedule allows
     const unsigned char *send = nullptr;
     unsigned char *recv = nullptr;
@@ -106,6 +107,8 @@ struct Request {
     int *h_err = nullptr;
     void *last_stream = nullptr;
     bool started = false;
+    std::vector<std::pair<long long, long long>> slab_plan;  // row ranges of the slabs (empty: whole torus at once)
+    int64_t inter_rows = 0;            // processes the intermediate buffer holds
     void *copy_stream = nullptr;       // download stream of the pipelined host-buffer path
     void *up_stream = nullptr;         // its upload stream
     std::vector<void *> slab_events;   // its events

@@ -78,7 +78,8 @@ def random_cases(chunk, trials=40):
             choices += [(iso.ISO_ALG_COMBINING, g) for g in (0, 1, 2, 3)]
         if not is_mesh and kind != "allgather":
             choices += [(iso.ISO_ALG_TORUS, 1)]
-        options = [(int(rng.integers(0, 2)), bool(rng.integers(0, 2)), int(rng.choice([0, 256, 512, 1024]))) for _ in choices]
+        options = [(int(rng.integers(0, 2)), bool(rng.integers(0, 2)), int(rng.choice([0, 256, 512, 1024])),
+                    int(rng.choice([0, 1, 2, 3, 5]))) for _ in choices]
         yield dict(trial=trial, d=d, dims=dims, P=P, s=s, offs=offs, kind=kind, periodic=periodic, is_mesh=is_mesh,
                    lens=lens, sd=sd, rd=rd, ss=ss, rs=rs, send_h=send_h, choices=choices, options=options)
 
@@ -114,8 +115,9 @@ def test_random_cases(chunk):
         recv = torch.full((P, rs), POISON, dtype=torch.uint8, device="cuda") if rs else torch.zeros(1, dtype=torch.uint8, device="cuda")
         comm, req = make_request(c, send, recv)
         want = expected(c) if rs else None
-        for (alg, fusion), (lay, single, bulk) in zip(c["choices"], c["options"]):
+        for (alg, fusion), (lay, single, bulk, slabs) in zip(c["choices"], c["options"]):
             iso.Iso_request_set_layout(req, lay)
+            iso.Iso_request_set_slabs(req, slabs)
             iso.Iso_request_set_single_launch(req, single)
             iso.Iso_request_set_bulk_threshold(req, bulk)
             iso.Iso_request_set_algorithm(req, alg, fusion)
@@ -137,7 +139,7 @@ def test_random_cases(chunk):
                 got = recv.cpu().numpy()
             if rs:
                 assert np.array_equal(got, want), dict(chunk=chunk, trial=c["trial"], dims=c["dims"], kind=c["kind"], s=c["s"],
-                                                       alg=alg, fusion=fusion, layout=lay, single=single, bulk=bulk, host=via_host,
+                                                       alg=alg, fusion=fusion, layout=lay, single=single, bulk=bulk, host=via_host, slabs=slabs,
                                                        periodic=c["periodic"], lens=c["lens"].tolist())
         iso.Iso_request_free(req)
         iso.Iso_comm_free(comm)
@@ -152,7 +154,7 @@ def test_random_cases_host_simulation(chunk):
             continue
         comm, req = make_request(c, None, None)
         want = expected(c)
-        for (alg, fusion), (lay, single, bulk) in zip(c["choices"], c["options"]):
+        for (alg, fusion), (lay, single, bulk, slabs) in zip(c["choices"], c["options"]):
             iso.Iso_request_set_layout(req, lay)
             iso.Iso_request_set_bulk_threshold(req, bulk)
             iso.Iso_request_set_algorithm(req, alg, fusion)

@@ -100,6 +100,25 @@ def test_all_phases_in_one_cooperative_launch(torch_cuda):
     run.close()
 
 
+def test_slab_execution(torch_cuda):
+    """Slab after slab along dimension 0 with a one-slab intermediate buffer: same result for
+    any slab count, and the intermediate buffer shrinks accordingly."""
+    torch = torch_cuda
+    for name, algs in [("cfg2_alltoall", [COMB1, COMB0, COMB2, ALT1, DIRECT]), ("cfg3_m64", [COMB1]),
+                       ("cfg2_allgather", [COMB1]), ("octant_d3r3_allgather", [COMB1])]:
+        w = wl.config(name)
+        run = Run(torch, w)
+        want = oracle_result(w, run.send_host)
+        for slabs in (2, 5, 32, 1, 0):
+            iso.Iso_request_set_slabs(run.req, slabs)
+            for alg, fusion in algs:
+                got = run.result(alg, fusion)
+                assert np.array_equal(got, want), (name, slabs, alg, fusion)
+                if slabs == 5 and (alg, fusion) == COMB1 and w.collective == "alltoall":
+                    assert iso.Iso_request_get_stats(run.req)["launches"] % 5 == 0
+        run.close()
+
+
 def test_cfg2_allgather(torch_cuda):
     check(torch_cuda, wl.config("cfg2_allgather"), [COMB0, COMB1, COMB2, COMBD, DIRECT])
 
