@@ -73,6 +73,20 @@ def pin_golden(lib):
     assert n == 3
 
 
+def pin_golden_allgather(lib):
+    dims, offs = (4, 4), moore_list(2, 1)
+    send = np.array([100 * q for q in range(16)], dtype=np.int32)
+    recv = oracle.allgather(dims, offs, 4, send, lib=lib).view(np.int32).reshape(16, 8)
+    n = 0
+    for line in open(os.path.join(GOLDEN, "moore_4x4_allgather.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        rank, vals = line.split(":")
+        assert recv[int(rank)].tolist() == [int(v) for v in vals.split()], "rank " + rank
+        n += 1
+    assert n == 2
+
+
 def pin_push_equals_pull(lib):
     rng = np.random.default_rng(7)
     cases = [((1,), 3), ((2,), 4), ((4,), 5), ((3, 2), 6), ((2, 3, 4), 9), ((1, 4), 4), ((4, 3), 12)]
@@ -181,7 +195,7 @@ def pin_chunks(lib):
     assert np.array_equal(np.concatenate(parts), full)
 
 
-PINS = [pin_golden, pin_push_equals_pull, pin_numpy_special_cases, pin_rank_helpers, pin_chunks]
+PINS = [pin_golden, pin_golden_allgather, pin_push_equals_pull, pin_numpy_special_cases, pin_rank_helpers, pin_chunks]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)

@@ -155,9 +155,13 @@ def test_alltoall_statistics_follow_section_v(name):
 
 
 def test_hand_worked_schedule_4x4():
-    # Moore r=1 on a 4x4 torus: rounds (0,+1)={5,6,7}, (0,-1)={0,1,2}, (1,+1)={2,4,7}, (1,-1)={0,3,5};
-    # hops = [2,1,2,1,1,2,1,2]; the first hop of a two-hop block lands in the intermediate
-    # buffer, the last hop of every block in the receive buffer (Algorithm 1's parity rule)
+    # tests/golden/moore_4x4_schedule.txt: rounds, hops and first-hop buffers worked by hand
+    golden = {}
+    for line in open(os.path.join(ROOT, "tests", "golden", "moore_4x4_schedule.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = [x.strip() for x in line.split(":")]
+        golden[f[0]] = f[1:]
     w = wl.Workload("hand", "alltoall", (4, 4), wl.moore(2, 1), 4)
     comm, req = make_request(w)
     iso.Iso_request_set_layout(req, iso.ISO_LAYOUT_ALTERNATING)
@@ -167,16 +171,20 @@ def test_hand_worked_schedule_4x4():
     for p in parts:
         rounds.setdefault(p["round"], []).append(p)
     assert sorted(rounds) == [0, 1, 2, 3]
-    assert [sorted(q["slot"] for q in rounds[k]) for k in range(4)] == [[5, 6, 7], [0, 1, 2], [2, 4, 7], [0, 3, 5]]
-    assert [rounds[k][0]["shift"][:2] for k in range(4)] == [[1, 0], [3, 0], [0, 1], [0, 3]]
+    for k in range(4):
+        dim, shift = golden[str(k)][0].split()
+        want_shift = [0, 0]
+        want_shift[int(dim)] = int(shift) % 4
+        assert sorted(q["slot"] for q in rounds[k]) == [int(x) for x in golden[str(k)][1].split()]
+        assert all(q["shift"][:2] == want_shift for q in rounds[k])
     hops = [sum(1 for p in parts if p["slot"] == i) for i in range(8)]
-    assert hops == [2, 1, 2, 1, 1, 2, 1, 2]
+    assert hops == [int(x) for x in golden["hops"][0].split()]
     first = {}
     for p in parts:
         first.setdefault(p["slot"], p)
-    for i in range(8):
-        assert first[i]["src_buf"] == iso.ISO_BUF_SEND
-        assert first[i]["dst_buf"] == (iso.ISO_BUF_INTER if hops[i] == 2 else iso.ISO_BUF_RECV)
+    via_inter = sorted(i for i in range(8) if first[i]["dst_buf"] == iso.ISO_BUF_INTER)
+    assert via_inter == [int(x) for x in golden["first_hop_into_intermediate"][0].split()]
+    assert all(first[i]["src_buf"] == iso.ISO_BUF_SEND for i in range(8))
     last = {p["slot"]: p for p in parts}
     assert all(p["dst_buf"] == iso.ISO_BUF_RECV for p in last.values())
     st = iso.Iso_request_get_stats(req)
