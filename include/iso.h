@@ -265,7 +265,9 @@ int Iso_comm_set_periodic(Iso_comm isocomm, const int periodic[]);
  * cast to void*, NULL = the default stream) and returns without waiting (the non-blocking
  * start proposed in Section VII).  The first start after an init or a set_* call also
  * allocates the intermediate buffer and uploads the index tables (cudaMalloc and a blocking
- * copy), so it must not happen inside a stream capture.
+ * copy), so it must not happen inside a stream capture.  Starts of one request are ordered
+ * by the stream they are enqueued on: a request owns one intermediate buffer, so two starts
+ * of the same request on different streams must not overlap.
  * Errors: ISO_ERR_STATE (request has no buffers), ISO_ERR_NOMEM, ISO_ERR_CUDA.
  */
 int Iso_Start(Iso_request request, void *cuda_stream);
