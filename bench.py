@@ -390,6 +390,11 @@ def run_ours(args):
                    "bytes": "value = bytes read + written by the schedule / device time"},
         "gpu_launches": iso.Iso_request_get_stats(b.req)["launches"] * args.steps,
         "frac_of_nominal_8TBs": per_gpu / NOMINAL_HBM_GBS,
+        "frac_of_measured": per_gpu / peak,
+        # the same time over the minimum one-read-one-write payload instead of the bytes moved
+        "payload": {"gbs": world * minimum / (ms * 1e-3) / 1e9,
+                    "frac_of_measured": minimum / (ms * 1e-3) / 1e9 / peak,
+                    "frac_of_nominal_8TBs": minimum / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
     }
 
     if rank == 0 and world == 1 and args.headline_only:
