@@ -135,6 +135,46 @@ int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
 LaunchDev make_launch_args(const Request &r, const LaunchPlan &L);
 void choose_slab_plan(Request &r);
 
+// One descriptor per unit position of a vector launch: parts in their order, the units of
+// a part in address order.
+void fill_units(const Request &r, const LaunchPlan &L, UnitDev *ud)
+{
+    const Comm &c = *r.comm;
+    const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
+    int used_index[ISO_MAX_DIMS];
+    for (int j = 0; j < ISO_MAX_DIMS; ++j) used_index[j] = -1;
+    for (int k = 0; k < L.n_used; ++k) used_index[L.used_dim[k]] = k;
+    std::vector<UnitDev> units(L.units_per_proc);
+    for (const LoweredPart &lp : L.parts) {
+        UnitDev u{};
+        long long delta = 0;
+        if (!L.compact) {
+            u.nnz = (uint8_t)L.n_used;
+            for (int z = 0; z < L.n_used; ++z) u.dim[z] = (uint8_t)z;
+        }
+        for (int j = 0; j < c.d; ++j) {
+            // periodic dimension: the shift (wrap test); mesh dimension: the check value
+            const int value = c.periodic[j] ? lp.p.shift[j] : lp.p.check[j];
+            delta -= (long long)lp.p.shift[j] * c.rank_stride[j];
+            if (!value) continue;
+            if (L.compact) {
+                u.dim[u.nnz] = (uint8_t)used_index[j];
+                u.c[u.nnz++] = value;
+            } else {
+                u.c[used_index[j]] = value;
+            }
+        }
+        u.src_buf = (uint8_t)lp.p.src_buf;
+        u.dst_buf = (uint8_t)lp.p.dst_buf;
+        for (uint32_t k = 0; k < lp.units; ++k) {
+            u.src_term = delta * stride[lp.p.src_buf] + lp.p.src_off + (int64_t)k * L.width;
+            u.dst_term = lp.p.dst_off + (int64_t)k * L.width;
+            units[lp.first_unit + k] = u;
+        }
+    }
+    std::copy(units.begin(), units.end(), ud);
+}
+
 // Uploads the lowered schedule and allocates the intermediate buffer.
 int materialise(Request &r)
 {
@@ -208,23 +248,7 @@ int materialise(Request &r)
         }
         if (!L.lookup.empty())
             std::memcpy(blob.data() + L.lookup_off, L.lookup.data(), L.lookup.size() * sizeof(uint16_t));
-        if (L.kernel == KERNEL_VEC) {
-            // one descriptor per unit position
-            const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
-            UnitDev *ud = reinterpret_cast<UnitDev *>(blob.data() + L.units_off);
-            for (size_t t = 0; t < L.parts.size(); ++t) {
-                const LoweredPart &lp = L.parts[t];
-                for (uint32_t k = 0; k < lp.units; ++k) {
-                    UnitDev u{};
-                    u.src_term = pd[t].rank_delta * stride[lp.p.src_buf] + lp.p.src_off + (int64_t)k * L.width;
-                    u.dst_term = lp.p.dst_off + (int64_t)k * L.width;
-                    for (int z = 0; z < pd[t].nnz; ++z) u.c[pd[t].dim[z]] = pd[t].c[z];
-                    u.src_buf = pd[t].src_buf;
-                    u.dst_buf = pd[t].dst_buf;
-                    ud[lp.first_unit + k] = u;
-                }
-            }
-        }
+        if (L.kernel == KERNEL_VEC) fill_units(r, L, reinterpret_cast<UnitDev *>(blob.data() + L.units_off));
     }
     if (r.d_blob) cudaFree(r.d_blob);
     r.d_blob = nullptr;
@@ -384,19 +408,25 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
                          : launch_kernel(iso_gather_rows_reg<1, 4>, L, a, stream, dependent);
     } else {
         // kernels specialised on the number of shifted dimensions; meshes take the general one
-        const int nu = L.n_used <= 3 ? L.n_used : ISO_MAX_DIMS;
-#define ISO_ROWS(W, NU, MESH)                                                                              \
-    e = (W == 16 && L.threads > 256)                                                                       \
-            ? launch_wide(iso_gather_rows_wide<16, kVecDepth, NU, MESH>, L, a, stream, dependent)            \
-            : launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH>, L, a, stream, dependent)
-#define ISO_ROWS_W(W)                                             \
-    do {                                                          \
-        if (a.mesh_mask) ISO_ROWS(W, ISO_MAX_DIMS, true);         \
-        else if (nu == 0) ISO_ROWS(W, 0, false);                  \
-        else if (nu == 1) ISO_ROWS(W, 1, false);                  \
-        else if (nu == 2) ISO_ROWS(W, 2, false);                  \
-        else if (nu == 3) ISO_ROWS(W, 3, false);                  \
-        else ISO_ROWS(W, ISO_MAX_DIMS, false);                    \
+        // (with compact unit descriptors: on the dimensions one unit is shifted along)
+        const int count = L.compact ? L.max_nnz : L.n_used;
+        const int nu = count <= 3 ? count : ISO_MAX_DIMS;
+#define ISO_ROWS(W, NU, MESH, COMPACT)                                                                          \
+    e = (W == 16 && L.threads > 256)                                                                            \
+            ? launch_wide(iso_gather_rows_wide<16, kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent)        \
+            : launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent)
+#define ISO_ROWS_W(W)                                                            \
+    do {                                                                         \
+        if (a.mesh_mask) ISO_ROWS(W, ISO_MAX_DIMS, true, false);                 \
+        else if (L.compact && nu == 1) ISO_ROWS(W, 1, false, true);              \
+        else if (L.compact && nu == 2) ISO_ROWS(W, 2, false, true);              \
+        else if (L.compact && nu == 3) ISO_ROWS(W, 3, false, true);              \
+        else if (L.compact) ISO_ROWS(W, ISO_MAX_DIMS, false, true);              \
+        else if (nu == 0) ISO_ROWS(W, 0, false, false);                          \
+        else if (nu == 1) ISO_ROWS(W, 1, false, false);                          \
+        else if (nu == 2) ISO_ROWS(W, 2, false, false);                          \
+        else if (nu == 3) ISO_ROWS(W, 3, false, false);                          \
+        else ISO_ROWS(W, ISO_MAX_DIMS, false, false);                            \
     } while (0)
         if (L.width == 16) ISO_ROWS_W(16);
         else if (L.width == 8) ISO_ROWS_W(8);
@@ -1137,29 +1167,7 @@ extern "C" int Iso_neighbor_alltoall_static(int d, const int dims[], int s, cons
 
     // unit tables, built on the host and copied behind the intermediate buffer
     std::vector<unsigned char> blob((size_t)table_bytes, 0);
-    const int64_t strides[3] = {r.send_stride, r.recv_stride, r.inter_stride};
-    for (const LaunchPlan &L : r.launches) {
-        int used_index[ISO_MAX_DIMS];
-        for (int j = 0; j < ISO_MAX_DIMS; ++j) used_index[j] = -1;
-        for (int k = 0; k < L.n_used; ++k) used_index[L.used_dim[k]] = k;
-        UnitDev *ud = reinterpret_cast<UnitDev *>(blob.data() + L.units_off);
-        for (const LoweredPart &lp : L.parts) {
-            long long delta = 0;
-            UnitDev u{};
-            for (int j = 0; j < d; ++j) {
-                if (!lp.p.shift[j]) continue;
-                delta -= (long long)lp.p.shift[j] * comm.rank_stride[j];
-                u.c[used_index[j]] = lp.p.shift[j];
-            }
-            u.src_buf = (uint8_t)lp.p.src_buf;
-            u.dst_buf = (uint8_t)lp.p.dst_buf;
-            for (uint32_t k = 0; k < lp.units; ++k) {
-                u.src_term = delta * strides[lp.p.src_buf] + lp.p.src_off + (int64_t)k * L.width;
-                u.dst_term = lp.p.dst_off + (int64_t)k * L.width;
-                ud[lp.first_unit + k] = u;
-            }
-        }
-    }
+    for (const LaunchPlan &L : r.launches) fill_units(r, L, reinterpret_cast<UnitDev *>(blob.data() + L.units_off));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     unsigned char *tables = scratch + inter_bytes;
     if (table_bytes > 0 &&

@@ -73,6 +73,8 @@ struct LaunchPlan {
     size_t smem = 0;
     int n_used = 0;
     int used_dim[ISO_MAX_DIMS] = {0};
+    int max_nnz = 0;       // most dimensions any one part shifts along
+    bool compact = false;  // vector kernel: unit descriptors list only the shifted dimensions
     // byte offsets of this launch's tables inside the request's device blob
     size_t parts_off = 0, lookup_off = 0, units_off = 0;
 };

@@ -41,10 +41,15 @@ struct alignas(16) PartDev {
 struct alignas(16) UnitDev {
     long long src_term;  // rank_delta * source stride + source offset of the unit (bytes)
     long long dst_term;  // destination offset of the unit (bytes)
-    int32_t c[ISO_MAX_DIMS];  // coordinate shift along each used dimension (0: none)
-    uint8_t src_buf, dst_buf;
-    uint8_t pad[14];
+    // Dense form (nnz = the launch's n_used, dim[e] = e): c[e] is the coordinate shift
+    // along used dimension e, 0 for none.  Compact form: only the shifted dimensions are
+    // listed, c[e] != 0 along used dimension dim[e] for e < nnz.
+    int32_t c[ISO_MAX_DIMS];
+    uint8_t src_buf, dst_buf, nnz, pad0;
+    uint8_t dim[ISO_MAX_DIMS];
+    uint8_t pad1[4];
 };
+static_assert(sizeof(UnitDev) == 64, "unit descriptors are read as four 16-byte words");
 
 struct LaunchDev {
     const PartDev *parts;
@@ -177,6 +182,8 @@ struct UnitRegs {
     unsigned char *B;        // destination base: buffer + dst_term
     long long stride_s, stride_d;
     int c[ISO_MAX_DIMS];
+    uint32_t nnz;
+    uint32_t dims_lo, dims_hi;  // dim[0..3], dim[4..7], one byte each
 };
 
 __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
@@ -193,6 +200,9 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
     R.stride_d = L.buf_stride[db];
     R.c[0] = (int)b.x; R.c[1] = (int)b.y; R.c[2] = (int)b.z; R.c[3] = (int)b.w;
     R.c[4] = (int)c.x; R.c[5] = (int)c.y; R.c[6] = (int)c.z; R.c[7] = (int)c.w;
+    R.nnz = (d.x >> 16) & 0xff;
+    R.dims_lo = d.y;
+    R.dims_hi = d.z;
     return R;
 }
 
@@ -211,10 +221,14 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
 // holding registers; a slot is read back and stored to its destination as soon as the
 // oldest group has landed, and refilled with the load of DEPTH rows ahead.
 //
-// NU is the number of shifted dimensions the kernel is compiled for (the launch's n_used
-// must not exceed it; ISO_MAX_DIMS is the general case), MESH whether some of them are
-// non-periodic (then a row whose source lies outside the mesh is skipped).
-template <int W, int DEPTH, int NU, bool MESH>
+// NU is the number of shifted dimensions per unit the kernel is compiled for (dense
+// descriptors: the launch's n_used must not exceed it; compact descriptors: no unit's nnz
+// may; ISO_MAX_DIMS is the general case), MESH whether some dimensions are non-periodic
+// (then a row whose source lies outside the mesh is skipped).  COMPACT selects the compact
+// descriptor form: a launch that shifts along many dimensions, each unit along few of
+// them (the last phase of a schedule whose final hops were postponed, the direct schedule
+// in high dimension), then tests per row only the dimensions its unit moves along.
+template <int W, int DEPTH, int NU, bool MESH, bool COMPACT>
 __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned char *ring_base, bool dependent_launch)
 {
     using V = typename VecOf<W>::type;
@@ -241,9 +255,14 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
 
     for (uint32_t u = ul; u < U; u += CU) {
         const UnitRegs R = u == ul ? R_first : load_unit(L, u);
+        // used dimension tested in position e: e itself (dense) or the unit's own list
+        auto dim_of = [&](int e) -> int {
+            return COMPACT ? (int)(((e < 4 ? R.dims_lo : R.dims_hi) >> (8 * (e & 3))) & 0xffu) : e;
+        };
+        const int n_tests = COMPACT ? (int)R.nnz : L.n_used;
         long long wrap_bytes[NU > 0 ? NU : 1];
 #pragma unroll
-        for (int e = 0; e < NU; ++e) wrap_bytes[e] = (long long)L.used_wrap[e] * R.stride_s;
+        for (int e = 0; e < NU; ++e) wrap_bytes[e] = (long long)L.used_wrap[dim_of(e)] * R.stride_s;
         const long long src_step = rstep * R.stride_s, dst_step = rstep * R.stride_d;
 
         auto source = [&](const unsigned char *nowrap, long long r, const unsigned char *&src) -> bool {
@@ -251,12 +270,13 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
             src = nowrap;
 #pragma unroll
             for (int e = 0; e < NU; ++e) {
-                if (NU < ISO_MAX_DIMS || e < L.n_used) {
-                    const uint32_t t = fastdiv(L.div_rstride[e], (uint32_t)r);
-                    const int x = (int)(t - fastdiv(L.div_size[e], t) * L.used_size[e]);
-                    if (MESH && ((L.mesh_mask >> e) & 1)) {
+                if ((!COMPACT && NU < ISO_MAX_DIMS) || e < n_tests) {
+                    const int k = dim_of(e);
+                    const uint32_t t = fastdiv(L.div_rstride[k], (uint32_t)r);
+                    const int x = (int)(t - fastdiv(L.div_size[k], t) * L.used_size[k]);
+                    if (MESH && ((L.mesh_mask >> k) & 1)) {
                         const int y = x - R.c[e];
-                        valid = valid && y >= 0 && y < (int)L.used_size[e];
+                        valid = valid && y >= 0 && y < (int)L.used_size[k];
                     } else if (x < R.c[e]) {
                         src += wrap_bytes[e];
                     }
@@ -302,21 +322,21 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
     }
 }
 
-template <int W, int DEPTH, int NU, bool MESH>
+template <int W, int DEPTH, int NU, bool MESH, bool COMPACT>
 __global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant__ LaunchDev L)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    gather_rows_body<W, DEPTH, NU, MESH>(L, smem_raw, true);
+    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true);
 }
 
 // The same body in CTAs of up to 1024 threads, for launches whose payload per process has
 // more than 256 unit positions: one CTA then covers up to 16 KB of a row at a time, so rows
 // are still visited one after the other instead of in 4 KB columns.
-template <int W, int DEPTH, int NU, bool MESH>
+template <int W, int DEPTH, int NU, bool MESH, bool COMPACT>
 __global__ void __launch_bounds__(1024, 1) iso_gather_rows_wide(const __grid_constant__ LaunchDev L)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    gather_rows_body<W, DEPTH, NU, MESH>(L, smem_raw, true);
+    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true);
 }
 
 // All phases of a schedule in ONE cooperative launch: the CTAs run phase after phase and
@@ -376,11 +396,11 @@ __global__ void __launch_bounds__(256, 4) iso_gather_rows_multi(const __grid_con
         for (uint32_t i = threadIdx.x; i < sizeof(LaunchDev) / 4; i += blockDim.x) dst[i] = __ldg(src + i);
         __syncthreads();
         switch (sL->n_used) {
-        case 0: gather_rows_body<16, DEPTH, 0, false>(*sL, ring, false); break;
-        case 1: gather_rows_body<16, DEPTH, 1, false>(*sL, ring, false); break;
-        case 2: gather_rows_body<16, DEPTH, 2, false>(*sL, ring, false); break;
-        case 3: gather_rows_body<16, DEPTH, 3, false>(*sL, ring, false); break;
-        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false>(*sL, ring, false); break;
+        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false); break;
+        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false); break;
+        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false); break;
+        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false); break;
+        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false); break;
         }
         if (ph + 1 < M.n && !grid_barrier(M, M.epoch + (unsigned long long)(ph + 1) * gridDim.x, &s_ok)) return;
     }

@@ -208,14 +208,25 @@ void pack_intermediates(Request &r, int s)
 {
     std::vector<std::vector<size_t>> chain(s);  // indices of a slot's hops, in execution order
     for (size_t k = 0; k < r.parts.size(); ++k) chain[r.parts[k].slot].push_back(k);
-    struct Place { int write_phase, read_phase, slot, hop; };
+    struct Place { int write_phase, read_phase, read_round, slot, hop; };
     std::vector<Place> places;
+    // Blocks that one round reads lie side by side: a process then fetches one contiguous
+    // run per source process instead of pieces interleaved with those of other rounds.
+    // Only where every block fills whole 32-byte sectors: with smaller blocks it is the
+    // writers' pieces that get split, which measured slower.
+    int64_t min_len = INT64_MAX;
+    for (int i = 0; i < s; ++i)
+        if (r.len[i] > 0) min_len = std::min(min_len, r.len[i]);
+    bool by_round = min_len >= 32;
+    if (const char *env = std::getenv("ISO_PACK_BY_ROUND")) by_round = std::atoi(env) != 0;
     for (int i = 0; i < s; ++i)
         for (size_t j = 0; j + 1 < chain[i].size(); ++j)
-            places.push_back(Place{r.parts[chain[i][j]].phase, r.parts[chain[i][j + 1]].phase, i, (int)j});
+            places.push_back(Place{r.parts[chain[i][j]].phase, r.parts[chain[i][j + 1]].phase,
+                                   by_round ? r.parts[chain[i][j + 1]].round : 0, i, (int)j});
     std::sort(places.begin(), places.end(), [](const Place &a, const Place &b) {
         if (a.write_phase != b.write_phase) return a.write_phase < b.write_phase;
         if (a.read_phase != b.read_phase) return a.read_phase < b.read_phase;
+        if (a.read_round != b.read_round) return a.read_round < b.read_round;
         return a.slot < b.slot;
     });
     int64_t cur = 0;
@@ -752,15 +763,25 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         lp.units = (uint32_t)n;
                         units += n;
                         if (!L.parts.empty() && L.parts[0].units != lp.units) uniform = false;
+                        int nnz = 0;
                         for (int j = 0; j < c.d; ++j)
-                            if (lp.p.shift[j] || lp.p.check[j]) used[j] = true;
+                            if (lp.p.shift[j] || lp.p.check[j]) { used[j] = true; ++nnz; }
+                        L.max_nnz = std::max(L.max_nnz, nnz);
                         L.parts.push_back(lp);
                         if (kernel == KERNEL_BULK) bulk_bytes += lp.p.len;
                     }
                     L.units_per_proc = (uint32_t)units;
                     L.uniform_units = uniform ? L.parts[0].units : 0;
+                    bool torus = true;
                     for (int j = 0; j < c.d; ++j)
-                        if (used[j]) L.used_dim[L.n_used++] = j;
+                        if (used[j]) {
+                            L.used_dim[L.n_used++] = j;
+                            torus = torus && c.periodic[j];
+                        }
+                    // many shifted dimensions in the launch, few per part: the kernel then
+                    // tests per row only the dimensions a unit moves along
+                    L.compact = kernel == KERNEL_VEC && width >= 4 && L.n_used > 3 && L.max_nnz < L.n_used &&
+                                torus && !r.persistent;
                     // coarse lookup: unit >> shift -> part
                     if (!uniform) {
                         int shift = 0;
@@ -786,7 +807,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         L.chunk_units = (uint32_t)std::min<uint64_t>(units, max_threads);
                         L.rows_per_pass = std::max<uint32_t>(1, max_threads == 256 ? 256 / L.chunk_units : 1);
                         L.threads = (int)((L.chunk_units * L.rows_per_pass + 31) / 32 * 32);
-                        int per_sm = L.threads > 512 ? 1 : (L.threads > 256 ? 2 : 4);
+                        // CTAs of fewer than 256 threads: as many per SM as keep 1024 threads resident
+                        int per_sm = L.threads > 512 ? 1 : (L.threads > 256 ? 2 : std::min(16, std::max(4, 1024 / L.threads)));
                         if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
                             int v = std::atoi(env);
                             if (v >= 1 && v <= 8 && L.threads <= 256) per_sm = v;
