@@ -202,15 +202,32 @@ class Bound:
 
     bulk_threshold = None
     single_launch = False
+    slabs = None      # None: the library's choice
+    chains = None
+    graph = None
+    tune = False      # let the library time its execution variants and keep the fastest
 
-    def set(self, alg, fusion):
-        self.iso.Iso_request_set_single_launch(self.req, Bound.single_launch)
-        self.iso.Iso_request_set_algorithm(self.req, alg, fusion)
+    def set(self, alg, fusion, execution=None):
+        """Selects the schedule; `execution` (slabs, chains, graph) copies another instance's
+        tuned choice instead of tuning again."""
+        iso = self.iso
+        iso.Iso_request_set_single_launch(self.req, Bound.single_launch)
+        iso.Iso_request_set_algorithm(self.req, alg, fusion)
         if Bound.bulk_threshold is not None:
-            self.iso.Iso_request_set_bulk_threshold(self.req, Bound.bulk_threshold)
-        self.iso.Iso_Start(self.req, self.torch.cuda.current_stream())    # materialise outside the timed region
-        self.iso.Iso_wait(self.req)
-        return self.iso.Iso_request_get_stats(self.req)
+            iso.Iso_request_set_bulk_threshold(self.req, Bound.bulk_threshold)
+        ex = execution or {"slabs": Bound.slabs, "chains": Bound.chains, "graph": Bound.graph}
+        iso.Iso_request_set_slabs(self.req, ex["slabs"] if ex["slabs"] is not None else 0)
+        iso.Iso_request_set_chains(self.req, ex["chains"] if ex["chains"] is not None else 1)
+        iso.Iso_request_set_graph(self.req, bool(ex["graph"]))
+        stream = self.torch.cuda.current_stream()
+        if Bound.tune and execution is None and not Bound.single_launch:
+            iso.Iso_request_tune(self.req, stream, cold=True)   # the timed steps rotate over instances: cold caches
+        iso.Iso_Start(self.req, stream)    # materialise outside the timed region
+        iso.Iso_wait(self.req)
+        return iso.Iso_request_get_stats(self.req)
+
+    def execution(self):
+        return self.iso.Iso_request_get_execution(self.req)
 
     def close(self):
         self.iso.Iso_request_free(self.req)
@@ -282,7 +299,14 @@ class Replicas:
         self.iso, self.torch = iso, torch
 
     def set(self, alg, fusion):
-        return [b.set(alg, fusion) for b in self.items][0]
+        st = self.items[0].set(alg, fusion)
+        ex = self.items[0].execution() if Bound.tune else None
+        for b in self.items[1:]:
+            b.set(alg, fusion, ex)
+        return st
+
+    def execution(self):
+        return self.items[0].execution()
 
     def start(self, k):
         b = self.items[k % len(self.items)]
@@ -371,6 +395,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     Bound.bulk_threshold = args.bulk_threshold
     Bound.single_launch = args.single_launch
+    Bound.slabs, Bound.chains, Bound.graph, Bound.tune = args.slabs, args.chains, args.graph, args.tune
     reps = Replicas(torch, iso, wl, args.workload)
     b = reps.items[0]
 
@@ -396,6 +421,7 @@ def run_ours(args):
     per_gpu = moved / (ms * 1e-3) / 1e9
 
     detail = {"combining": {"fusion_level": args.fusion, "rounds": st["rounds"], "launches": st["launches"],
+                            "execution": dict(reps.execution(), tuned=bool(args.tune)),
                             "bytes_moved": moved, "bytes_min": minimum, "ms": ms, "gbs_moved": per_gpu,
                             "gbs_payload": minimum / (ms * 1e-3) / 1e9, "replicas": len(reps.items),
                             "footprint_bytes_per_replica": reps.footprint}}
@@ -498,7 +524,8 @@ def sweep(torch, iso, wl, peak, args):
             st = reps.set(alg, fusion)
             steps = 40 if st["bytes_moved"] < (4 << 30) else 6
             ms = time_run(torch, reps.start, steps, 4)
-            row[key] = {"rounds": st["rounds"], "launches": st["launches"], "bytes_moved": st["bytes_moved"],
+            row[key] = {"rounds": st["rounds"], "launches": st["launches"], "execution": reps.execution(),
+                        "bytes_moved": st["bytes_moved"],
                         "bytes_min": st["bytes_min"], "bulk_bytes": st["bulk_bytes"], "ms": ms,
                         "replicas": len(reps.items),
                         "gbs_moved": st["bytes_moved"] / ms / 1e6, "gbs_payload": st["bytes_min"] / ms / 1e6,
@@ -557,6 +584,12 @@ def main():
                     help="run all phases in one cooperative launch instead of one launch per phase")
     ap.add_argument("--bulk-threshold", type=int, default=None,
                     help="override the size from which parts go to the bulk-copy kernel (0: never)")
+    ap.add_argument("--slabs", type=int, default=None, help="slabs of dimension 0 (default: the library's choice)")
+    ap.add_argument("--chains", type=int, default=None, help="slabs that run side by side")
+    ap.add_argument("--graph", action="store_true", help="replay the launches from a captured graph")
+    ap.add_argument("--tune", action="store_true",
+                    help="call Iso_request_tune before timing: the library times its execution variants "
+                         "(slabs, chains, graph replay) and keeps the fastest")
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture, if one is current")
     ap.add_argument("--init-times", action="store_true",

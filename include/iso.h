@@ -241,6 +241,47 @@ int Iso_request_set_single_launch(Iso_request request, int enable);
  */
 int Iso_request_set_slabs(Iso_request request, int slabs);
 
+/*
+ * Slabs side by side (no counterpart in the paper).  With `chains` = n >= 2 the slabs of
+ * Iso_request_set_slabs are dealt to n chains that run at the same time, each on 1/n of
+ * the CTA slots and with its own one-slab part of the intermediate buffer: the start and
+ * the drain of one chain's short kernels are covered by the other chains.  The number of
+ * slabs is rounded to a multiple of n; the launches are then replayed from a captured
+ * graph (see Iso_request_set_graph).  1 (default) turns it off; at most 8.  Ignored where
+ * slab execution is (see there).  The result never depends on it.
+ */
+int Iso_request_set_chains(Iso_request request, int chains);
+
+/*
+ * Graph replay (no counterpart in the paper).  With `enable` != 0 the first Iso_Start after
+ * a change of the request captures its launches into a CUDA graph on a stream of the
+ * library's own and every Iso_Start replays that graph on the caller's stream: one
+ * submission per start instead of one per launch, which pays for schedules of many short
+ * launches and costs a few microseconds on schedules of few long ones.  Default off.
+ * Ignored in single-launch mode.  The result never depends on it.
+ */
+int Iso_request_set_graph(Iso_request request, int enable);
+
+/*
+ * Measures instead of guessing (no counterpart in the paper; in the spirit of its
+ * persistent requests, which are set up once and started many times): runs the request
+ * with 1, 2, 4, ... slabs, with 1, 2 and 4 chains, with and without graph replay, timing a
+ * few starts of each on `cuda_stream` with events, and leaves the request on the fastest
+ * combination (a less plain plan has to win by 2 %).  `cold` = 0 times the starts back to
+ * back, as in a loop over the same buffers; `cold` != 0 overwrites a scratch buffer of twice
+ * the L2 size before every timed start (allocated for the duration of the call), as when
+ * other work runs between the starts.  The collective is executed many times meanwhile:
+ * the send buffers must hold readable data and the receive buffers are overwritten (with
+ * the collective's result).  Blocks the host until done.  Does nothing in single-launch
+ * mode.  On error the settings from before the call are restored.
+ */
+int Iso_request_tune(Iso_request request, void *cuda_stream, int cold);
+
+/* What Iso_Start does at present: slabs (1: none), chains (1: none), graph replay (0/1).
+ * Before the first Iso_Start after a change these are the values asked for (slabs 0:
+ * automatic); any of the pointers may be NULL. */
+int Iso_request_get_execution(Iso_request request, int *slabs, int *chains, int *graph);
+
 /* Parts of at least `bytes` bytes whose addresses and length are multiples of 16 are moved
  * by the bulk-copy kernel (asynchronous bulk copies staged through shared memory), the rest
  * by the vector kernel.  Default 512 (measured crossover: the bulk kernel wins from 512-byte

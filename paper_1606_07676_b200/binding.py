@@ -30,7 +30,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), LIB_NAME)
 EXPORTS = (
     "Iso_neighborhood_create", "Iso_comm_free", "Iso_comm_set_periodic",
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
-    "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_bulk_threshold",
+    "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_chains", "Iso_request_set_graph", "Iso_request_tune", "Iso_request_get_execution", "Iso_request_set_bulk_threshold",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
     "Iso_neighbor_alltoall_static", "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
@@ -94,6 +94,10 @@ def load_library() -> ctypes.CDLL:
         "Iso_request_set_layout": [vp, ci],
         "Iso_request_set_single_launch": [vp, ci],
         "Iso_request_set_slabs": [vp, ci],
+        "Iso_request_set_chains": [vp, ci],
+        "Iso_request_set_graph": [vp, ci],
+        "Iso_request_tune": [vp, vp, ci],
+        "Iso_request_get_execution": [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)],
         "Iso_request_set_bulk_threshold": [vp, i64],
         "Iso_Start": [vp, vp],
         "Iso_Start_host": [vp, vp, vp, vp],
@@ -241,6 +245,27 @@ def Iso_request_set_single_launch(request: int, enable: bool) -> None:
 
 def Iso_request_set_slabs(request: int, slabs: int) -> None:
     _check(load_library().Iso_request_set_slabs(request, slabs), "Iso_request_set_slabs")
+
+
+def Iso_request_set_chains(request: int, chains: int) -> None:
+    _check(load_library().Iso_request_set_chains(request, chains), "Iso_request_set_chains")
+
+
+def Iso_request_set_graph(request: int, enable: bool) -> None:
+    _check(load_library().Iso_request_set_graph(request, 1 if enable else 0), "Iso_request_set_graph")
+
+
+def Iso_request_tune(request: int, cuda_stream=None, cold: bool = False) -> dict:
+    """Times the execution variants on the device and keeps the fastest; returns it."""
+    _check(load_library().Iso_request_tune(request, _stream(cuda_stream), 1 if cold else 0), "Iso_request_tune")
+    return Iso_request_get_execution(request)
+
+
+def Iso_request_get_execution(request: int) -> dict:
+    slabs, chains, graph = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    _check(load_library().Iso_request_get_execution(request, ctypes.byref(slabs), ctypes.byref(chains),
+                                                    ctypes.byref(graph)), "Iso_request_get_execution")
+    return {"slabs": slabs.value, "chains": chains.value, "graph": graph.value}
 
 
 def Iso_request_set_bulk_threshold(request: int, nbytes: int) -> None:

@@ -37,6 +37,8 @@ int cuda_fail(cudaError_t e)
 
 void release_device(Request &r)
 {
+    if (r.graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.graph_exec));
+    r.graph_exec = nullptr;
     if (r.d_blob) cudaFree(r.d_blob);
     if (r.d_inter) cudaFree(r.d_inter);
     if (r.d_err) cudaFree(r.d_err);
@@ -179,6 +181,9 @@ void fill_units(const Request &r, const LaunchPlan &L, UnitDev *ud)
 int materialise(Request &r)
 {
     const Comm &c = *r.comm;
+    // a captured graph holds the addresses of the tables and buffers that are replaced below
+    if (r.graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.graph_exec));
+    r.graph_exec = nullptr;
     choose_slab_plan(r);
     // device tables depend on the alignment of the intermediate buffer: allocate it first
     const int64_t inter_bytes = r.inter_rows * r.inter_stride;
@@ -325,6 +330,7 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
     a.tile_procs = L.tile_procs;
     a.n_used = L.n_used;
     a.mesh_mask = 0;
+    a.grid_share = 1;
     FastDiv f = make_fastdiv(L.units_per_proc);
     a.div_units = FastDivDev{f.m, f.s1, f.s2, f.div};
     f = make_fastdiv(L.uniform_units ? L.uniform_units : 1);
@@ -345,13 +351,15 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
 }
 
 // Grid for the rows [a.row_lo, a.row_hi): the plan's grid scaled to the share of the rows.
-unsigned grid_for_rows(const LaunchPlan &L, const LaunchDev &a)
+unsigned grid_for_rows(const LaunchPlan &L, const LaunchDev &a, int share = 1)
 {
     const long long rows = a.row_hi - a.row_lo;
     if (rows >= a.P) return (unsigned)L.grid;
     if (L.kernel == KERNEL_BULK) return (unsigned)((rows + L.tile_procs - 1) / L.tile_procs);
     const long long groups = (rows + L.rows_per_pass - 1) / L.rows_per_pass;
-    const long long g = std::max<long long>(1, std::min<long long>(L.grid, groups));
+    // `share` launches of this kind run side by side: each takes its part of the CTA slots
+    const long long full = std::max<long long>(1, L.grid / std::max(1, share));
+    const long long g = std::max<long long>(1, std::min<long long>(full, groups));
     return (unsigned)g;
 }
 
@@ -359,7 +367,7 @@ template <typename Kernel>
 cudaError_t launch_kernel(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, cudaStream_t stream, bool dependent)
 {
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid_for_rows(L, a));
+    cfg.gridDim = dim3(grid_for_rows(L, a, a.grid_share));
     cfg.blockDim = dim3((unsigned)L.threads);
     cfg.dynamicSmemBytes = L.smem;
     cfg.stream = stream;
@@ -388,10 +396,11 @@ cudaError_t launch_wide(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, 
 }
 
 int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool dependent, long long row_lo = 0,
-               long long row_hi = -1, long long inter_row_base = 0)
+               long long row_hi = -1, long long inter_row_base = 0, int grid_share = 1)
 {
     if (L.grid == 0 || L.units_per_proc == 0) return ISO_SUCCESS;
     LaunchDev a = make_launch_args(r, L);
+    a.grid_share = grid_share;
     if (row_hi >= 0) {
         a.row_lo = row_lo;
         a.row_hi = row_hi;
@@ -509,6 +518,9 @@ void choose_slab_plan(Request &r)
     const Comm &c = *r.comm;
     r.slab_plan.clear();
     r.inter_rows = c.P;
+    r.chains = 1;
+    r.use_graph = !r.persistent && r.graph_request;
+    if (const char *env = std::getenv("ISO_GRAPH")) r.use_graph = !r.persistent && std::atoi(env) != 0;
     if (r.persistent || r.inter_stride == 0) return;
     int want = r.slab_request;
     if (const char *env = std::getenv("ISO_SLABS")) want = std::atoi(env);
@@ -526,6 +538,9 @@ void choose_slab_plan(Request &r)
         want = 1;
         while (want * 2 <= per && want * 2 <= 64 && c.P / (want * 2) >= 12 * rows_per_pass) want *= 2;
     }
+    int chains = std::max(1, r.chains_request);
+    if (const char *env = std::getenv("ISO_CHAINS")) chains = std::max(1, std::min(8, std::atoi(env)));
+    if (chains > 1) want = std::max(want, chains) / chains * chains;
     if (want < 2) return;
     std::vector<SlabPlan> slabs;
     plan_slabs(r, slabs, want);
@@ -534,6 +549,12 @@ void choose_slab_plan(Request &r)
     for (const SlabPlan &w : slabs) {
         r.slab_plan.push_back({w.row_lo, w.row_hi});
         rows = std::max(rows, w.row_hi - w.row_lo);
+    }
+    if (chains > 1 && slabs.size() % chains == 0) {
+        // slabs side by side: every chain has its own one-slab part of the intermediate buffer
+        r.chains = chains;
+        r.use_graph = true;
+        rows *= chains;
     }
     // the pipelined host-buffer path cuts dimension 0 into up to eight slabs of its own
     std::vector<SlabPlan> host;
@@ -545,6 +566,73 @@ void choose_slab_plan(Request &r)
 int check_handle(Iso_request request)
 {
     return request && request->comm ? ISO_SUCCESS : ISO_ERR_ARG;
+}
+
+// Captures the launches of one Iso_Start into a graph.  With r.chains > 1 the slabs are
+// dealt to that many chains, which run side by side: chain k takes the slabs k, k + chains,
+// ..., a 1/chains share of the CTA slots and its own part of the intermediate buffer, so
+// that the ramp and the drain of one chain's kernels are covered by the other chains.
+int build_graph(Request &r, bool use_pdl)
+{
+    const int n = std::max(1, r.chains);
+    std::vector<cudaStream_t> st(n, nullptr);
+    std::vector<cudaEvent_t> ev(n, nullptr);
+    cudaError_t e = cudaSuccess;
+    for (int k = 0; k < n && e == cudaSuccess; ++k) {
+        e = cudaStreamCreateWithFlags(&st[k], cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev[k], cudaEventDisableTiming);
+    }
+    cudaGraph_t graph = nullptr;
+    int rc = ISO_SUCCESS;
+    bool capturing = false;
+    if (e == cudaSuccess) e = cudaStreamBeginCapture(st[0], cudaStreamCaptureModeThreadLocal);
+    if (e == cudaSuccess) {
+        capturing = true;
+        e = cudaEventRecord(ev[0], st[0]);
+        for (int k = 1; k < n && e == cudaSuccess; ++k) e = cudaStreamWaitEvent(st[k], ev[0], 0);
+    }
+    if (e == cudaSuccess) {
+        if (r.slab_plan.size() > 1) {
+            long long slab_rows = 0;
+            for (const auto &w : r.slab_plan) slab_rows = std::max(slab_rows, w.second - w.first);
+            for (size_t i = 0; i < r.slab_plan.size() && rc == ISO_SUCCESS; ++i) {
+                const int k = (int)(i % (size_t)n);
+                const auto &w = r.slab_plan[i];
+                bool first = i < (size_t)n;  // nothing of this chain precedes it in its stream
+                for (const LaunchPlan &L : r.launches) {
+                    rc = launch_one(r, L, st[k], use_pdl && !first, w.first, w.second, w.first - (long long)k * slab_rows, n);
+                    first = false;
+                    if (rc != ISO_SUCCESS) break;
+                }
+            }
+        } else {
+            bool first = true;
+            for (const LaunchPlan &L : r.launches) {
+                rc = launch_one(r, L, st[0], use_pdl && !first);
+                first = false;
+                if (rc != ISO_SUCCESS) break;
+            }
+        }
+        for (int k = 1; k < n && e == cudaSuccess; ++k) {
+            e = cudaEventRecord(ev[k], st[k]);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(st[0], ev[k], 0);
+        }
+    }
+    if (capturing) {
+        cudaError_t e2 = cudaStreamEndCapture(st[0], &graph);
+        if (e == cudaSuccess) e = e2;
+    }
+    cudaGraphExec_t exec = nullptr;
+    if (e == cudaSuccess && rc == ISO_SUCCESS) e = cudaGraphInstantiate(&exec, graph, 0);
+    if (graph) cudaGraphDestroy(graph);
+    for (int k = 0; k < n; ++k) {
+        if (ev[k]) cudaEventDestroy(ev[k]);
+        if (st[k]) cudaStreamDestroy(st[k]);
+    }
+    if (rc != ISO_SUCCESS) return rc;
+    if (e != cudaSuccess) return cuda_fail(e);
+    r.graph_exec = exec;
+    return ISO_SUCCESS;
 }
 
 }  // namespace
@@ -762,6 +850,150 @@ int Iso_request_set_slabs(Iso_request request, int slabs)
     });
 }
 
+int Iso_request_set_chains(Iso_request request, int chains)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request) || chains < 1 || chains > 8) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    request->chains_request = chains;
+    request->dirty = true;
+    return ISO_SUCCESS;
+    });
+}
+
+int Iso_request_set_graph(Iso_request request, int enable)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request)) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    request->graph_request = enable != 0;
+    request->dirty = true;
+    return ISO_SUCCESS;
+    });
+}
+
+int Iso_request_get_execution(Iso_request request, int *slabs, int *chains, int *graph)
+{
+    if (check_handle(request)) return ISO_ERR_ARG;
+    const Request &r = *request;
+    if (slabs) *slabs = r.dirty ? r.slab_request : (int)std::max<size_t>(1, r.slab_plan.size());
+    if (chains) *chains = r.dirty ? r.chains_request : r.chains;
+    if (graph) *graph = r.dirty ? (r.graph_request ? 1 : 0) : (r.use_graph ? 1 : 0);
+    return ISO_SUCCESS;
+}
+
+int Iso_request_tune(Iso_request request, void *cuda_stream, int cold)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request)) return ISO_ERR_ARG;
+    Request &r = *request;
+    if (!r.send || !r.recv) return ISO_ERR_STATE;
+    if (r.persistent) return ISO_SUCCESS;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaEvent_t t0 = nullptr, t1 = nullptr;
+    ISO_CUDA(cudaEventCreate(&t0));
+    if (cudaEventCreate(&t1) != cudaSuccess) {
+        cudaEventDestroy(t0);
+        return cuda_fail(cudaGetLastError());
+    }
+    // cold: a scratch buffer of twice the L2 size is overwritten before every timed start
+    // (inside the timed span: the same cost for every variant)
+    unsigned char *scratch = nullptr;
+    size_t scratch_bytes = 0;
+    if (cold) {
+        int device = 0, l2 = 0;
+        cudaGetDevice(&device);
+        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device);
+        scratch_bytes = 2 * (size_t)std::max(l2, 32 << 20);
+        if (cudaMalloc((void **)&scratch, scratch_bytes) != cudaSuccess) {
+            cudaEventDestroy(t0);
+            cudaEventDestroy(t1);
+            return cuda_fail(cudaGetLastError());
+        }
+    }
+    static const bool log = std::getenv("ISO_TUNE_LOG") != nullptr;
+    struct Choice { int slabs, chains, graph; };
+    const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0};
+    Choice best = before;
+    float best_ms = -1.0f;
+    int rc = ISO_SUCCESS;
+    const int p0 = r.comm->dims[0];
+    auto apply = [&](const Choice &c) {
+        r.slab_request = c.slabs;
+        r.chains_request = c.chains;
+        r.graph_request = c.graph != 0;
+        r.dirty = true;
+    };
+    // time `reps` starts back to back (the collective only reads the send buffers, so
+    // repeating it leaves the same result)
+    auto measure = [&](int reps, float &ms) -> int {
+        for (int k = 0; k < 2; ++k) {
+            int e = Iso_Start(request, cuda_stream);
+            if (e != ISO_SUCCESS) return e;
+        }
+        if (cudaEventRecord(t0, stream) != cudaSuccess) return cuda_fail(cudaGetLastError());
+        for (int k = 0; k < reps; ++k) {
+            if (scratch && cudaMemsetAsync(scratch, k & 0xff, scratch_bytes, stream) != cudaSuccess)
+                return cuda_fail(cudaGetLastError());
+            int e = Iso_Start(request, cuda_stream);
+            if (e != ISO_SUCCESS) return e;
+        }
+        if (cudaEventRecord(t1, stream) != cudaSuccess) return cuda_fail(cudaGetLastError());
+        int e = Iso_wait(request);
+        if (e != ISO_SUCCESS) return e;
+        if (cudaEventElapsedTime(&ms, t0, t1) != cudaSuccess) return cuda_fail(cudaGetLastError());
+        ms /= (float)reps;
+        return ISO_SUCCESS;
+    };
+    std::vector<Choice> tried;
+    for (int graph = 0; graph <= 1 && rc == ISO_SUCCESS; ++graph)
+        for (int chains = 1; chains <= 4 && rc == ISO_SUCCESS; chains *= 2) {
+            if (chains > 1 && !graph) continue;  // chains only exist inside a graph
+            for (int slabs = 1; slabs <= 64 && slabs <= std::max(1, p0) && rc == ISO_SUCCESS; slabs *= 2) {
+                if (chains > 1 && slabs < chains) continue;
+                apply(Choice{slabs, chains, graph});
+                if (r.started) rc = Iso_wait(request);
+                if (rc == ISO_SUCCESS) rc = materialise(r);
+                if (rc != ISO_SUCCESS) break;
+                // what the schedule allowed may differ from what was asked for: skip repeats
+                const Choice got{(int)std::max<size_t>(1, r.slab_plan.size()), r.chains, r.use_graph ? 1 : 0};
+                bool seen = false;
+                for (const Choice &c : tried) seen = seen || (c.slabs == got.slabs && c.chains == got.chains && c.graph == got.graph);
+                if (seen) continue;
+                tried.push_back(got);
+                float ms = 0.0f;
+                rc = measure(3, ms);  // a first look, then the real measurement scaled to it
+                if (rc != ISO_SUCCESS) break;
+                const int reps = (int)std::max(5.0f, std::min(200.0f, 2.0f / std::max(ms, 1e-3f)));
+                rc = measure(reps, ms);
+                if (rc != ISO_SUCCESS) break;
+                if (log) std::fprintf(stderr, "iso tune: slabs %d chains %d graph %d: %.4f ms\n", got.slabs, got.chains, got.graph, ms);
+                // the plainer plans come first; a later one must win by 2 % to replace them
+                if (best_ms < 0.0f || ms < 0.98f * best_ms) {
+                    best_ms = ms;
+                    best = Choice{slabs, chains, graph};
+                }
+            }
+        }
+    cudaEventDestroy(t0);
+    cudaEventDestroy(t1);
+    if (scratch) cudaFree(scratch);
+    apply(rc == ISO_SUCCESS ? best : before);
+    if (r.started) {
+        int e = Iso_wait(request);
+        if (rc == ISO_SUCCESS) rc = e;
+    }
+    int e = materialise(r);
+    return rc != ISO_SUCCESS ? rc : e;
+    });
+}
+
 int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
 {
     return guarded([&]() -> int {
@@ -776,6 +1008,7 @@ int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
     return rc;
     });
 }
+
 
 int Iso_Start(Iso_request request, void *cuda_stream)
 {
@@ -813,6 +1046,17 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         ISO_CUDA(cudaLaunchKernelEx(&cfg, iso_gather_rows_multi<kVecDepth>, m));
+        r.last_stream = cuda_stream;
+        r.started = true;
+        return ISO_SUCCESS;
+    }
+    if (r.use_graph) {
+        // replay of the captured launches (chains of slabs side by side when asked for)
+        if (!r.graph_exec) {
+            int rc = build_graph(r, use_pdl);
+            if (rc != ISO_SUCCESS) return rc;
+        }
+        ISO_CUDA(cudaGraphLaunch(static_cast<cudaGraphExec_t>(r.graph_exec), stream));
         r.last_stream = cuda_stream;
         r.started = true;
         return ISO_SUCCESS;

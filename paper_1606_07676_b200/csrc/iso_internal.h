@@ -115,6 +115,11 @@ struct Request {
     void *up_stream = nullptr;         // its upload stream
     std::vector<void *> slab_events;   // its events
     int sm_count = 148;  // replaced by the device's count when the request is materialised
+    int chains_request = 1;     // slabs to run side by side, as asked for
+    bool graph_request = false; // graph replay, as asked for
+    int chains = 1;             // slabs that run side by side (each on its share of the SMs)
+    bool use_graph = false;     // Iso_Start replays a captured graph of the launches
+    void *graph_exec = nullptr; // cudaGraphExec_t, built at the first Iso_Start after a change
 };
 
 // Builds r.parts, r.inter_stride and the schedule statistics from r.comm, r.kind, r.alg,

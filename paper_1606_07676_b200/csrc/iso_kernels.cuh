@@ -70,6 +70,7 @@ struct LaunchDev {
     int tile_procs;
     int n_used;
     int mesh_mask;           // bit k set: used dimension k is not periodic
+    int grid_share;          // host side only: launches of this kind that run side by side
     FastDivDev div_units;    // division by units_per_proc
     FastDivDev div_uniform;  // division by uniform_units
     int used_dim[ISO_MAX_DIMS];

@@ -119,6 +119,43 @@ def test_slab_execution(torch_cuda):
         run.close()
 
 
+def test_chains_graph_replay_and_tuning(torch_cuda):
+    """Slabs side by side inside a captured graph, plain graph replay, and the measuring
+    tuner: the result is the oracle's whatever the execution plan, also after the plan is
+    changed on a request that has already run, and on repeated starts of one graph."""
+    torch = torch_cuda
+    for name, algs in [("cfg2_alltoall", [COMB1, COMB0, DIRECT]), ("cfg3_m64", [COMB1]), ("stencil_d3_m16", [COMB1]),
+                       ("cfg2_allgather", [COMB1]), ("cfg1", [COMB1, TORUS])]:
+        w = wl.config(name)
+        run = Run(torch, w)
+        want = oracle_result(w, run.send_host)
+        for slabs, chains, graph in [(0, 1, True), (4, 2, False), (8, 4, True), (6, 3, True), (2, 1, True), (0, 1, False)]:
+            iso.Iso_request_set_slabs(run.req, slabs)
+            iso.Iso_request_set_chains(run.req, chains)
+            iso.Iso_request_set_graph(run.req, graph)
+            for alg, fusion in algs:
+                got = run.result(alg, fusion)
+                assert np.array_equal(got, want), (name, slabs, chains, graph, alg, fusion)
+                ex = iso.Iso_request_get_execution(run.req)
+                assert ex["chains"] in (1, chains) and (ex["chains"] == 1 or ex["graph"] == 1)
+                if graph:
+                    assert ex["graph"] == 1
+                    # the same graph again, on poisoned receive buffers
+                    run.recv.fill_(0xA5)
+                    iso.Iso_Start(run.req, torch.cuda.current_stream())
+                    iso.Iso_wait(run.req)
+                    assert np.array_equal(run.recv.cpu().numpy().reshape(want.shape), want), (name, "replay")
+        for cold in (False, True):
+            chosen = iso.Iso_request_tune(run.req, torch.cuda.current_stream(), cold)
+            assert chosen["slabs"] >= 1 and chosen["chains"] in (1, 2, 4) and chosen["graph"] in (0, 1)
+            run.recv.fill_(0xA5)
+            iso.Iso_Start(run.req, torch.cuda.current_stream())
+            iso.Iso_wait(run.req)
+            assert np.array_equal(run.recv.cpu().numpy().reshape(want.shape), want), (name, "tuned", chosen)
+            assert iso.Iso_request_get_execution(run.req) == chosen
+        run.close()
+
+
 def test_cfg2_allgather(torch_cuda):
     check(torch_cuda, wl.config("cfg2_allgather"), [COMB0, COMB1, COMB2, COMBD, DIRECT])
 
