@@ -206,6 +206,7 @@ class Bound:
     chains = None
     graph = None
     tune = False      # let the library time its execution variants and keep the fastest
+    pipeline = None   # slabs of the pipelined one-launch execution (None: off)
 
     def set(self, alg, fusion, execution=None):
         """Selects the schedule; `execution` (slabs, chains, graph) copies another instance's
@@ -219,6 +220,7 @@ class Bound:
         iso.Iso_request_set_slabs(self.req, ex["slabs"] if ex["slabs"] is not None else 0)
         iso.Iso_request_set_chains(self.req, ex["chains"] if ex["chains"] is not None else 1)
         iso.Iso_request_set_graph(self.req, bool(ex["graph"]))
+        iso.Iso_request_set_pipeline(self.req, Bound.pipeline or 0)
         stream = self.torch.cuda.current_stream()
         if Bound.tune and execution is None and not Bound.single_launch:
             iso.Iso_request_tune(self.req, stream, cold=True)   # the timed steps rotate over instances: cold caches
@@ -396,6 +398,7 @@ def run_ours(args):
     Bound.bulk_threshold = args.bulk_threshold
     Bound.single_launch = args.single_launch
     Bound.slabs, Bound.chains, Bound.graph, Bound.tune = args.slabs, args.chains, args.graph, args.tune
+    Bound.pipeline = args.pipeline
     reps = Replicas(torch, iso, wl, args.workload)
     b = reps.items[0]
 
@@ -586,6 +589,8 @@ def main():
                     help="override the size from which parts go to the bulk-copy kernel (0: never)")
     ap.add_argument("--slabs", type=int, default=None, help="slabs of dimension 0 (default: the library's choice)")
     ap.add_argument("--chains", type=int, default=None, help="slabs that run side by side")
+    ap.add_argument("--pipeline", type=int, default=None,
+                    help="pipelined one-launch execution over this many slabs (Iso_request_set_pipeline)")
     ap.add_argument("--graph", action="store_true", help="replay the launches from a captured graph")
     ap.add_argument("--tune", action="store_true",
                     help="call Iso_request_tune before timing: the library times its execution variants "

@@ -229,6 +229,28 @@ int Iso_request_set_layout(Iso_request request, int layout);
 int Iso_request_set_single_launch(Iso_request request, int enable);
 
 /*
+ * Pipelined one-launch execution (no counterpart in the paper).  `slabs` >= 1 makes Iso_Start
+ * a single cooperative kernel launch that needs no grid-wide barrier: the torus is cut into
+ * `slabs` slabs of consecutive planes of dimension 0 (as for Iso_request_set_slabs, under the
+ * same condition; 1, or a schedule that cannot be cut, means the whole torus) and the work
+ * into items (slab, launch of the schedule).  All thread blocks go through the items in one
+ * order - the launches of two slabs interleaved - and every item has a counter of the thread
+ * blocks that have finished it; a block starts an item when the item it depends on (the
+ * same slab's previous phase, or the last reader of the intermediate place it overwrites) is
+ * complete, which in that order has normally happened already.  A slab's intermediate blocks
+ * are read back out of the L2 cache a few items after they were written, and from three
+ * slabs on the intermediate buffer holds only two slabs.  Requires what the single launch
+ * requires (16-byte vector launches on periodic dimensions: blocks that are multiples of
+ * 16 bytes and below the bulk threshold, or Iso_request_set_bulk_threshold(request, 0));
+ * where that does not hold the request runs as if this had not been called.  It takes
+ * precedence over Iso_request_set_single_launch, _set_slabs, _set_chains and _set_graph, and
+ * Iso_request_tune leaves such a request alone.  Every wait is bounded; on expiry the
+ * kernel stops and Iso_wait returns ISO_ERR_TIMEOUT.  0 (default) turns it off.  The result
+ * never depends on it.
+ */
+int Iso_request_set_pipeline(Iso_request request, int slabs);
+
+/*
  * Slab execution.  When only blocks read from the send buffer move along dimension 0 (the
  * combining and direct schedules on periodic tori) the torus can be processed in slabs of
  * consecutive planes of dimension 0, all phases of one slab before the next slab: a slab's

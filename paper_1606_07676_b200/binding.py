@@ -30,7 +30,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), LIB_NAME)
 EXPORTS = (
     "Iso_neighborhood_create", "Iso_comm_free", "Iso_comm_set_periodic",
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
-    "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_chains", "Iso_request_set_graph", "Iso_request_tune", "Iso_request_get_execution", "Iso_request_set_bulk_threshold",
+    "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_pipeline", "Iso_request_set_chains", "Iso_request_set_graph", "Iso_request_tune", "Iso_request_get_execution", "Iso_request_set_bulk_threshold",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
     "Iso_neighbor_alltoall_static", "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
@@ -94,6 +94,7 @@ def load_library() -> ctypes.CDLL:
         "Iso_request_set_layout": [vp, ci],
         "Iso_request_set_single_launch": [vp, ci],
         "Iso_request_set_slabs": [vp, ci],
+        "Iso_request_set_pipeline": [vp, ci],
         "Iso_request_set_chains": [vp, ci],
         "Iso_request_set_graph": [vp, ci],
         "Iso_request_tune": [vp, vp, ci],
@@ -241,6 +242,10 @@ def Iso_request_set_layout(request: int, layout: int) -> None:
 
 def Iso_request_set_single_launch(request: int, enable: bool) -> None:
     _check(load_library().Iso_request_set_single_launch(request, 1 if enable else 0), "Iso_request_set_single_launch")
+
+
+def Iso_request_set_pipeline(request: int, slabs: int) -> None:
+    _check(load_library().Iso_request_set_pipeline(request, slabs), "Iso_request_set_pipeline")
 
 
 def Iso_request_set_slabs(request: int, slabs: int) -> None:

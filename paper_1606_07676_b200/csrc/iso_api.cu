@@ -50,7 +50,9 @@ void release_device(Request &r)
     r.slab_events.clear();
     if (r.d_counter) cudaFree(r.d_counter);
     r.d_counter = nullptr;
+    r.wave_counters = 0;
     r.multi_grid = 0;
+    r.wave_grid = 0;
     if (r.h_err) cudaFreeHost(r.h_err);
     r.d_blob = nullptr;
     r.d_inter = nullptr;
@@ -136,6 +138,7 @@ int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
 
 LaunchDev make_launch_args(const Request &r, const LaunchPlan &L);
 void choose_slab_plan(Request &r);
+int build_wave(Request &r, unsigned char *blob, size_t launches_off, size_t items_off, size_t slabs);
 
 // One descriptor per unit position of a vector launch: parts in their order, the units of
 // a part in address order.
@@ -168,9 +171,10 @@ void fill_units(const Request &r, const LaunchPlan &L, UnitDev *ud)
         }
         u.src_buf = (uint8_t)lp.p.src_buf;
         u.dst_buf = (uint8_t)lp.p.dst_buf;
+        u.width = (uint8_t)lp.width;
         for (uint32_t k = 0; k < lp.units; ++k) {
-            u.src_term = delta * stride[lp.p.src_buf] + lp.p.src_off + (int64_t)k * L.width;
-            u.dst_term = lp.p.dst_off + (int64_t)k * L.width;
+            u.src_term = delta * stride[lp.p.src_buf] + lp.p.src_off + (int64_t)k * lp.width;
+            u.dst_term = lp.p.dst_off + (int64_t)k * lp.width;
             units[lp.first_unit + k] = u;
         }
     }
@@ -184,6 +188,23 @@ int materialise(Request &r)
     // a captured graph holds the addresses of the tables and buffers that are replaced below
     if (r.graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.graph_exec));
     r.graph_exec = nullptr;
+    // pipelined one-launch execution: every launch must be a 16-byte vector launch of at most
+    // 256 threads on periodic dimensions.  Decided on a trial lowering (device allocations
+    // are 256-byte aligned) because the size of the intermediate buffer depends on it.
+    r.wave_ok = false;
+    r.wave_grid = 0;
+    r.wave_slabs = 0;
+    if (r.wave_request > 0) {
+        int rc0 = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, 0);
+        if (rc0 != ISO_SUCCESS) return rc0;
+        bool ok = !r.launches.empty();
+        for (const LaunchPlan &L : r.launches) {
+            if (L.kernel != KERNEL_VEC || L.width != 16 || L.threads > 256) ok = false;
+            for (int k = 0; k < L.n_used; ++k)
+                if (!c.periodic[L.used_dim[k]]) ok = false;
+        }
+        r.wave_ok = ok;
+    }
     choose_slab_plan(r);
     // device tables depend on the alignment of the intermediate buffer: allocate it first
     const int64_t inter_bytes = r.inter_rows * r.inter_stride;
@@ -211,7 +232,7 @@ int materialise(Request &r)
         if (L.kernel == KERNEL_VEC) bytes += (size_t)L.units_per_proc * sizeof(UnitDev);
     }
     // one-launch execution: every launch is a 16-byte vector launch on periodic dimensions
-    bool single = r.persistent && r.launches.size() >= 2;
+    bool single = r.persistent && !r.wave_ok && r.launches.size() >= 2;
     for (const LaunchPlan &L : r.launches) {
         if (L.kernel != KERNEL_VEC || L.width != 16 || L.threads > 256) single = false;
         for (int k = 0; k < L.n_used; ++k)
@@ -220,6 +241,15 @@ int materialise(Request &r)
     bytes = (bytes + 127) / 128 * 128;
     const size_t launches_off = bytes;
     if (single) bytes += r.launches.size() * sizeof(LaunchDev);
+    // pipelined one-launch execution: one descriptor and one item record per (slab, launch)
+    const size_t wave_slabs = r.wave_ok ? std::max<size_t>(1, r.slab_plan.size()) : 0;
+    const size_t wave_n = wave_slabs * r.launches.size();
+    bytes = (bytes + 127) / 128 * 128;
+    const size_t wave_launches_off = bytes;
+    bytes += wave_n * sizeof(LaunchDev);
+    bytes = (bytes + 127) / 128 * 128;
+    const size_t wave_items_off = bytes;
+    bytes += wave_n * sizeof(WaveItem);
     std::vector<unsigned char> blob(bytes ? bytes : 16, 0);
     for (const LaunchPlan &L : r.launches) {
         int used_index[ISO_MAX_DIMS];
@@ -259,12 +289,24 @@ int materialise(Request &r)
     r.d_blob = nullptr;
     ISO_CUDA(cudaMalloc(&r.d_blob, blob.size()));
     r.multi_grid = 0;
-    if (single) {
-        if (!r.d_counter) {
-            ISO_CUDA(cudaMalloc((void **)&r.d_counter, sizeof(unsigned long long)));
-            ISO_CUDA(cudaMemset(r.d_counter, 0, sizeof(unsigned long long)));
-            r.epoch = 0;
+    if (single || wave_n > 0) {
+        const int need = (int)std::max<size_t>(1, wave_n);
+        if (!r.d_counter || r.wave_counters < need) {
+            if (r.d_counter) cudaFree(r.d_counter);
+            r.d_counter = nullptr;
+            ISO_CUDA(cudaMalloc((void **)&r.d_counter, (size_t)need * sizeof(unsigned long long)));
+            r.wave_counters = need;
         }
+        // a changed plan counts afresh
+        ISO_CUDA(cudaMemset(r.d_counter, 0, (size_t)r.wave_counters * sizeof(unsigned long long)));
+        r.epoch = 0;
+        r.wave_run = 0;
+    }
+    if (wave_n > 0) {
+        int rcw = build_wave(r, blob.data(), wave_launches_off, wave_items_off, wave_slabs);
+        if (rcw != ISO_SUCCESS) return rcw;
+    }
+    if (single) {
         // the grid must be resident as a whole: ask how many CTAs fit
         const size_t smem = (sizeof(LaunchDev) + 127) / 128 * 128 + (size_t)kVecDepth * 256 * 16;
         ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows_multi<kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -350,6 +392,82 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
     return a;
 }
 
+// Item list of the pipelined one-launch execution.  Slabs are taken two at a time and
+// their launches interleaved: (a, l0), (b, l0), (a, l1), (b, l1), ... so that between an
+// item and the one it waits for lies an item of the other slab.  With three or more slabs
+// the intermediate buffer holds two slabs (even and odd ones alternate between the halves).
+// An item waits for the latest of: the launches of earlier phases on its own slab, and -
+// if it writes intermediate places - every launch of the slab that used its half before.
+int build_wave(Request &r, unsigned char *blob, size_t launches_off, size_t items_off, size_t n_slabs)
+{
+    const Comm &c = *r.comm;
+    const size_t nl = r.launches.size();
+    const size_t n = n_slabs * nl;
+    const size_t smem = (sizeof(LaunchDev) + 127) / 128 * 128 + (size_t)kVecDepth * 256 * 16;
+    ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows_wave<kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_wave<kVecDepth>, 256, smem));
+    int want = 4;
+    if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
+        int v = std::atoi(env);
+        if (v >= 1 && v <= 8) want = v;
+    }
+    per_sm = std::min(per_sm, want);
+    if (per_sm < 1) return ISO_SUCCESS;  // cannot be resident: Iso_Start falls back to one launch per phase
+    const int grid = per_sm * r.sm_count;
+
+    std::vector<std::pair<long long, long long>> slabs = r.slab_plan;
+    if (slabs.empty()) slabs.push_back({0, c.P});
+    long long slab_rows = 0;
+    for (const auto &w : slabs) slab_rows = std::max(slab_rows, w.second - w.first);
+    const bool halves = slabs.size() >= 3;
+
+    LaunchDev *ld = reinterpret_cast<LaunchDev *>(blob + launches_off);
+    WaveItem *items = reinterpret_cast<WaveItem *>(blob + items_off);
+    std::vector<int> index_of(n, -1);        // (slab, launch) -> item
+    std::vector<int> last_of_slab(slabs.size(), -1);
+    std::vector<char> writes_inter(nl, 0);
+    for (size_t l = 0; l < nl; ++l)
+        for (const LoweredPart &lp : r.launches[l].parts)
+            if (lp.p.dst_buf == ISO_BUF_INTER) writes_inter[l] = 1;
+    size_t i = 0;
+    unsigned long long groups_so_far = 0;
+    for (size_t k0 = 0; k0 < slabs.size(); k0 += 2) {
+        const size_t k1 = std::min(slabs.size(), k0 + 2);
+        for (size_t l = 0; l < nl; ++l)
+            for (size_t k = k0; k < k1; ++k) {
+                const LaunchPlan &L = r.launches[l];
+                LaunchDev a = make_launch_args(r, L);
+                a.row_lo = slabs[k].first;
+                a.row_hi = slabs[k].second;
+                if (halves && a.buf[ISO_BUF_INTER])
+                    a.buf[ISO_BUF_INTER] -= (slabs[k].first - (long long)(k & 1) * slab_rows) * r.inter_stride;
+                ld[i] = a;
+                WaveItem it{};
+                it.wait_item = -1;
+                for (size_t l2 = 0; l2 < nl; ++l2)
+                    if (r.launches[l2].phase < L.phase && index_of[k * nl + l2] >= 0)
+                        it.wait_item = std::max(it.wait_item, index_of[k * nl + l2]);
+                if (halves && writes_inter[l] && k >= 2) it.wait_item = std::max(it.wait_item, last_of_slab[k - 2]);
+                it.cta_offset = (uint32_t)(groups_so_far % (unsigned long long)grid);
+                const int count = L.compact ? L.max_nnz : L.n_used;
+                it.variant = L.compact ? (count <= 3 ? 4 + std::max(1, count) : 8) : (count <= 3 ? count : 4);
+                items[i] = it;
+                index_of[k * nl + l] = (int)i;
+                last_of_slab[k] = (int)i;
+                groups_so_far += (unsigned long long)((a.row_hi - a.row_lo + L.rows_per_pass - 1) / L.rows_per_pass);
+                ++i;
+            }
+    }
+    r.wave_grid = grid;
+    r.wave_items = (int)n;
+    r.wave_smem = smem;
+    r.wave_launches_off = launches_off;
+    r.wave_items_off = items_off;
+    r.wave_slabs = (int)slabs.size();
+    return ISO_SUCCESS;
+}
+
 // Grid for the rows [a.row_lo, a.row_hi): the plan's grid scaled to the share of the rows.
 unsigned grid_for_rows(const LaunchPlan &L, const LaunchDev &a, int share = 1)
 {
@@ -412,7 +530,7 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
     cudaError_t e;
     if (L.kernel == KERNEL_BULK) {
         e = launch_kernel(iso_gather_bulk, L, a, stream, dependent);
-    } else if (L.width < 4) {
+    } else if (L.width > 0 && L.width < 4) {
         e = L.width == 2 ? launch_kernel(iso_gather_rows_reg<2, 4>, L, a, stream, dependent)
                          : launch_kernel(iso_gather_rows_reg<1, 4>, L, a, stream, dependent);
     } else {
@@ -421,8 +539,8 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
         const int count = L.compact ? L.max_nnz : L.n_used;
         const int nu = count <= 3 ? count : ISO_MAX_DIMS;
 #define ISO_ROWS(W, NU, MESH, COMPACT)                                                                          \
-    e = (W == 16 && L.threads > 256)                                                                            \
-            ? launch_wide(iso_gather_rows_wide<16, kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent)        \
+    e = ((W == 16 || W == 0) && L.threads > 256)                                                                \
+            ? launch_wide(iso_gather_rows_wide<(W == 0 ? 0 : 16), kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent) \
             : launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent)
 #define ISO_ROWS_W(W)                                                            \
     do {                                                                         \
@@ -437,7 +555,8 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
         else if (nu == 3) ISO_ROWS(W, 3, false, false);                          \
         else ISO_ROWS(W, ISO_MAX_DIMS, false, false);                            \
     } while (0)
-        if (L.width == 16) ISO_ROWS_W(16);
+        if (L.width == 0) ISO_ROWS_W(0);
+        else if (L.width == 16) ISO_ROWS_W(16);
         else if (L.width == 8) ISO_ROWS_W(8);
         else ISO_ROWS_W(4);
 #undef ISO_ROWS_W
@@ -521,6 +640,23 @@ void choose_slab_plan(Request &r)
     r.chains = 1;
     r.use_graph = !r.persistent && r.graph_request;
     if (const char *env = std::getenv("ISO_GRAPH")) r.use_graph = !r.persistent && std::atoi(env) != 0;
+    if (r.wave_ok) {
+        // pipelined one-launch execution: its own slabs; from three slabs on the
+        // intermediate buffer holds two of them
+        r.use_graph = false;
+        if (r.wave_request >= 2 && r.inter_stride > 0) {
+            std::vector<SlabPlan> slabs;
+            plan_slabs(r, slabs, r.wave_request);
+            long long rows = 0;
+            if (slabs.size() >= 2)
+                for (const SlabPlan &w : slabs) {
+                    r.slab_plan.push_back({w.row_lo, w.row_hi});
+                    rows = std::max(rows, w.row_hi - w.row_lo);
+                }
+            if (r.slab_plan.size() >= 3) r.inter_rows = 2 * rows;
+        }
+        return;
+    }
     if (r.persistent || r.inter_stride == 0) return;
     int want = r.slab_request;
     if (const char *env = std::getenv("ISO_SLABS")) want = std::atoi(env);
@@ -836,6 +972,20 @@ int Iso_request_set_single_launch(Iso_request request, int enable)
     });
 }
 
+int Iso_request_set_pipeline(Iso_request request, int slabs)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request) || slabs < 0) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    request->wave_request = slabs;
+    request->dirty = true;
+    return ISO_SUCCESS;
+    });
+}
+
 int Iso_request_set_slabs(Iso_request request, int slabs)
 {
     return guarded([&]() -> int {
@@ -894,7 +1044,7 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int cold)
     if (check_handle(request)) return ISO_ERR_ARG;
     Request &r = *request;
     if (!r.send || !r.recv) return ISO_ERR_STATE;
-    if (r.persistent) return ISO_SUCCESS;
+    if (r.persistent || r.wave_request > 0) return ISO_SUCCESS;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaEvent_t t0 = nullptr, t1 = nullptr;
     ISO_CUDA(cudaEventCreate(&t0));
@@ -1026,6 +1176,31 @@ int Iso_Start(Iso_request request, void *cuda_stream)
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     static const bool use_pdl = !(std::getenv("ISO_NO_PDL") && std::atoi(std::getenv("ISO_NO_PDL")) != 0);
+    if (r.wave_grid > 0) {
+        // one cooperative launch that works through the (slab, launch) items
+        WaveDev m{};
+        m.launches = reinterpret_cast<const LaunchDev *>(static_cast<unsigned char *>(r.d_blob) + r.wave_launches_off);
+        m.items = reinterpret_cast<const WaveItem *>(static_cast<unsigned char *>(r.d_blob) + r.wave_items_off);
+        m.n = r.wave_items;
+        m.done = r.d_counter;
+        r.wave_run += 1;
+        m.target = r.wave_run * (unsigned long long)r.wave_grid;
+        m.err = r.d_err;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)r.wave_grid);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = r.wave_smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        ISO_CUDA(cudaLaunchKernelEx(&cfg, iso_gather_rows_wave<kVecDepth>, m));
+        r.last_stream = cuda_stream;
+        r.started = true;
+        return ISO_SUCCESS;
+    }
     if (r.multi_grid > 0) {
         // all phases in one cooperative launch with grid barriers in between
         MultiDev m{};
@@ -1104,7 +1279,7 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
     const unsigned char *hs = static_cast<const unsigned char *>(host_sendbuf);
     unsigned char *hr = static_cast<unsigned char *>(host_recvbuf);
     std::vector<SlabPlan> slabs;
-    if (r.multi_grid == 0) plan_slabs(r, slabs);
+    if (r.multi_grid == 0 && r.wave_grid == 0) plan_slabs(r, slabs);
     // with a one-slab intermediate buffer the upload slabs must fit into it
     for (const SlabPlan &w : slabs)
         if (w.row_hi - w.row_lo > r.inter_rows) { slabs.clear(); break; }
@@ -1188,8 +1363,9 @@ int Iso_wait(Iso_request request)
         cudaMemsetAsync(r.d_err, 0, sizeof(int), stream);
         if (r.d_counter) {
             // a barrier gave up: start counting afresh
-            cudaMemsetAsync(r.d_counter, 0, sizeof(unsigned long long), stream);
+            cudaMemsetAsync(r.d_counter, 0, (size_t)std::max(1, r.wave_counters) * sizeof(unsigned long long), stream);
             r.epoch = 0;
+            r.wave_run = 0;
         }
         return ISO_ERR_TIMEOUT;
     }
@@ -1200,8 +1376,8 @@ int Iso_request_get_stats(Iso_request request, Iso_stats *out)
 {
     if (check_handle(request) || !out) return ISO_ERR_ARG;
     *out = request->stats;
-    if (!request->dirty && request->multi_grid > 0) out->launches = 1;
-    if (!request->dirty && request->slab_plan.size() > 1) out->launches *= (int)request->slab_plan.size();
+    if (!request->dirty && (request->multi_grid > 0 || request->wave_grid > 0)) out->launches = 1;
+    else if (!request->dirty && request->slab_plan.size() > 1) out->launches *= (int)request->slab_plan.size();
     return ISO_SUCCESS;
 }
 
@@ -1220,7 +1396,7 @@ int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int 
                 q.src_buf = lp.p.src_buf;
                 q.dst_buf = lp.p.dst_buf;
                 q.kernel = L.kernel;
-                q.width = L.width;
+                q.width = lp.width;
                 q.src_off = lp.p.src_off;
                 q.dst_off = lp.p.dst_off;
                 q.len = lp.p.len;

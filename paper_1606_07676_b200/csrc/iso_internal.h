@@ -50,6 +50,7 @@ struct LoweredPart {
     Part p;            // offsets / len of this piece
     uint32_t first_unit = 0;
     uint32_t units = 0;
+    int width = 16;    // bytes per unit of this piece (differs between pieces in a launch of mixed widths)
 };
 
 enum { KERNEL_VEC = 0, KERNEL_BULK = 1 };
@@ -58,7 +59,7 @@ constexpr int kVecDepth = 8;        // cp.async ring slots per thread in the vec
 
 struct LaunchPlan {
     int kernel = KERNEL_VEC;
-    int width = 16;       // bytes per unit (vector kernel); chunk bytes (bulk kernel)
+    int width = 16;       // bytes per unit (vector kernel; 0: mixed, every piece has its own); chunk bytes (bulk kernel)
     int phase = 0;
     std::vector<LoweredPart> parts;
     uint32_t units_per_proc = 0;
@@ -120,6 +121,15 @@ struct Request {
     int chains = 1;             // slabs that run side by side (each on its share of the SMs)
     bool use_graph = false;     // Iso_Start replays a captured graph of the launches
     void *graph_exec = nullptr; // cudaGraphExec_t, built at the first Iso_Start after a change
+    // pipelined one-launch execution (items = slab x launch, per-item completion counters)
+    int wave_request = 0;       // 0: off, 1: one slab, n >= 2: n slabs of dimension 0
+    bool wave_ok = false;       // the lowered schedule allows it (decided before the buffers are sized)
+    int wave_slabs = 0;         // slabs in use (0: not in this mode)
+    int wave_grid = 0;          // > 0: Iso_Start makes one cooperative launch of this many CTAs
+    int wave_items = 0;
+    size_t wave_smem = 0, wave_launches_off = 0, wave_items_off = 0;
+    unsigned long long wave_run = 0;  // starts since the counters were last zeroed
+    int wave_counters = 0;      // counters allocated in d_counter
 };
 
 // Builds r.parts, r.inter_stride and the schedule statistics from r.comm, r.kind, r.alg,

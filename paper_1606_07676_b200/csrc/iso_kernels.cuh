@@ -45,7 +45,8 @@ struct alignas(16) UnitDev {
     // along used dimension e, 0 for none.  Compact form: only the shifted dimensions are
     // listed, c[e] != 0 along used dimension dim[e] for e < nnz.
     int32_t c[ISO_MAX_DIMS];
-    uint8_t src_buf, dst_buf, nnz, pad0;
+    uint8_t src_buf, dst_buf, nnz;
+    uint8_t width;  // bytes of this unit (launches of mixed unit widths; otherwise the launch's width)
     uint8_t dim[ISO_MAX_DIMS];
     uint8_t pad1[4];
 };
@@ -146,6 +147,7 @@ __device__ __forceinline__ UnitAddr decode_unit(const LaunchDev &L, long long r0
 }
 
 template <int W> struct VecOf;
+template <> struct VecOf<0> { using type = uint4; };  // mixed widths: slots of the widest unit
 template <> struct VecOf<16> { using type = uint4; };
 template <> struct VecOf<8> { using type = uint2; };
 template <> struct VecOf<4> { using type = uint32_t; };
@@ -174,6 +176,31 @@ template <> __device__ __forceinline__ void cp_async<4>(void *smem_dst, const vo
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
                  : "memory");
 }
+// W = 0: the width is the unit's own (4, 8 or 16 bytes), known only at run time
+template <int W> __device__ __forceinline__ void cp_async_unit(void *smem_dst, const void *gsrc, uint32_t w)
+{
+    if (W != 0) {
+        cp_async<(W != 0 ? W : 16)>(smem_dst, gsrc);
+    } else if (w == 16) {
+        cp_async<16>(smem_dst, gsrc);
+    } else if (w == 8) {
+        cp_async<8>(smem_dst, gsrc);
+    } else {
+        cp_async<4>(smem_dst, gsrc);
+    }
+}
+template <int W> __device__ __forceinline__ void store_unit(unsigned char *dst, const typename VecOf<W>::type *slot, uint32_t w)
+{
+    if (W != 0) {
+        *reinterpret_cast<typename VecOf<W>::type *>(dst) = *slot;
+    } else if (w == 16) {
+        *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(slot);
+    } else if (w == 8) {
+        *reinterpret_cast<uint2 *>(dst) = *reinterpret_cast<const uint2 *>(slot);
+    } else {
+        *reinterpret_cast<uint32_t *>(dst) = *reinterpret_cast<const uint32_t *>(slot);
+    }
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -184,6 +211,7 @@ struct UnitRegs {
     long long stride_s, stride_d;
     int c[ISO_MAX_DIMS];
     uint32_t nnz;
+    uint32_t width;
     uint32_t dims_lo, dims_hi;  // dim[0..3], dim[4..7], one byte each
 };
 
@@ -202,6 +230,7 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
     R.c[0] = (int)b.x; R.c[1] = (int)b.y; R.c[2] = (int)b.z; R.c[3] = (int)b.w;
     R.c[4] = (int)c.x; R.c[5] = (int)c.y; R.c[6] = (int)c.z; R.c[7] = (int)c.w;
     R.nnz = (d.x >> 16) & 0xff;
+    R.width = d.x >> 24;
     R.dims_lo = d.y;
     R.dims_hi = d.z;
     return R;
@@ -217,6 +246,11 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
 // shifted dimension - the row's coordinate by exact 32-bit division - and two pointer
 // increments.
 //
+// W = 0 is a launch of mixed unit widths (every unit 4, 8 or 16 bytes wide, as its
+// descriptor says): the ragged rows of the irregular collectives then take one launch per
+// phase instead of one per width, and pieces that share a 32-byte sector are moved at the
+// same time by the same CTA.
+//
 // Data path for W in {16, 8, 4}: cp.async from global memory into a thread-private ring of
 // DEPTH slots in shared memory, so that DEPTH loads per thread are in flight without
 // holding registers; a slot is read back and stored to its destination as soon as the
@@ -230,7 +264,8 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
 // them (the last phase of a schedule whose final hops were postponed, the direct schedule
 // in high dimension), then tests per row only the dimensions its unit moves along.
 template <int W, int DEPTH, int NU, bool MESH, bool COMPACT>
-__device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned char *ring_base, bool dependent_launch)
+__device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned char *ring_base, bool dependent_launch,
+                                                 uint32_t cta, uint32_t n_cta)
 {
     using V = typename VecOf<W>::type;
     V *const ring = reinterpret_cast<V *>(ring_base) + threadIdx.x;  // slot k at ring[k * blockDim.x]
@@ -240,7 +275,7 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
     const int G = (int)L.rows_per_pass;
     const int g = (int)(threadIdx.x / CU);
     const uint32_t ul = threadIdx.x - (uint32_t)g * CU;
-    const long long r0 = L.row_lo + (long long)G * blockIdx.x + g;
+    const long long r0 = L.row_lo + (long long)G * cta + g;
     const bool active = g < G && r0 < L.row_hi && ul < U;
     // the tables are not produced by kernels: fetch the first descriptor before ordering
     // behind the previous kernel
@@ -251,7 +286,7 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
         grid_launch_dependents();
     }
     if (!active) return;
-    const long long rstep = (long long)G * gridDim.x;
+    const long long rstep = (long long)G * n_cta;
     const long long r_end = L.row_hi;
 
     for (uint32_t u = ul; u < U; u += CU) {
@@ -293,7 +328,7 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
         for (int i = 0; i < DEPTH; ++i) {
             if (r_ld < r_end) {
                 const unsigned char *src;
-                if (source(src_ld, r_ld, src)) cp_async<W>(ring + i * blockDim.x, src);
+                if (source(src_ld, r_ld, src)) cp_async_unit<W>(ring + i * blockDim.x, src, R.width);
                 r_ld += rstep;
                 src_ld += src_step;
             }
@@ -307,11 +342,11 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
                 const unsigned char *ignored;
                 valid = source(nullptr, r, ignored);
             }
-            if (valid) *reinterpret_cast<V *>(dst) = *slot;
+            if (valid) store_unit<W>(dst, slot, R.width);
             dst += dst_step;
             if (r_ld < r_end) {
                 const unsigned char *src;
-                if (source(src_ld, r_ld, src)) cp_async<W>(slot, src);
+                if (source(src_ld, r_ld, src)) cp_async_unit<W>(slot, src, R.width);
                 r_ld += rstep;
                 src_ld += src_step;
             }
@@ -327,7 +362,7 @@ template <int W, int DEPTH, int NU, bool MESH, bool COMPACT>
 __global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant__ LaunchDev L)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true);
+    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true, blockIdx.x, gridDim.x);
 }
 
 // The same body in CTAs of up to 1024 threads, for launches whose payload per process has
@@ -337,7 +372,7 @@ template <int W, int DEPTH, int NU, bool MESH, bool COMPACT>
 __global__ void __launch_bounds__(1024, 1) iso_gather_rows_wide(const __grid_constant__ LaunchDev L)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true);
+    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true, blockIdx.x, gridDim.x);
 }
 
 // All phases of a schedule in ONE cooperative launch: the CTAs run phase after phase and
@@ -397,13 +432,95 @@ __global__ void __launch_bounds__(256, 4) iso_gather_rows_multi(const __grid_con
         for (uint32_t i = threadIdx.x; i < sizeof(LaunchDev) / 4; i += blockDim.x) dst[i] = __ldg(src + i);
         __syncthreads();
         switch (sL->n_used) {
-        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false); break;
-        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false); break;
-        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false); break;
-        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false); break;
-        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false); break;
+        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
+        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
+        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
+        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
+        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
         }
         if (ph + 1 < M.n && !grid_barrier(M, M.epoch + (unsigned long long)(ph + 1) * gridDim.x, &s_ok)) return;
+    }
+}
+
+// Pipelined one-launch execution.  The torus is cut into slabs of planes of dimension 0
+// and the work into items (slab, launch of the schedule); all CTAs go through the items in
+// one fixed order, each taking its share of an item's rows.  Instead of a grid barrier
+// between phases, every item has a counter of the CTAs that have finished it, and a CTA
+// starts item i once the item it depends on (the slab's previous phase, or the last reader
+// of the intermediate place it overwrites) has been finished by all CTAs.  The order puts
+// other items in between, so that wait is normally over before it begins, and a slab's
+// intermediate blocks are read back a few items after they were written, out of L2.
+struct WaveItem {
+    int wait_item;        // item that must be complete first (-1: none)
+    uint32_t cta_offset;  // rotation of the CTA numbering, continues the round robin of the item before
+    int variant;          // 0..4: dense descriptors with 0, 1, 2, 3, any shifted dimensions; 5..8: compact with 1, 2, 3, any
+    int pad;
+};
+
+struct WaveDev {
+    const LaunchDev *launches;  // one complete descriptor per item (row range and buffers set)
+    const WaveItem *items;
+    int n;
+    unsigned long long *done;   // per item: arrivals of CTAs, never reset
+    unsigned long long target;  // arrivals that mean "complete" for this start
+    int *err;                   // set to 2 when a wait gives up
+};
+
+template <int DEPTH>
+__global__ void __launch_bounds__(256, 4) iso_gather_rows_wave(const __grid_constant__ WaveDev M)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ int s_ok;
+    __shared__ WaveItem s_item;
+    LaunchDev *sL = reinterpret_cast<LaunchDev *>(smem_raw);
+    unsigned char *ring = smem_raw + ((sizeof(LaunchDev) + 127) / 128) * 128;
+    for (int i = 0; i < M.n; ++i) {
+        const uint32_t *src = reinterpret_cast<const uint32_t *>(M.launches + i);
+        uint32_t *dst = reinterpret_cast<uint32_t *>(sL);
+        for (uint32_t k = threadIdx.x; k < sizeof(LaunchDev) / 4; k += blockDim.x) dst[k] = __ldg(src + k);
+        if (threadIdx.x == 0) {
+            const WaveItem it = M.items[i];
+            s_item = it;
+            bool ok = true;
+            if (it.wait_item >= 0) {
+                const unsigned long long *flag = M.done + it.wait_item;
+                uint32_t polls = 0;
+                for (;;) {
+                    unsigned long long seen;
+                    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(flag) : "memory");
+                    if (seen >= M.target) break;
+                    if (++polls >= kBarrierPolls) {
+                        ok = false;
+                        break;
+                    }
+                    __nanosleep(32);
+                }
+                if (!ok) atomicExch(M.err, 2);
+            }
+            s_ok = ok ? 1 : 0;
+        }
+        __syncthreads();
+        if (!s_ok) return;
+        const uint32_t n_cta = gridDim.x;
+        uint32_t cta = blockIdx.x + n_cta - s_item.cta_offset;
+        if (cta >= n_cta) cta -= n_cta;
+        switch (s_item.variant) {
+        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false, cta, n_cta); break;
+        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false, cta, n_cta); break;
+        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false, cta, n_cta); break;
+        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false, cta, n_cta); break;
+        case 4: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false, cta, n_cta); break;
+        case 5: gather_rows_body<16, DEPTH, 1, false, true>(*sL, ring, false, cta, n_cta); break;
+        case 6: gather_rows_body<16, DEPTH, 2, false, true>(*sL, ring, false, cta, n_cta); break;
+        case 7: gather_rows_body<16, DEPTH, 3, false, true>(*sL, ring, false, cta, n_cta); break;
+        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, true>(*sL, ring, false, cta, n_cta); break;
+        }
+        // all stores of this CTA for the item are issued: publish them and count the CTA in
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();
+            atomicAdd(M.done + i, 1ULL);
+        }
     }
 }
 

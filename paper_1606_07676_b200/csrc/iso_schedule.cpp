@@ -651,7 +651,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
         while (end < r.parts.size() && r.parts[end].phase == r.parts[begin].phase) ++end;
 
         // split every part into pieces that share one alignment class
-        struct Piece { Part p; int kernel; int width; };
+        struct Piece { Part p; int kernel; int width; int cls; };  // cls: width class of the launch (0: mixed widths)
         std::vector<Piece> pieces;
         for (size_t k = begin; k < end; ++k) {
             const Part &p = r.parts[k];
@@ -665,6 +665,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                 q.p.len = len;
                 q.width = std::min(base, common_alignment({q.p.src_off, q.p.dst_off, len}));
                 q.kernel = (q.width == 16 && r.bulk_threshold > 0 && len >= r.bulk_threshold) ? KERNEL_BULK : KERNEL_VEC;
+                q.cls = q.width;
                 pieces.push_back(q);
             };
             const bool co_aligned = base == 16 && ((p.src_off - p.dst_off) & 15) == 0;
@@ -692,16 +693,34 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     if (q.kernel == KERNEL_VEC && q.width == w2) { narrower = w2; break; }
             if (!narrower) continue;
             for (Piece &q : pieces)
-                if (q.kernel == KERNEL_VEC && q.width == width) q.width = narrower;
+                if (q.kernel == KERNEL_VEC && q.width == width) q.width = q.cls = narrower;
+        }
+
+        // Ragged rows (pieces of 4, 8 and 16 bytes in one phase): one launch of mixed unit
+        // widths for all of them instead of one launch per width, so that pieces which share
+        // a 32-byte sector are moved together.  Parts below 4 KB that would have gone to the
+        // bulk kernel join it; they lie between the small pieces.
+        {
+            int classes = 0;
+            for (int width = 16; width >= 4; width >>= 1)
+                for (const Piece &q : pieces)
+                    if (q.kernel == KERNEL_VEC && q.width == width) { ++classes; break; }
+            bool mixed = classes >= 2 && r.wave_request == 0 && !r.persistent;
+            if (const char *env = std::getenv("ISO_MIXED")) mixed = mixed && std::atoi(env) != 0;
+            if (mixed)
+                for (Piece &q : pieces) {
+                    if (q.kernel == KERNEL_BULK && q.p.len < 4096) q.kernel = KERNEL_VEC;
+                    if (q.kernel == KERNEL_VEC && q.width >= 4) q.cls = 0;
+                }
         }
 
         // one launch per (kernel, width) class, in a fixed order
         for (int kernel = 0; kernel < 2; ++kernel) {
-            for (int width = 16; width >= 1; width >>= 1) {
+            for (int width : {0, 16, 8, 4, 2, 1}) {  // 0: the launch of mixed unit widths
                 std::vector<Piece> cls;
                 std::vector<std::pair<size_t, size_t>> ranges;
                 for (const Piece &q : pieces)
-                    if (q.kernel == kernel && q.width == width) cls.push_back(q);
+                    if (q.kernel == kernel && q.cls == width) cls.push_back(q);
                 // a vector launch holds at most kMaxVecUnits unit positions per process (each
                 // gets a descriptor): cut longer lists, splitting a piece at a unit boundary
                 if (kernel == KERNEL_VEC) {
@@ -711,6 +730,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     int64_t used_units = 0;
                     for (Piece q : cls) {
                         while (q.p.len > 0) {
+                            const int width = q.width;  // the piece's own unit width
                             int64_t n = q.p.len / width;
                             int64_t room = cap - used_units;
                             if (room == 0) { bounds.push_back(cut.size()); used_units = 0; room = cap; }
@@ -738,7 +758,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     LaunchPlan L;
                     L.kernel = kernel;
                     L.phase = r.parts[begin].phase;
-                    int64_t unit = width;
+                    int64_t unit = width;  // 0 for mixed widths: every part then counts in its own
                     if (kernel == KERNEL_BULK) {
                         int64_t min_len = INT64_MAX;
                         for (size_t k = lo; k < hi; ++k) min_len = std::min(min_len, cls[k].p.len);
@@ -757,7 +777,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     for (size_t k = lo; k < hi; ++k) {
                         LoweredPart lp;
                         lp.p = cls[k].p;
-                        uint64_t n = (uint64_t)((lp.p.len + unit - 1) / unit);
+                        lp.width = kernel == KERNEL_BULK ? (int)unit : cls[k].width;
+                        uint64_t n = (uint64_t)((lp.p.len + lp.width - 1) / lp.width);
                         if (units + n > 0x7fffffffull) return ISO_ERR_COUNT;
                         lp.first_unit = (uint32_t)units;
                         lp.units = (uint32_t)n;
@@ -780,8 +801,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         }
                     // many shifted dimensions in the launch, few per part: the kernel then
                     // tests per row only the dimensions a unit moves along
-                    L.compact = kernel == KERNEL_VEC && width >= 4 && L.n_used > 3 && L.max_nnz < L.n_used &&
-                                torus && !r.persistent;
+                    L.compact = kernel == KERNEL_VEC && (width >= 4 || width == 0) && L.n_used > 3 && L.max_nnz < L.n_used &&
+                                torus && !r.persistent;  // (the pipelined one-launch kernel does take compact launches)
                     // coarse lookup: unit >> shift -> part
                     if (!uniform) {
                         int shift = 0;
@@ -803,7 +824,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     if (kernel == KERNEL_VEC) {
                         // a row slot covers up to 256 unit positions; short rows share a CTA
                         // 16-byte launches with long rows use CTAs of up to 1024 threads
-                        const uint32_t max_threads = (width == 16 && units > 256) ? 1024 : 256;
+                        const uint32_t max_threads = ((width == 16 || width == 0) && units > 256 && r.wave_request == 0) ? 1024 : 256;
                         L.chunk_units = (uint32_t)std::min<uint64_t>(units, max_threads);
                         L.rows_per_pass = std::max<uint32_t>(1, max_threads == 256 ? 256 / L.chunk_units : 1);
                         L.threads = (int)((L.chunk_units * L.rows_per_pass + 31) / 32 * 32);
@@ -835,7 +856,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     L.grid = grid;
                     if (L.grid > 0x7fffffff) return ISO_ERR_DIMS;
                     L.smem = (size_t)L.n_used * (size_t)tp * sizeof(uint32_t);
-                    if (kernel == KERNEL_VEC) L.smem = width >= 4 ? (size_t)kVecDepth * L.threads * width : 0;
+                    if (kernel == KERNEL_VEC) L.smem = width >= 4 ? (size_t)kVecDepth * L.threads * width : (width == 0 ? (size_t)kVecDepth * L.threads * 16 : 0);
                     if (kernel == KERNEL_BULK)
                         L.smem = (L.smem + 15) / 16 * 16 + (size_t)L.threads * 2 * (size_t)unit + (size_t)L.threads * 2 * 8;
                     r.launches.push_back(std::move(L));

@@ -156,6 +156,49 @@ def test_chains_graph_replay_and_tuning(torch_cuda):
         run.close()
 
 
+def test_pipelined_one_launch_execution(torch_cuda):
+    """One cooperative launch over (slab, launch) items with per-item completion counters:
+    the oracle's result for any slab count, on repeated starts (the counters carry over),
+    for schedules with compact descriptors (cfg4) and wide rows (342 neighbours), and the
+    plain execution again after it is switched off."""
+    torch = torch_cuda
+    for name, algs in [("cfg2_alltoall", [COMB1, COMB0, COMB2, ALT1, DIRECT, TORUS]), ("cfg3_m64", [COMB1, TORUS]),
+                       ("cfg4", [COMB1]), ("cfg2_allgather", [COMB1, COMB0]), ("moore_d3r3_alltoall", [COMB1]),
+                       ("cfg1", [COMB1])]:
+        w = wl.config(name)
+        run = Run(torch, w)
+        want = oracle_result(w, run.send_host)
+        for slabs in (1, 2, 3, 8, 5, 0):
+            iso.Iso_request_set_pipeline(run.req, slabs)
+            for alg, fusion in algs:
+                got = run.result(alg, fusion)
+                assert np.array_equal(got, want), (name, slabs, alg, fusion)
+                st = iso.Iso_request_get_stats(run.req)
+                if slabs > 0 and w.block_bytes % 16 == 0:   # cfg1's 8-byte blocks run as if it were off
+                    assert st["launches"] == 1, (name, slabs, st["launches"])
+                for _ in range(2):   # again, on poisoned receive buffers
+                    run.recv.fill_(0xA5)
+                    iso.Iso_Start(run.req, torch.cuda.current_stream())
+                iso.Iso_wait(run.req)
+                assert np.array_equal(run.recv.cpu().numpy().reshape(want.shape), want), (name, slabs, "restart")
+        run.close()
+    # ragged sizes; a schedule the mode cannot take (4-byte units) runs as if it were off
+    w = wl.Workload("ragged", "alltoall", (37, 53), wl.moore(2, 2), 48, seed=7)
+    run = Run(torch, w)
+    want = oracle_result(w, run.send_host)
+    for slabs in (1, 4, 37):
+        iso.Iso_request_set_pipeline(run.req, slabs)
+        assert np.array_equal(run.result(*COMB1), want), slabs
+    run.close()
+    w = wl.config("cfg5")
+    run = Run(torch, w)
+    iso.Iso_request_set_pipeline(run.req, 4)
+    got = run.result(*COMB1)
+    assert iso.Iso_request_get_stats(run.req)["launches"] > 1
+    assert np.array_equal(got, oracle_result(w, run.send_host))
+    run.close()
+
+
 def test_cfg2_allgather(torch_cuda):
     check(torch_cuda, wl.config("cfg2_allgather"), [COMB0, COMB1, COMB2, COMBD, DIRECT])
 
