@@ -46,7 +46,7 @@ struct alignas(16) UnitDev {
     // listed, c[e] != 0 along used dimension dim[e] for e < nnz.
     int32_t c[ISO_MAX_DIMS];
     uint8_t src_buf, dst_buf, nnz;
-    uint8_t width;  // bytes of this unit (launches of mixed unit widths; otherwise the launch's width)
+    uint8_t width;  // bytes of this unit: 1, 2, 4, 8 or 16 (launches of mixed unit widths; otherwise the launch's width)
     uint8_t dim[ISO_MAX_DIMS];
     uint8_t pad1[4];
 };
@@ -176,29 +176,39 @@ template <> __device__ __forceinline__ void cp_async<4>(void *smem_dst, const vo
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
                  : "memory");
 }
-// W = 0: the width is the unit's own (4, 8 or 16 bytes), known only at run time
-template <int W> __device__ __forceinline__ void cp_async_unit(void *smem_dst, const void *gsrc, uint32_t w)
+// W = 0: the width is the unit's own (1, 2, 4, 8 or 16 bytes), known only at run time.
+// `w` holds the width in its low byte and, for 1- and 2-byte units, the unit's offset inside
+// its aligned 4-byte word in the next one: cp.async moves at least 4 bytes, so such a unit
+// fetches the whole word (rows start on 4-byte boundaries in these launches, so the word
+// lies inside the same row) and stores only its own bytes.
+template <int W> __device__ __forceinline__ void cp_async_unit(void *smem_dst, const unsigned char *gsrc, uint32_t w)
 {
     if (W != 0) {
         cp_async<(W != 0 ? W : 16)>(smem_dst, gsrc);
-    } else if (w == 16) {
+    } else if ((w & 0xff) == 16) {
         cp_async<16>(smem_dst, gsrc);
-    } else if (w == 8) {
+    } else if ((w & 0xff) == 8) {
         cp_async<8>(smem_dst, gsrc);
-    } else {
+    } else if ((w & 0xff) == 4) {
         cp_async<4>(smem_dst, gsrc);
+    } else {
+        cp_async<4>(smem_dst, gsrc - (w >> 8));
     }
 }
 template <int W> __device__ __forceinline__ void store_unit(unsigned char *dst, const typename VecOf<W>::type *slot, uint32_t w)
 {
     if (W != 0) {
         *reinterpret_cast<typename VecOf<W>::type *>(dst) = *slot;
-    } else if (w == 16) {
+    } else if ((w & 0xff) == 16) {
         *reinterpret_cast<uint4 *>(dst) = *reinterpret_cast<const uint4 *>(slot);
-    } else if (w == 8) {
+    } else if ((w & 0xff) == 8) {
         *reinterpret_cast<uint2 *>(dst) = *reinterpret_cast<const uint2 *>(slot);
-    } else {
+    } else if ((w & 0xff) == 4) {
         *reinterpret_cast<uint32_t *>(dst) = *reinterpret_cast<const uint32_t *>(slot);
+    } else {
+        const uint32_t word = *reinterpret_cast<const uint32_t *>(slot) >> (8 * (w >> 8));
+        if ((w & 0xff) == 2) *reinterpret_cast<uint16_t *>(dst) = (uint16_t)word;
+        else *dst = (uint8_t)word;
     }
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -231,6 +241,7 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
     R.c[4] = (int)c.x; R.c[5] = (int)c.y; R.c[6] = (int)c.z; R.c[7] = (int)c.w;
     R.nnz = (d.x >> 16) & 0xff;
     R.width = d.x >> 24;
+    if (R.width < 4) R.width |= ((uint32_t)(uintptr_t)R.A & 3u) << 8;  // offset inside the aligned word
     R.dims_lo = d.y;
     R.dims_hi = d.z;
     return R;
@@ -246,7 +257,7 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
 // shifted dimension - the row's coordinate by exact 32-bit division - and two pointer
 // increments.
 //
-// W = 0 is a launch of mixed unit widths (every unit 4, 8 or 16 bytes wide, as its
+// W = 0 is a launch of mixed unit widths (every unit 1, 2, 4, 8 or 16 bytes wide, as its
 // descriptor says): the ragged rows of the irregular collectives then take one launch per
 // phase instead of one per width, and pieces that share a 32-byte sector are moved at the
 // same time by the same CTA.

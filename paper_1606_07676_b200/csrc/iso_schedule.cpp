@@ -651,7 +651,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
         while (end < r.parts.size() && r.parts[end].phase == r.parts[begin].phase) ++end;
 
         // split every part into pieces that share one alignment class
-        struct Piece { Part p; int kernel; int width; int cls; };  // cls: width class of the launch (0: mixed widths)
+        // cls: width class of the launch (0: mixed widths); base: alignment of the rows it touches
+        struct Piece { Part p; int kernel; int width; int cls; int base; };
         std::vector<Piece> pieces;
         for (size_t k = begin; k < end; ++k) {
             const Part &p = r.parts[k];
@@ -666,6 +667,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                 q.width = std::min(base, common_alignment({q.p.src_off, q.p.dst_off, len}));
                 q.kernel = (q.width == 16 && r.bulk_threshold > 0 && len >= r.bulk_threshold) ? KERNEL_BULK : KERNEL_VEC;
                 q.cls = q.width;
+                q.base = base;
                 pieces.push_back(q);
             };
             const bool co_aligned = base == 16 && ((p.src_off - p.dst_off) & 15) == 0;
@@ -696,21 +698,23 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                 if (q.kernel == KERNEL_VEC && q.width == width) q.width = q.cls = narrower;
         }
 
-        // Ragged rows (pieces of 4, 8 and 16 bytes in one phase): one launch of mixed unit
+        // Ragged rows (pieces of several widths in one phase): one launch of mixed unit
         // widths for all of them instead of one launch per width, so that pieces which share
         // a 32-byte sector are moved together.  Parts below 4 KB that would have gone to the
-        // bulk kernel join it; they lie between the small pieces.
+        // bulk kernel join it; they lie between the small pieces.  1- and 2-byte pieces take
+        // part where every row starts on a 4-byte boundary (they fetch their aligned word).
         {
+            auto eligible = [](const Piece &q) { return q.kernel == KERNEL_VEC && (q.width >= 4 || q.base >= 4); };
             int classes = 0;
-            for (int width = 16; width >= 4; width >>= 1)
+            for (int width = 16; width >= 1; width >>= 1)
                 for (const Piece &q : pieces)
-                    if (q.kernel == KERNEL_VEC && q.width == width) { ++classes; break; }
+                    if (eligible(q) && q.width == width) { ++classes; break; }
             bool mixed = classes >= 2 && r.wave_request == 0 && !r.persistent;
             if (const char *env = std::getenv("ISO_MIXED")) mixed = mixed && std::atoi(env) != 0;
             if (mixed)
                 for (Piece &q : pieces) {
                     if (q.kernel == KERNEL_BULK && q.p.len < 4096) q.kernel = KERNEL_VEC;
-                    if (q.kernel == KERNEL_VEC && q.width >= 4) q.cls = 0;
+                    if (eligible(q)) q.cls = 0;
                 }
         }
 
