@@ -650,6 +650,9 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
         size_t end = begin;
         while (end < r.parts.size() && r.parts[end].phase == r.parts[begin].phase) ++end;
 
+        // whether this phase may run as one launch of mixed unit widths
+        bool allow_mixed = r.wave_request == 0 && !r.persistent;
+        if (const char *env = std::getenv("ISO_MIXED")) allow_mixed = allow_mixed && std::atoi(env) != 0;
         // split every part into pieces that share one alignment class
         // cls: width class of the launch (0: mixed widths); base: alignment of the rows it touches
         struct Piece { Part p; int kernel; int width; int cls; int base; };
@@ -671,7 +674,30 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                 pieces.push_back(q);
             };
             const bool co_aligned = base == 16 && ((p.src_off - p.dst_off) & 15) == 0;
-            if (co_aligned && p.len >= 48 && ((p.src_off & 15) || (p.len & 15))) {
+            // ragged ends are cut into pieces of at most 4 bytes: with 8-byte end pieces the
+            // irregular 64x64x32 workload measured 8 % slower (1.70 against 1.57 ms)
+            const int64_t split_cap = 4;
+            if (co_aligned && allow_mixed && ((p.src_off & 15) || (p.len & 15))) {
+                // the launch of mixed widths takes any unit width: cut the ragged ends into
+                // few aligned power-of-two pieces (a 15-byte head at offset 1 is
+                // 1 + 2 + 4 + 4 + 4) around a body of whole 16-byte units
+                int64_t rel = 0;
+                while (rel < p.len && ((p.src_off + rel) & 15)) {
+                    int64_t a = (p.src_off + rel) & -(p.src_off + rel);  // lowest set bit
+                    a = std::min(a, split_cap);
+                    while (a > p.len - rel) a >>= 1;
+                    push(rel, a);
+                    rel += a;
+                }
+                const int64_t body = (p.len - rel) / 16 * 16;
+                push(rel, body);
+                rel += body;
+                for (int64_t a = split_cap; a >= 1; a >>= 1)
+                    while (p.len - rel >= a) {
+                        push(rel, a);
+                        rel += a;
+                    }
+            } else if (co_aligned && p.len >= 48 && ((p.src_off & 15) || (p.len & 15))) {
                 int64_t head = (16 - (p.src_off & 15)) & 15;
                 int64_t body = (p.len - head) / 16 * 16;
                 push(0, head);
@@ -709,9 +735,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
             for (int width = 16; width >= 1; width >>= 1)
                 for (const Piece &q : pieces)
                     if (eligible(q) && q.width == width) { ++classes; break; }
-            bool mixed = classes >= 2 && r.wave_request == 0 && !r.persistent;
-            if (const char *env = std::getenv("ISO_MIXED")) mixed = mixed && std::atoi(env) != 0;
-            if (mixed)
+            if (classes >= 2 && allow_mixed)
                 for (Piece &q : pieces) {
                     if (q.kernel == KERNEL_BULK && q.p.len < 4096) q.kernel = KERNEL_VEC;
                     if (eligible(q)) q.cls = 0;
