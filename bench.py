@@ -523,8 +523,13 @@ def sweep(torch, iso, wl, peak, args):
         reps = Replicas(torch, iso, wl, name)
         row = {}
         for key, alg, fusion in (("combining", iso.ISO_ALG_COMBINING, 1), ("combining_per_round", iso.ISO_ALG_COMBINING, 0),
-                                 ("direct", iso.ISO_ALG_DIRECT, 1)):
+                                 ("direct", iso.ISO_ALG_DIRECT, 1), ("combining_tuned", iso.ISO_ALG_COMBINING, 1)):
+            # the last row: the same schedule after Iso_request_tune has timed slabs x chains x
+            # graph replay (cold caches) and kept the fastest plan
+            was = Bound.tune
+            Bound.tune = was or key == "combining_tuned"
             st = reps.set(alg, fusion)
+            Bound.tune = was
             steps = 40 if st["bytes_moved"] < (4 << 30) else 6
             ms = time_run(torch, reps.start, steps, 4)
             row[key] = {"rounds": st["rounds"], "launches": st["launches"], "execution": reps.execution(),

@@ -204,7 +204,7 @@ void emit_hop(Request &r, int phase, int round, int slot, const int *shift, int 
 // region per process and reads a few contiguous regions, and the receive buffer is written
 // only by final hops.  The hops, their order and the bytes moved are unchanged; the
 // intermediate buffer grows from one place per multi-hop block to (hops - 1) places.
-void pack_intermediates(Request &r, int s)
+void pack_intermediates(Request &r, int s, bool final_by_dst)
 {
     std::vector<std::vector<size_t>> chain(s);  // indices of a slot's hops, in execution order
     for (size_t k = 0; k < r.parts.size(); ++k) chain[r.parts[k].slot].push_back(k);
@@ -253,8 +253,17 @@ void pack_intermediates(Request &r, int s)
     }
     r.inter_stride = round_up(cur, 16);
     // inside a phase, take the parts in the order of their source addresses
-    std::stable_sort(r.parts.begin(), r.parts.end(), [](const Part &a, const Part &b) {
+    // (the phase of the postponed final hops of 16-byte blocks in the order of the receive
+    // buffer instead: whole-row stores and scattered loads measured 5 % faster there than
+    // the other way round, 185 against 196 microseconds on the 8^5 torus)
+    int last_phase = 0;
+    for (const Part &p : r.parts) last_phase = std::max(last_phase, p.phase);
+    std::stable_sort(r.parts.begin(), r.parts.end(), [&](const Part &a, const Part &b) {
         if (a.phase != b.phase) return a.phase < b.phase;
+        if (final_by_dst && a.phase == last_phase) {
+            if (a.dst_buf != b.dst_buf) return a.dst_buf < b.dst_buf;
+            return a.dst_off < b.dst_off;
+        }
         if (a.src_buf != b.src_buf) return a.src_buf < b.src_buf;
         return a.src_off < b.src_off;
     });
@@ -354,7 +363,10 @@ int build_combining_alltoall(Request &r, const Geometry &g)
     }
     // on a mesh the receive buffer must not serve as scratch (an undelivered slot keeps its
     // contents), so the packed layout is used whatever was asked for
-    if (r.layout == ISO_LAYOUT_PACKED || mesh) pack_intermediates(r, g.s);
+    bool full_units = true;  // every block fills whole 16-byte units
+    for (int i = 0; i < g.s; ++i)
+        if (r.len[i] > 0 && r.len[i] % 16 != 0) full_units = false;
+    if (r.layout == ISO_LAYOUT_PACKED || mesh) pack_intermediates(r, g.s, lazy_final && full_units);
     // blocks for the process itself: one local copy, together with the first phase
     for (Part &p : locals_parts) p.phase = 0;
     r.parts.insert(r.parts.begin(), locals_parts.begin(), locals_parts.end());
