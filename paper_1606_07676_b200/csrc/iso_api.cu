@@ -570,6 +570,7 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
 struct SlabPlan {
     long long row_lo, row_hi;
     int last_needed;  // index of the last slab whose send buffers this slab's schedule reads
+    unsigned long long needs;  // bit j: the slab's schedule reads send buffers of slab j (valid up to 64 slabs)
 };
 
 // Fills `slabs` when the schedule can run slab by slab: every part that shifts along
@@ -605,12 +606,13 @@ void plan_slabs(const Request &r, std::vector<SlabPlan> &slabs, int want = 0)
     for (int k = 0; k < n; ++k) {
         const int a = (int)((long long)p0 * k / n), b = (int)((long long)p0 * (k + 1) / n);
         for (int x = a; x < b; ++x) slab_of[x] = k;
-        slabs.push_back(SlabPlan{a * plane, b * plane, k});
+        slabs.push_back(SlabPlan{a * plane, b * plane, k, 0ULL});
     }
     for (int x = 0; x < p0; ++x)
         for (int s0 : shifts) {
             const int src = ((x - s0) % p0 + p0) % p0;
             slabs[slab_of[x]].last_needed = std::max(slabs[slab_of[x]].last_needed, slab_of[src]);
+            if (slab_of[src] < 64) slabs[slab_of[x]].needs |= 1ULL << slab_of[src];
         }
 }
 
@@ -1315,16 +1317,31 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
     ISO_CUDA(cudaStreamWaitEvent(up, fence, 0));
     ISO_CUDA(cudaStreamWaitEvent(down, fence, 0));
     static const bool use_pdl = !(std::getenv("ISO_NO_PDL") && std::atoi(std::getenv("ISO_NO_PDL")) != 0);
+    // Upload order: the last slab first, then 0, 1, ...: on a torus slab 0 reads the last slab,
+    // so in natural order it (and its download) would have to wait for the very last upload.
+    std::vector<size_t> order(S), pos(S);
+    for (size_t i = 0; i < S; ++i) order[i] = S <= 64 ? (i + S - 1) % S : i;
+    for (size_t i = 0; i < S; ++i) pos[order[i]] = i;
+    std::vector<size_t> ready_at(S, 0);  // position in the upload order after which a slab can run
+    for (size_t k = 0; k < S; ++k) {
+        if (S <= 64) {
+            for (size_t j = 0; j < S; ++j)
+                if (slabs[k].needs >> j & 1ULL) ready_at[k] = std::max(ready_at[k], pos[j]);
+            ready_at[k] = std::max(ready_at[k], pos[k]);
+        } else {
+            ready_at[k] = (size_t)std::max(slabs[k].last_needed, (int)k);
+        }
+    }
     std::vector<char> done(S, 0);
     for (size_t upi = 0; upi < S; ++upi) {
-        const SlabPlan &u = slabs[upi];
+        const SlabPlan &u = slabs[order[upi]];
         const size_t off = (size_t)(u.row_lo * r.send_stride), n = (size_t)((u.row_hi - u.row_lo) * r.send_stride);
         if (n) ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send) + off, hs + off, n, cudaMemcpyHostToDevice, up));
         cudaEvent_t arrived = static_cast<cudaEvent_t>(r.slab_events[S + upi]);
         ISO_CUDA(cudaEventRecord(arrived, up));
         // every slab whose last needed upload this was
         for (size_t k = 0; k < S; ++k) {
-            if (done[k] || slabs[k].last_needed > (int)upi) continue;
+            if (done[k] || ready_at[k] > upi) continue;
             const SlabPlan &w = slabs[k];
             ISO_CUDA(cudaStreamWaitEvent(stream, arrived, 0));
             for (const LaunchPlan &L : r.launches) {
