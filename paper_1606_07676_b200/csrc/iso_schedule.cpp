@@ -722,7 +722,9 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
 
         // a vector class that carries next to nothing per process is not worth a launch of
         // its own: its pieces join the next narrower class that is in use
-        for (int width = 16; width > 1; width >>= 1) {
+        // (only where every width takes a launch of its own: in a launch of mixed widths a
+        // piece keeps its widest unit)
+        for (int width = 16; width > 1 && !allow_mixed; width >>= 1) {
             int64_t bytes = 0;
             for (const Piece &q : pieces)
                 if (q.kernel == KERNEL_VEC && q.width == width) bytes += q.p.len;

@@ -267,15 +267,16 @@ def test_fused_levels_interpolate_between_combining_and_direct():
 
 def test_alignment_classes_and_bulk_selection():
     # 4-byte aligned packed displacements: long blocks are split into a 16-byte aligned
-    # body (bulk kernel from 1 KB) and narrow head / tail pieces
-    w = wl.Workload("v", "alltoallv", (4, 4), wl.moore(2, 1), 0, lens=np.array([4, 1024, 16, 2048, 64, 4, 256, 1024]))
+    # body and narrow head / tail pieces; in such a ragged phase bodies from 4 KB on go to the
+    # bulk kernel, shorter ones stay with the small pieces in the launch of mixed widths
+    w = wl.Workload("v", "alltoallv", (4, 4), wl.moore(2, 1), 0, lens=np.array([4, 1024, 16, 8192, 64, 4, 256, 1024]))
     comm, req = make_request(w)
     parts = iso.Iso_request_get_parts(req)
     assert any(p["kernel"] == 1 for p in parts)
     for p in parts:
         assert p["src_off"] % p["width"] == 0 or p["kernel"] == 1
         if p["kernel"] == 1:
-            assert p["src_off"] % 16 == 0 and p["dst_off"] % 16 == 0 and p["len"] % 16 == 0 and p["len"] >= 512
+            assert p["src_off"] % 16 == 0 and p["dst_off"] % 16 == 0 and p["len"] % 16 == 0 and p["len"] >= 4096
     st = iso.Iso_request_get_stats(req)
     send = send_buffer_np(w, st["send_stride"])
     assert np.array_equal(simulate(parts, w.dims, st, send), oracle_result(w, send))
@@ -284,6 +285,42 @@ def test_alignment_classes_and_bulk_selection():
     assert iso.Iso_request_get_stats(req)["bulk_bytes"] == 0
     iso.Iso_request_free(req)
     iso.Iso_comm_free(comm)
+
+
+def test_ragged_phases_lower_to_one_launch_of_mixed_widths(monkeypatch):
+    """Irregular sizes: a phase whose pieces need several unit widths is one launch (the unit
+    descriptors carry their width); ragged ends are cut into aligned power-of-two pieces of
+    at most 4 bytes around a body of whole 16-byte units.  The exported parts still
+    reproduce the oracle, with and without that lowering."""
+    for name, phases in (("cfg5_32x32x32", 3), ("stencil_d3_m32", 3)):
+        w = wl.config(name)
+        comm, req = make_request(w)
+        st = iso.Iso_request_get_stats(req)
+        assert st["phases"] == phases and st["launches"] == phases, st
+        parts = iso.Iso_request_get_parts(req)
+        for ph in range(phases):
+            assert len({p["width"] for p in parts if p["phase"] == ph}) >= 2
+        for p in parts:
+            assert p["kernel"] == 0 and p["width"] in (1, 2, 4, 8, 16)
+            assert p["src_off"] % p["width"] == 0 and p["dst_off"] % p["width"] == 0 and p["len"] % p["width"] == 0
+        iso.Iso_request_free(req)
+        iso.Iso_comm_free(comm)
+    # a small ragged case, executed on the host, both ways
+    lens = np.array([1, 1024, 7, 33, 4, 250, 16, 2])
+    w = wl.Workload("v", "alltoallv", (4, 3, 5), wl.moore(3, 1)[:8], 0, lens=lens, seed=11)
+    for mixed in ("1", "0"):
+        monkeypatch.setenv("ISO_MIXED", mixed)
+        comm, req = make_request(w)
+        st = iso.Iso_request_get_stats(req)
+        parts = iso.Iso_request_get_parts(req)
+        send = send_buffer_np(w, st["send_stride"])
+        assert np.array_equal(simulate(parts, w.dims, st, send), oracle_result(w, send)), mixed
+        if mixed == "1":
+            assert st["launches"] == st["phases"]
+        else:
+            assert st["launches"] > st["phases"]
+        iso.Iso_request_free(req)
+        iso.Iso_comm_free(comm)
 
 
 def _mesh_expected(w, send, periodic):
