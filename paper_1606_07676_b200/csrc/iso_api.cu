@@ -506,7 +506,7 @@ cudaError_t launch_wide(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, 
     static std::vector<const void *> opted_in;  // kernels that already have the larger limit
     const void *key = reinterpret_cast<const void *>(kernel);
     if (std::find(opted_in.begin(), opted_in.end(), key) == opted_in.end()) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kVecDepth * 1024 * 16);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWideDepth * 1024 * 16);
         if (e != cudaSuccess) return e;
         opted_in.push_back(key);
     }
@@ -540,7 +540,7 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
         const int nu = count <= 3 ? count : ISO_MAX_DIMS;
 #define ISO_ROWS(W, NU, MESH, COMPACT)                                                                          \
     e = ((W == 16 || W == 0) && L.threads > 256)                                                                \
-            ? launch_wide(iso_gather_rows_wide<(W == 0 ? 0 : 16), kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent) \
+            ? launch_wide(iso_gather_rows_wide<(W == 0 ? 0 : 16), kWideDepth, NU, MESH, COMPACT>, L, a, stream, dependent) \
             : launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent)
 #define ISO_ROWS_W(W)                                                            \
     do {                                                                         \

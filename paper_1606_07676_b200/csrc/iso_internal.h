@@ -56,6 +56,7 @@ struct LoweredPart {
 enum { KERNEL_VEC = 0, KERNEL_BULK = 1 };
 constexpr int kMaxVecUnits = 4096;  // unit positions per process in one vector launch
 constexpr int kVecDepth = 8;        // cp.async ring slots per thread in the vector kernel
+constexpr int kWideDepth = 12;      // the same in CTAs of more than 256 threads (one CTA per SM)
 
 struct LaunchPlan {
     int kernel = KERNEL_VEC;

@@ -898,7 +898,10 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     L.grid = grid;
                     if (L.grid > 0x7fffffff) return ISO_ERR_DIMS;
                     L.smem = (size_t)L.n_used * (size_t)tp * sizeof(uint32_t);
-                    if (kernel == KERNEL_VEC) L.smem = width >= 4 ? (size_t)kVecDepth * L.threads * width : (width == 0 ? (size_t)kVecDepth * L.threads * 16 : 0);
+                    if (kernel == KERNEL_VEC) {
+                        const size_t depth = L.threads > 256 ? kWideDepth : kVecDepth;
+                        L.smem = width >= 4 ? depth * L.threads * width : (width == 0 ? depth * L.threads * 16 : 0);
+                    }
                     if (kernel == KERNEL_BULK)
                         L.smem = (L.smem + 15) / 16 * 16 + (size_t)L.threads * 2 * (size_t)unit + (size_t)L.threads * 2 * 8;
                     r.launches.push_back(std::move(L));
