@@ -120,6 +120,10 @@ def test_random_cases(chunk):
             iso.Iso_request_set_slabs(req, slabs)
             iso.Iso_request_set_single_launch(req, single)
             iso.Iso_request_set_bulk_threshold(req, bulk)
+            # two runs in five ask for the pipelined one-launch execution (1 or 3 slabs); it
+            # applies where the schedule allows and is ignored elsewhere
+            pipe = (0, 0, 1, 0, 3)[(c["trial"] + 2 * alg + fusion) % 5]
+            iso.Iso_request_set_pipeline(req, pipe)
             iso.Iso_request_set_algorithm(req, alg, fusion)
             if rs:
                 recv.fill_(POISON)
@@ -139,7 +143,7 @@ def test_random_cases(chunk):
                 got = recv.cpu().numpy()
             if rs:
                 assert np.array_equal(got, want), dict(chunk=chunk, trial=c["trial"], dims=c["dims"], kind=c["kind"], s=c["s"],
-                                                       alg=alg, fusion=fusion, layout=lay, single=single, bulk=bulk, host=via_host, slabs=slabs,
+                                                       alg=alg, fusion=fusion, layout=lay, single=single, bulk=bulk, host=via_host, slabs=slabs, pipeline=pipe,
                                                        periodic=c["periodic"], lens=c["lens"].tolist())
         iso.Iso_request_free(req)
         iso.Iso_comm_free(comm)
