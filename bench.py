@@ -32,9 +32,9 @@ import numpy as np
 METRIC = "neighbor-alltoall effective GB/s (device-timed) and % of B200 HBM peak, combining vs direct"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + written) per launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (iso_gather_rows on cfg2_alltoall); only valid for that kernel build
+# summarised under profiles/ (iso_gather_rows_wide on cfg2_alltoall); only valid for that kernel build
 # and workload, so it is reported for the default workload and schedule only.
-TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_alltoall": 44.89e6}
+TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_alltoall": 44.56e6}
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 512 << 20
 
@@ -480,7 +480,7 @@ def run_ours(args):
 
         # ---- roofline of the dominant kernel ------------------------------------------
         launches = max(1, st["launches"])
-        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_rows<16,8>"
+        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_rows_wide<16,12>"
         line["roofline"] = {
             "bound": "hbm", "kernel": kernel, "achieved": per_gpu, "peak": peak, "unit": "GB/s",
             "frac": per_gpu / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
