@@ -199,6 +199,18 @@ def test_pipelined_one_launch_execution(torch_cuda):
     run.close()
 
 
+def test_narrow_cta_shapes(torch_cuda, monkeypatch):
+    """16-byte and mixed-width launches run in CTAs of up to 1024 threads by default; the shapes of
+    256 and 512 threads (ISO_VEC_THREADS) stay available and must give the same bytes."""
+    for threads in ("256", "512"):
+        monkeypatch.setenv("ISO_VEC_THREADS", threads)
+        check(torch_cuda, wl.config("cfg2_alltoall"), [COMB1, COMB0, DIRECT])
+        check(torch_cuda, wl.config("cfg4"), [COMB1])
+        check(torch_cuda, wl.config("cfg5_32x32x32"), [COMB1, DIRECT])
+        check(torch_cuda, wl.config("cfg2_allgather"), [COMB1])
+        check(torch_cuda, wl.Workload("ragged", "alltoall", (37, 53), wl.moore(2, 2), 48, seed=7), [COMB1])
+
+
 def test_cfg2_allgather(torch_cuda):
     check(torch_cuda, wl.config("cfg2_allgather"), [COMB0, COMB1, COMB2, COMBD, DIRECT])
 
