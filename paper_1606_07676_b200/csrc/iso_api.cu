@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <mutex>
 #include <vector>
 
 #include "iso.h"
@@ -335,11 +336,15 @@ int materialise(Request &r)
         ISO_CUDA(cudaMallocHost((void **)&r.h_err, sizeof(int)));
         *r.h_err = 0;
     }
-    // opt in to large dynamic shared memory once per kernel
-    static bool attrs_set = false;
-    if (!attrs_set) {
-        ISO_CUDA(cudaFuncSetAttribute(iso_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attrs_set = true;
+    // opt in to large dynamic shared memory once per kernel and device
+    {
+        static std::vector<int> devices_set;
+        static std::mutex guard;
+        std::lock_guard<std::mutex> lock(guard);
+        if (std::find(devices_set.begin(), devices_set.end(), device) == devices_set.end()) {
+            ISO_CUDA(cudaFuncSetAttribute(iso_gather_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+            devices_set.push_back(device);
+        }
     }
     r.dirty = false;
     return ISO_SUCCESS;
@@ -503,12 +508,20 @@ cudaError_t launch_kernel(Kernel kernel, const LaunchPlan &L, const LaunchDev &a
 template <typename Kernel>
 cudaError_t launch_wide(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, cudaStream_t stream, bool dependent)
 {
-    static std::vector<const void *> opted_in;  // kernels that already have the larger limit
-    const void *key = reinterpret_cast<const void *>(kernel);
-    if (std::find(opted_in.begin(), opted_in.end(), key) == opted_in.end()) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWideDepth * 1024 * 16);
-        if (e != cudaSuccess) return e;
-        opted_in.push_back(key);
+    // (device, kernel) pairs that already have the larger limit: the attribute is per device
+    static std::vector<std::pair<int, const void *>> opted_in;
+    static std::mutex guard;
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return e;
+    const std::pair<int, const void *> key(device, reinterpret_cast<const void *>(kernel));
+    {
+        std::lock_guard<std::mutex> lock(guard);
+        if (std::find(opted_in.begin(), opted_in.end(), key) == opted_in.end()) {
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWideDepth * 1024 * 16);
+            if (e != cudaSuccess) return e;
+            opted_in.push_back(key);
+        }
     }
     return launch_kernel(kernel, L, a, stream, dependent);
 }
