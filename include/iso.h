@@ -221,9 +221,8 @@ int Iso_request_set_layout(Iso_request request, int layout);
  * saves the ramp-up and drain of one kernel per phase.  The barrier wait is bounded; if it
  * expires the kernel stops and Iso_wait returns ISO_ERR_TIMEOUT.  enable = 0 goes back to
  * one launch per phase, which is the default: with programmatic dependent launches between
- * the phases the per-phase kernels were faster for schedules of two or three phases
- * (40.8 against 48.5 microseconds on the 32^3 torus), the single launch only from about
- * five phases on (285 against 302 microseconds on the 8^5 torus).  Iso_request_get_stats
+ * the phases the per-phase kernels are faster (36.1 against 44.9 microseconds on the 32^3
+ * torus, 161 against 197 microseconds on the 8^5 torus with five phases).  Iso_request_get_stats
  * reports launches = 1 once the request has been started in this mode.
  */
 int Iso_request_set_single_launch(Iso_request request, int enable);

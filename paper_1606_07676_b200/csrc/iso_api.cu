@@ -200,7 +200,7 @@ int materialise(Request &r)
         if (rc0 != ISO_SUCCESS) return rc0;
         bool ok = !r.launches.empty();
         for (const LaunchPlan &L : r.launches) {
-            if (L.kernel != KERNEL_VEC || L.width != 16 || L.threads > 256) ok = false;
+            if (L.kernel != KERNEL_VEC || L.width != 16 || L.threads > 1024) ok = false;
             for (int k = 0; k < L.n_used; ++k)
                 if (!c.periodic[L.used_dim[k]]) ok = false;
         }
@@ -235,7 +235,7 @@ int materialise(Request &r)
     // one-launch execution: every launch is a 16-byte vector launch on periodic dimensions
     bool single = r.persistent && !r.wave_ok && r.launches.size() >= 2;
     for (const LaunchPlan &L : r.launches) {
-        if (L.kernel != KERNEL_VEC || L.width != 16 || L.threads > 256) single = false;
+        if (L.kernel != KERNEL_VEC || L.width != 16 || L.threads > 1024) single = false;
         for (int k = 0; k < L.n_used; ++k)
             if (!c.periodic[L.used_dim[k]]) single = false;
     }
@@ -309,10 +309,10 @@ int materialise(Request &r)
     }
     if (single) {
         // the grid must be resident as a whole: ask how many CTAs fit
-        const size_t smem = (sizeof(LaunchDev) + 127) / 128 * 128 + (size_t)kVecDepth * 256 * 16;
-        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows_multi<kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        const size_t smem = (sizeof(LaunchDev) + 127) / 128 * 128 + (size_t)kWideDepth * 1024 * 16;
+        ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows_multi<kWideDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         int per_sm = 0;
-        ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_multi<kVecDepth>, 256, smem));
+        ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_multi<kWideDepth>, 1024, smem));
         int want = 4;
         if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
             int v = std::atoi(env);
@@ -408,10 +408,10 @@ int build_wave(Request &r, unsigned char *blob, size_t launches_off, size_t item
     const Comm &c = *r.comm;
     const size_t nl = r.launches.size();
     const size_t n = n_slabs * nl;
-    const size_t smem = (sizeof(LaunchDev) + 127) / 128 * 128 + (size_t)kVecDepth * 256 * 16;
-    ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows_wave<kVecDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const size_t smem = (sizeof(LaunchDev) + 127) / 128 * 128 + (size_t)kWideDepth * 1024 * 16;
+    ISO_CUDA(cudaFuncSetAttribute(iso_gather_rows_wave<kWideDepth>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
-    ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_wave<kVecDepth>, 256, smem));
+    ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_wave<kWideDepth>, 1024, smem));
     int want = 4;
     if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
         int v = std::atoi(env);
@@ -1203,7 +1203,7 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         m.err = r.d_err;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)r.wave_grid);
-        cfg.blockDim = dim3(256);
+        cfg.blockDim = dim3(1024);
         cfg.dynamicSmemBytes = r.wave_smem;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
@@ -1211,7 +1211,7 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         attr[0].val.cooperative = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        ISO_CUDA(cudaLaunchKernelEx(&cfg, iso_gather_rows_wave<kVecDepth>, m));
+        ISO_CUDA(cudaLaunchKernelEx(&cfg, iso_gather_rows_wave<kWideDepth>, m));
         r.last_stream = cuda_stream;
         r.started = true;
         return ISO_SUCCESS;
@@ -1227,7 +1227,7 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         r.epoch += (unsigned long long)(m.n - 1) * (unsigned long long)r.multi_grid;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)r.multi_grid);
-        cfg.blockDim = dim3(256);
+        cfg.blockDim = dim3(1024);
         cfg.dynamicSmemBytes = r.multi_smem;
         cfg.stream = stream;
         cudaLaunchAttribute attr[1];
@@ -1235,7 +1235,7 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         attr[0].val.cooperative = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        ISO_CUDA(cudaLaunchKernelEx(&cfg, iso_gather_rows_multi<kVecDepth>, m));
+        ISO_CUDA(cudaLaunchKernelEx(&cfg, iso_gather_rows_multi<kWideDepth>, m));
         r.last_stream = cuda_stream;
         r.started = true;
         return ISO_SUCCESS;

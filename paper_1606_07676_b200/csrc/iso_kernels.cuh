@@ -431,7 +431,7 @@ __device__ __forceinline__ bool grid_barrier(const MultiDev &M, unsigned long lo
 }
 
 template <int DEPTH>
-__global__ void __launch_bounds__(256, 4) iso_gather_rows_multi(const __grid_constant__ MultiDev M)
+__global__ void __launch_bounds__(1024, 1) iso_gather_rows_multi(const __grid_constant__ MultiDev M)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ int s_ok;
@@ -478,7 +478,7 @@ struct WaveDev {
 };
 
 template <int DEPTH>
-__global__ void __launch_bounds__(256, 4) iso_gather_rows_wave(const __grid_constant__ WaveDev M)
+__global__ void __launch_bounds__(1024, 1) iso_gather_rows_wave(const __grid_constant__ WaveDev M)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ int s_ok;

@@ -870,7 +870,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         // (measured against four CTAs of 256 threads: 36.1 against 40.3 microseconds
                         // per all-to-all on the 32^3 torus, 161 against 184 on the 8^5 torus);
                         // ISO_VEC_THREADS=256 or 512 selects the narrower shapes
-                        uint32_t max_threads = ((width == 16 || width == 0) && r.wave_request == 0 && !r.persistent) ? 1024 : 256;
+                        uint32_t max_threads = (width == 16 || width == 0) ? 1024 : 256;
                         if (const char *env = std::getenv("ISO_VEC_THREADS")) {
                             const int v = std::atoi(env);
                             if ((v == 256 || v == 512) && max_threads == 1024) max_threads = units > 256 ? 1024 : (uint32_t)v;
