@@ -312,13 +312,14 @@ int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes);
 /*
  * Non-periodic dimensions (the extension Section VII mentions).  periodic[j] = 0 makes
  * dimension j a mesh: a block whose source R - C^i falls outside the mesh is not delivered
- * and the receive slot keeps its previous contents.  Supported by ISO_ALG_DIRECT (all
- * collectives) and by ISO_ALG_COMBINING for the all-to-all collectives: every hop of a block
- * is skipped for the processes on whose route the original sender or the final receiver
- * would lie outside (always with the packed layout: the receive buffer cannot double as
- * scratch when undelivered slots must keep their contents).  Allgather requests on a mesh
- * start with the direct schedule.  Call it
- * before creating requests.  Default: all dimensions periodic.
+ * and the receive slot keeps its previous contents.  Supported by ISO_ALG_DIRECT and by
+ * ISO_ALG_COMBINING for all collectives.  All-to-all: every hop of a block is skipped for
+ * the processes on whose route the original sender or the final receiver would lie outside
+ * (always with the packed layout: the receive buffer cannot double as scratch when
+ * undelivered slots must keep their contents).  Allgather: a trie node is produced only at
+ * the processes whose source for that prefix exists.  ISO_ALG_TORUS (Algorithm 1 as
+ * printed, whose blocks alternate through their receive slots) is refused with ISO_ERR_ARG.
+ * Call it before creating requests.  Default: all dimensions periodic.
  */
 int Iso_comm_set_periodic(Iso_comm isocomm, const int periodic[]);
 
@@ -349,8 +350,47 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
                    void *cuda_stream);
 
 /* Local completion (Section VII): blocks until the last start has finished and returns
- * ISO_ERR_TIMEOUT if a kernel gave up a bounded wait, ISO_ERR_CUDA on a CUDA error. */
+ * ISO_ERR_TIMEOUT if a kernel gave up a bounded wait, ISO_ERR_CUDA on a CUDA error.
+ * After ISO_ERR_TIMEOUT the receive buffers are incomplete, the request's arrival counters
+ * have been cleared and the request can be started again. */
 int Iso_wait(Iso_request request);
+
+/*
+ * Race detection aid (no counterpart in the paper).  The library's intermediate buffer is
+ * allocated with a guard band of 4096 bytes of a fixed pattern on either side; a schedule
+ * never writes there.  This call waits for the request's work in flight, reads both bands
+ * back and stores the number of bytes that no longer hold the pattern in `*violations`
+ * (0 when the request has no intermediate buffer yet).  Meant for tests, together with
+ * bands the caller puts around its own send and receive buffers.
+ */
+int Iso_request_check_guards(Iso_request request, int64_t *violations);
+
+/*
+ * Bound of the device-side waits (no counterpart in the paper, whose processes block in
+ * MPI_Sendrecv).  The one-launch execution modes (Iso_request_set_single_launch,
+ * Iso_request_set_pipeline) make thread blocks wait for each other; every such wait polls
+ * at most `polls` times (about 40 ns apart) and then gives up: the kernel returns by itself
+ * and Iso_wait reports ISO_ERR_TIMEOUT.  Default 2^22 (a fraction of a second).  polls >= 1.
+ */
+int Iso_request_set_wait_limit(Iso_request request, unsigned int polls);
+
+/*
+ * Testing aid for the time-out path.  The NEXT start of a one-launch execution mode waits
+ * for `extra` more arrivals than there are thread blocks, so its first wait cannot be
+ * satisfied and runs into the limit set with Iso_request_set_wait_limit; nothing faults
+ * and nothing waits without bound.  One shot: later starts are normal.  0 <= extra <= 1024.
+ * Has no effect on the default execution (one launch per phase), which has no such waits.
+ */
+int Iso_request_test_skew_arrivals(Iso_request request, int extra);
+
+/*
+ * Launch-latency floor (measurement aid, no counterpart in the paper): enqueues `launches`
+ * launches of an empty kernel back to back on `cuda_stream`, as programmatic dependent
+ * launches when `dependent` != 0 (the way Iso_Start chains its phases), times them with
+ * events and stores the device time per launch in microseconds.  Blocks until done.
+ * A phase of a schedule cannot be shorter than this.
+ */
+int Iso_measure_launch_floor(void *cuda_stream, int launches, int dependent, float *microseconds_per_launch);
 
 /* Statistics of the current schedule.  Host only; valid before the first start. */
 int Iso_request_get_stats(Iso_request request, Iso_stats *out);
@@ -383,8 +423,11 @@ int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int 
  *  - P * (intermediate bytes per process) + the unit tables must fit the scratch array,
  *    else ISO_ERR_TOO_LARGE and nothing is enqueued;
  *  - the first call on a device looks up the device address of the scratch array
- *    (cudaGetSymbolAddress, with that device current); make that first call outside any
- *    stream capture;
+ *    (cudaGetSymbolAddress, with that device current);
+ *  - NO call of this function, first or later, may be made while `cuda_stream` is being
+ *    captured into a graph: every call copies freshly built tables from host memory that
+ *    is released when the call returns, so a captured copy node would read freed memory
+ *    at every replay;
  *  - all calls on one device share the scratch array and it keeps the previous call's
  *    contents; nothing in it has to start at zero, because every byte a kernel reads from
  *    it was written earlier in the same call (tables by the copy, intermediate places by

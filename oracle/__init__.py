@@ -55,6 +55,14 @@ def _declare(lib: ctypes.CDLL) -> ctypes.CDLL:
         f.argtypes = [ci, vp, ci, vp, i64, vp, vp, i64, i64]
     lib.iso_oracle_alltoallv.restype = ci
     lib.iso_oracle_alltoallv.argtypes = [ci, vp, ci, vp, vp, vp, vp, i64, i64, vp, vp, i64, i64]
+    lib.iso_oracle_source_rank_mesh.restype = i64
+    lib.iso_oracle_source_rank_mesh.argtypes = [ci, vp, vp, i64, vp]
+    for name in ("iso_oracle_alltoall_mesh", "iso_oracle_allgather_mesh"):
+        f = getattr(lib, name)
+        f.restype = ci
+        f.argtypes = [ci, vp, vp, ci, vp, i64, vp, vp, i64, i64]
+    lib.iso_oracle_alltoallv_mesh.restype = ci
+    lib.iso_oracle_alltoallv_mesh.argtypes = [ci, vp, vp, ci, vp, vp, vp, vp, i64, i64, vp, vp, i64, i64]
     return lib
 
 
@@ -100,9 +108,30 @@ def target_rank(dims, r: int, C, lib=None) -> int:
     return int(lib.iso_oracle_target_rank(dims.size, _ptr(dims), int(r), _ptr(C)))
 
 
+def source_rank_mesh(dims, periodic, r: int, C, lib=None) -> int:
+    """rank(R - C) on a torus whose dimensions with periodic[j] == 0 do not wrap; -1 when
+    that process does not exist (Section VII)."""
+    lib = lib or load()
+    dims, periodic, C = _ints(dims), _ints(periodic), _ints(C)
+    return int(lib.iso_oracle_source_rank_mesh(dims.size, _ptr(dims), _ptr(periodic), int(r), _ptr(C)))
+
+
+def _mesh_flags(periodic, d):
+    """None when every dimension wraps (the plain functions apply), else the flags."""
+    if periodic is None:
+        return None
+    flags = _ints(periodic)
+    if flags.size != d:
+        raise ValueError("periodic must hold d flags")
+    return None if bool(flags.all()) else flags
+
+
 def alltoall(dims, offsets, m: int, send: np.ndarray, r0: int = 0, r1: int | None = None,
-             lib=None) -> np.ndarray:
-    """Receive buffers (uint8, shape [r1-r0, s*m]) of a regular all-to-all."""
+             lib=None, periodic=None, fill: int = 0) -> np.ndarray:
+    """Receive buffers (uint8, shape [r1-r0, s*m]) of a regular all-to-all.
+
+    With non-periodic dimensions (`periodic`), slots whose source lies outside the mesh
+    keep the value ``fill``."""
     lib = lib or load()
     dims, d, offs, s = _geometry(dims, offsets)
     P = int(np.prod(dims, dtype=np.int64))
@@ -110,6 +139,13 @@ def alltoall(dims, offsets, m: int, send: np.ndarray, r0: int = 0, r1: int | Non
     sb = _bytes_view(send)
     if sb.size != P * s * m:
         raise ValueError("send buffer must hold P*s*m bytes")
+    flags = _mesh_flags(periodic, d)
+    if flags is not None:
+        out = np.full((r1 - r0, s * m), fill, dtype=np.uint8)
+        rc = lib.iso_oracle_alltoall_mesh(d, _ptr(dims), _ptr(flags), s, _ptr(offs), m, _ptr(sb), _ptr(out), r0, r1)
+        if rc:
+            raise ValueError("oracle rejected the arguments")
+        return out
     out = np.empty((r1 - r0, s * m), dtype=np.uint8)
     rc = lib.iso_oracle_alltoall(d, _ptr(dims), s, _ptr(offs), m, _ptr(sb), _ptr(out), r0, r1)
     if rc:
@@ -118,8 +154,9 @@ def alltoall(dims, offsets, m: int, send: np.ndarray, r0: int = 0, r1: int | Non
 
 
 def allgather(dims, offsets, m: int, send: np.ndarray, r0: int = 0, r1: int | None = None,
-              lib=None) -> np.ndarray:
-    """Receive buffers (uint8, shape [r1-r0, s*m]) of an allgather."""
+              lib=None, periodic=None, fill: int = 0) -> np.ndarray:
+    """Receive buffers (uint8, shape [r1-r0, s*m]) of an allgather (`periodic`, `fill`: as
+    for `alltoall`)."""
     lib = lib or load()
     dims, d, offs, s = _geometry(dims, offsets)
     P = int(np.prod(dims, dtype=np.int64))
@@ -127,6 +164,13 @@ def allgather(dims, offsets, m: int, send: np.ndarray, r0: int = 0, r1: int | No
     sb = _bytes_view(send)
     if sb.size != P * m:
         raise ValueError("send buffer must hold P*m bytes")
+    flags = _mesh_flags(periodic, d)
+    if flags is not None:
+        out = np.full((r1 - r0, s * m), fill, dtype=np.uint8)
+        rc = lib.iso_oracle_allgather_mesh(d, _ptr(dims), _ptr(flags), s, _ptr(offs), m, _ptr(sb), _ptr(out), r0, r1)
+        if rc:
+            raise ValueError("oracle rejected the arguments")
+        return out
     out = np.empty((r1 - r0, s * m), dtype=np.uint8)
     rc = lib.iso_oracle_allgather(d, _ptr(dims), s, _ptr(offs), m, _ptr(sb), _ptr(out), r0, r1)
     if rc:
@@ -136,7 +180,7 @@ def allgather(dims, offsets, m: int, send: np.ndarray, r0: int = 0, r1: int | No
 
 def alltoallv(dims, offsets, lens, sdispls, rdispls, send_stride: int, recv_stride: int,
               send: np.ndarray, r0: int = 0, r1: int | None = None, fill: int = 0,
-              lib=None) -> np.ndarray:
+              lib=None, periodic=None) -> np.ndarray:
     """Receive buffers (uint8, shape [r1-r0, recv_stride]) of an irregular all-to-all.
 
     Bytes of the receive buffer that no block covers keep the value ``fill``.
@@ -154,6 +198,13 @@ def alltoallv(dims, offsets, lens, sdispls, rdispls, send_stride: int, recv_stri
     if sb.size != P * send_stride:
         raise ValueError("send buffer must hold P*send_stride bytes")
     out = np.full((r1 - r0, recv_stride), fill, dtype=np.uint8)
+    flags = _mesh_flags(periodic, d)
+    if flags is not None:
+        rc = lib.iso_oracle_alltoallv_mesh(d, _ptr(dims), _ptr(flags), s, _ptr(offs), _ptr(lens), _ptr(sdispls),
+                                           _ptr(rdispls), send_stride, recv_stride, _ptr(sb), _ptr(out), r0, r1)
+        if rc:
+            raise ValueError("oracle rejected the arguments")
+        return out
     rc = lib.iso_oracle_alltoallv(d, _ptr(dims), s, _ptr(offs), _ptr(lens), _ptr(sdispls),
                                   _ptr(rdispls), send_stride, recv_stride, _ptr(sb), _ptr(out),
                                   r0, r1)

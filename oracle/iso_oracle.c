@@ -150,3 +150,107 @@ int iso_oracle_alltoallv(int d, const int *dims, int s, const int *offsets,
     }
     return 0;
 }
+
+/* ---- non-periodic (mesh) dimensions ------------------------------------------------
+ *
+ * Section VII of the paper mentions the extension to tori in which some dimensions do
+ * not wrap around.  Reading used here: along a dimension j with periodic[j] == 0 the
+ * coordinates are not reduced; process R receives block i only if its source R - C^i
+ * exists, i.e. 0 <= r_j - c_j < p_j in every such dimension.  Otherwise nothing is
+ * delivered and the receive slot keeps whatever it held before the call.  Periodic
+ * dimensions wrap as above.
+ *
+ * Returns the source rank, or -1 when the source lies outside the mesh. */
+int64_t iso_oracle_source_rank_mesh(int d, const int *dims, const int *periodic, int64_t r, const int *C)
+{
+    int64_t coord[ISO_ORACLE_MAX_DIMS];
+    int64_t rest = r;
+    int j;
+    for (j = d - 1; j >= 0; j--) {
+        coord[j] = rest % dims[j];
+        rest = rest / dims[j];
+    }
+    for (j = 0; j < d; j++) {
+        int64_t p = dims[j];
+        int64_t y = coord[j] - (int64_t)C[j];
+        if (periodic[j]) {
+            y = y % p;
+            if (y < 0)
+                y += p;
+        } else if (y < 0 || y >= p) {
+            return -1;
+        }
+        coord[j] = y;
+    }
+    rest = 0;
+    for (j = 0; j < d; j++)
+        rest = rest * dims[j] + coord[j];
+    return rest;
+}
+
+/* All-to-all on a mesh: recv[r][i] = send[R - C^i][i] where that process exists;
+ * other slots of `recv` are left as they are. */
+int iso_oracle_alltoall_mesh(int d, const int *dims, const int *periodic, int s, const int *offsets,
+                             int64_t m, const unsigned char *send, unsigned char *recv,
+                             int64_t r0, int64_t r1)
+{
+    int64_t r;
+    int i;
+    if (!args_ok(d, dims, s, r0, r1) || m < 0 || periodic == 0)
+        return -1;
+    for (r = r0; r < r1; r++) {
+        for (i = 0; i < s; i++) {
+            int64_t q = iso_oracle_source_rank_mesh(d, dims, periodic, r, offsets + (int64_t)i * d);
+            if (q < 0)
+                continue;
+            memcpy(recv + ((r - r0) * s + i) * m, send + (q * s + i) * m, (size_t)m);
+        }
+    }
+    return 0;
+}
+
+/* Allgather on a mesh: recv[r][i] = send[R - C^i] where that process exists. */
+int iso_oracle_allgather_mesh(int d, const int *dims, const int *periodic, int s, const int *offsets,
+                              int64_t m, const unsigned char *send, unsigned char *recv,
+                              int64_t r0, int64_t r1)
+{
+    int64_t r;
+    int i;
+    if (!args_ok(d, dims, s, r0, r1) || m < 0 || periodic == 0)
+        return -1;
+    for (r = r0; r < r1; r++) {
+        for (i = 0; i < s; i++) {
+            int64_t q = iso_oracle_source_rank_mesh(d, dims, periodic, r, offsets + (int64_t)i * d);
+            if (q < 0)
+                continue;
+            memcpy(recv + ((r - r0) * s + i) * m, send + q * m, (size_t)m);
+        }
+    }
+    return 0;
+}
+
+/* Irregular all-to-all on a mesh. */
+int iso_oracle_alltoallv_mesh(int d, const int *dims, const int *periodic, int s, const int *offsets,
+                              const int64_t *len, const int64_t *sdispl, const int64_t *rdispl,
+                              int64_t send_stride, int64_t recv_stride,
+                              const unsigned char *send, unsigned char *recv,
+                              int64_t r0, int64_t r1)
+{
+    int64_t r;
+    int i;
+    if (!args_ok(d, dims, s, r0, r1) || periodic == 0)
+        return -1;
+    for (i = 0; i < s; i++)
+        if (len[i] < 0 || sdispl[i] < 0 || rdispl[i] < 0)
+            return -1;
+    for (r = r0; r < r1; r++) {
+        for (i = 0; i < s; i++) {
+            int64_t q = iso_oracle_source_rank_mesh(d, dims, periodic, r, offsets + (int64_t)i * d);
+            if (q < 0)
+                continue;
+            memcpy(recv + (r - r0) * recv_stride + rdispl[i],
+                   send + q * send_stride + sdispl[i], (size_t)len[i]);
+        }
+    }
+    return 0;
+}

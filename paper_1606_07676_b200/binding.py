@@ -31,6 +31,7 @@ EXPORTS = (
     "Iso_neighborhood_create", "Iso_comm_free", "Iso_comm_set_periodic",
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
     "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_pipeline", "Iso_request_set_chains", "Iso_request_set_graph", "Iso_request_tune", "Iso_request_get_execution", "Iso_request_set_bulk_threshold",
+    "Iso_request_check_guards", "Iso_request_set_wait_limit", "Iso_request_test_skew_arrivals", "Iso_measure_launch_floor",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
     "Iso_neighbor_alltoall_static", "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
@@ -100,6 +101,10 @@ def load_library() -> ctypes.CDLL:
         "Iso_request_tune": [vp, vp, ci],
         "Iso_request_get_execution": [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)],
         "Iso_request_set_bulk_threshold": [vp, i64],
+        "Iso_request_check_guards": [vp, ctypes.POINTER(i64)],
+        "Iso_request_set_wait_limit": [vp, ctypes.c_uint],
+        "Iso_request_test_skew_arrivals": [vp, ci],
+        "Iso_measure_launch_floor": [vp, ci, ci, ctypes.POINTER(ctypes.c_float)],
         "Iso_Start": [vp, vp],
         "Iso_Start_host": [vp, vp, vp, vp],
         "Iso_wait": [vp],
@@ -275,6 +280,29 @@ def Iso_request_get_execution(request: int) -> dict:
 
 def Iso_request_set_bulk_threshold(request: int, nbytes: int) -> None:
     _check(load_library().Iso_request_set_bulk_threshold(request, nbytes), "Iso_request_set_bulk_threshold")
+
+
+def Iso_request_check_guards(request: int) -> int:
+    """Bytes of the guard bands around the intermediate buffer that were overwritten."""
+    bad = ctypes.c_int64(-1)
+    _check(load_library().Iso_request_check_guards(request, ctypes.byref(bad)), "Iso_request_check_guards")
+    return int(bad.value)
+
+
+def Iso_request_set_wait_limit(request: int, polls: int) -> None:
+    _check(load_library().Iso_request_set_wait_limit(request, polls), "Iso_request_set_wait_limit")
+
+
+def Iso_request_test_skew_arrivals(request: int, extra: int) -> None:
+    _check(load_library().Iso_request_test_skew_arrivals(request, extra), "Iso_request_test_skew_arrivals")
+
+
+def Iso_measure_launch_floor(stream=None, launches: int = 1000, dependent: bool = True) -> float:
+    """Device time per launch of an empty kernel, in microseconds."""
+    us = ctypes.c_float(0.0)
+    _check(load_library().Iso_measure_launch_floor(_stream(stream), launches, 1 if dependent else 0,
+                                                   ctypes.byref(us)), "Iso_measure_launch_floor")
+    return float(us.value)
 
 
 def Iso_Start(request: int, stream=None) -> None:

@@ -41,7 +41,8 @@ void release_device(Request &r)
     if (r.graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.graph_exec));
     r.graph_exec = nullptr;
     if (r.d_blob) cudaFree(r.d_blob);
-    if (r.d_inter) cudaFree(r.d_inter);
+    if (r.d_inter_alloc) cudaFree(r.d_inter_alloc);
+    r.d_inter_alloc = nullptr;
     if (r.d_err) cudaFree(r.d_err);
     if (r.copy_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.copy_stream));
     if (r.up_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.up_stream));
@@ -124,8 +125,7 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
     r->comm = comm;
     comm->refcount++;
     r->kind = kind;
-    for (int j = 0; j < comm->d; ++j)
-        if (!comm->periodic[j] && kind == ISO_KIND_ALLGATHER) r->alg = ISO_ALG_DIRECT;  // mesh allgather: direct only
+    r->knobs = read_knobs();
     r->send = static_cast<const unsigned char *>(sendbuf);
     r->recv = static_cast<unsigned char *>(recvbuf);
     r->s = comm->s;
@@ -136,6 +136,11 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
 }
 
 int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
+
+// Guard bands around the library's intermediate buffer (a multiple of 256 bytes, so that the
+// buffer keeps the allocation's alignment).
+constexpr size_t kGuardBytes = 4096;
+constexpr int kGuardPattern = 0xC3;
 
 LaunchDev make_launch_args(const Request &r, const LaunchPlan &L);
 void choose_slab_plan(Request &r);
@@ -189,6 +194,15 @@ int materialise(Request &r)
     // a captured graph holds the addresses of the tables and buffers that are replaced below
     if (r.graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.graph_exec));
     r.graph_exec = nullptr;
+    // grids are sized for the device that runs them (the host-only lowering at init assumed a B200)
+    int device = 0, sms = 0;
+    ISO_CUDA(cudaGetDevice(&device));
+    ISO_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    if (sms > 0 && sms != r.sm_count) {
+        r.sm_count = sms;
+        int rc0 = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
+        if (rc0 != ISO_SUCCESS) return rc0;
+    }
     // pipelined one-launch execution: every launch must be a 16-byte vector launch of at most
     // 256 threads on periodic dimensions.  Decided on a trial lowering (device allocations
     // are 256-byte aligned) because the size of the intermediate buffer depends on it.
@@ -209,17 +223,20 @@ int materialise(Request &r)
     choose_slab_plan(r);
     // device tables depend on the alignment of the intermediate buffer: allocate it first
     const int64_t inter_bytes = r.inter_rows * r.inter_stride;
-    if (inter_bytes > r.d_inter_bytes) {
-        if (r.d_inter) cudaFree(r.d_inter);
-        r.d_inter = nullptr;
+    if (inter_bytes != r.d_inter_bytes) {  // exactly sized, so that the trailing band sits right behind it
+        if (r.d_inter_alloc) cudaFree(r.d_inter_alloc);
+        r.d_inter = r.d_inter_alloc = nullptr;
         r.d_inter_bytes = 0;
-        ISO_CUDA(cudaMalloc((void **)&r.d_inter, (size_t)inter_bytes));
+        // a guard band of a fixed pattern on either side: no schedule may ever write there
+        // (Iso_request_check_guards)
+        if (inter_bytes > 0) {
+        ISO_CUDA(cudaMalloc((void **)&r.d_inter_alloc, (size_t)inter_bytes + 2 * kGuardBytes));
+        r.d_inter = r.d_inter_alloc + kGuardBytes;
         r.d_inter_bytes = inter_bytes;
+        ISO_CUDA(cudaMemset(r.d_inter_alloc, kGuardPattern, kGuardBytes));
+        ISO_CUDA(cudaMemset(r.d_inter + inter_bytes, kGuardPattern, kGuardBytes));
+        }
     }
-    int device = 0, sms = 0;
-    ISO_CUDA(cudaGetDevice(&device));
-    ISO_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    r.sm_count = sms > 0 ? sms : r.sm_count;
     int rc = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
     if (rc != ISO_SUCCESS) return rc;
 
@@ -314,10 +331,7 @@ int materialise(Request &r)
         int per_sm = 0;
         ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_multi<kWideDepth>, 1024, smem));
         int want = 4;
-        if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
-            int v = std::atoi(env);
-            if (v >= 1 && v <= 8) want = v;
-        }
+        if (r.knobs.vec_ctas_per_sm >= 1 && r.knobs.vec_ctas_per_sm <= 8) want = r.knobs.vec_ctas_per_sm;
         per_sm = std::min(per_sm, want);
         if (per_sm >= 1) {
             r.multi_grid = per_sm * r.sm_count;
@@ -413,10 +427,7 @@ int build_wave(Request &r, unsigned char *blob, size_t launches_off, size_t item
     int per_sm = 0;
     ISO_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iso_gather_rows_wave<kWideDepth>, 1024, smem));
     int want = 4;
-    if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
-        int v = std::atoi(env);
-        if (v >= 1 && v <= 8) want = v;
-    }
+    if (r.knobs.vec_ctas_per_sm >= 1 && r.knobs.vec_ctas_per_sm <= 8) want = r.knobs.vec_ctas_per_sm;
     per_sm = std::min(per_sm, want);
     if (per_sm < 1) return ISO_SUCCESS;  // cannot be resident: Iso_Start falls back to one launch per phase
     const int grid = per_sm * r.sm_count;
@@ -609,8 +620,8 @@ void plan_slabs(const Request &r, std::vector<SlabPlan> &slabs, int want = 0)
     int n = std::min(p0, 8);
     if (want > 0) {
         n = std::min(p0, want);
-    } else if (const char *env = std::getenv("ISO_HOST_SLABS")) {
-        int v = std::atoi(env);
+    } else if (r.knobs.host_slabs >= 0) {
+        const int v = r.knobs.host_slabs;
         if (v <= 1) return;
         n = std::min(p0, v);
     }
@@ -654,7 +665,7 @@ void choose_slab_plan(Request &r)
     r.inter_rows = c.P;
     r.chains = 1;
     r.use_graph = !r.persistent && r.graph_request;
-    if (const char *env = std::getenv("ISO_GRAPH")) r.use_graph = !r.persistent && std::atoi(env) != 0;
+    if (r.knobs.graph >= 0) r.use_graph = !r.persistent && r.knobs.graph != 0;
     if (r.wave_ok) {
         // pipelined one-launch execution: its own slabs; from three slabs on the
         // intermediate buffer holds two of them
@@ -674,7 +685,7 @@ void choose_slab_plan(Request &r)
     }
     if (r.persistent || r.inter_stride == 0) return;
     int want = r.slab_request;
-    if (const char *env = std::getenv("ISO_SLABS")) want = std::atoi(env);
+    if (r.knobs.slabs >= 0) want = r.knobs.slabs;
     if (want == 0) {
         // automatic: all-to-all schedules made of vector launches only; a slab's launch should
         // still last about 12 microseconds and give every CTA a dozen rows
@@ -690,7 +701,7 @@ void choose_slab_plan(Request &r)
         while (want * 2 <= per && want * 2 <= 64 && c.P / (want * 2) >= 12 * rows_per_pass) want *= 2;
     }
     int chains = std::max(1, r.chains_request);
-    if (const char *env = std::getenv("ISO_CHAINS")) chains = std::max(1, std::min(8, std::atoi(env)));
+    if (r.knobs.chains >= 0) chains = std::max(1, std::min(8, r.knobs.chains));
     if (chains > 1) want = std::max(want, chains) / chains * chains;
     if (want < 2) return;
     std::vector<SlabPlan> slabs;
@@ -1082,7 +1093,7 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int cold)
             return cuda_fail(cudaGetLastError());
         }
     }
-    static const bool log = std::getenv("ISO_TUNE_LOG") != nullptr;
+    const bool log = r.knobs.tune_log;
     struct Choice { int slabs, chains, graph; };
     const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0};
     Choice best = before;
@@ -1190,7 +1201,7 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         if (rc != ISO_SUCCESS) return rc;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    static const bool use_pdl = !(std::getenv("ISO_NO_PDL") && std::atoi(std::getenv("ISO_NO_PDL")) != 0);
+    const bool use_pdl = !r.knobs.no_pdl;
     if (r.wave_grid > 0) {
         // one cooperative launch that works through the (slab, launch) items
         WaveDev m{};
@@ -1199,8 +1210,10 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         m.n = r.wave_items;
         m.done = r.d_counter;
         r.wave_run += 1;
-        m.target = r.wave_run * (unsigned long long)r.wave_grid;
+        m.target = r.wave_run * (unsigned long long)r.wave_grid + (unsigned long long)r.skew_next;
+        r.skew_next = 0;
         m.err = r.d_err;
+        m.max_polls = r.wait_limit;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)r.wave_grid);
         cfg.blockDim = dim3(1024);
@@ -1224,6 +1237,9 @@ int Iso_Start(Iso_request request, void *cuda_stream)
         m.counter = r.d_counter;
         m.epoch = r.epoch;
         m.err = r.d_err;
+        m.max_polls = r.wait_limit;
+        m.arrivals = (uint32_t)(r.multi_grid + r.skew_next);
+        r.skew_next = 0;
         r.epoch += (unsigned long long)(m.n - 1) * (unsigned long long)r.multi_grid;
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)r.multi_grid);
@@ -1329,7 +1345,7 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
     ISO_CUDA(cudaEventRecord(fence, stream));
     ISO_CUDA(cudaStreamWaitEvent(up, fence, 0));
     ISO_CUDA(cudaStreamWaitEvent(down, fence, 0));
-    static const bool use_pdl = !(std::getenv("ISO_NO_PDL") && std::atoi(std::getenv("ISO_NO_PDL")) != 0);
+    const bool use_pdl = !r.knobs.no_pdl;
     // Upload order: the last slab first, then 0, 1, ...: on a torus slab 0 reads the last slab,
     // so in natural order it (and its download) would have to wait for the very last upload.
     std::vector<size_t> order(S), pos(S);
@@ -1380,6 +1396,7 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
 
 int Iso_wait(Iso_request request)
 {
+    return guarded([&]() -> int {
     if (check_handle(request)) return ISO_ERR_ARG;
     Request &r = *request;
     if (!r.started) return ISO_SUCCESS;
@@ -1390,16 +1407,88 @@ int Iso_wait(Iso_request request)
     ISO_CUDA(cudaStreamSynchronize(stream));
     if (r.h_err && *r.h_err) {
         *r.h_err = 0;
-        cudaMemsetAsync(r.d_err, 0, sizeof(int), stream);
+        ISO_CUDA(cudaMemsetAsync(r.d_err, 0, sizeof(int), stream));
         if (r.d_counter) {
-            // a barrier gave up: start counting afresh
-            cudaMemsetAsync(r.d_counter, 0, (size_t)std::max(1, r.wave_counters) * sizeof(unsigned long long), stream);
+            // a wait gave up: the arrival counters hold a partial count, start afresh
+            ISO_CUDA(cudaMemsetAsync(r.d_counter, 0, (size_t)std::max(1, r.wave_counters) * sizeof(unsigned long long), stream));
             r.epoch = 0;
             r.wave_run = 0;
         }
+        ISO_CUDA(cudaStreamSynchronize(stream));
         return ISO_ERR_TIMEOUT;
     }
     return ISO_SUCCESS;
+    });
+}
+
+int Iso_request_check_guards(Iso_request request, int64_t *violations)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request) || !violations) return ISO_ERR_ARG;
+    Request &r = *request;
+    if (r.started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS && rc != ISO_ERR_TIMEOUT) return rc;
+    }
+    int64_t bad = 0;
+    if (r.d_inter_alloc) {
+        std::vector<unsigned char> band(2 * kGuardBytes);
+        ISO_CUDA(cudaMemcpy(band.data(), r.d_inter_alloc, kGuardBytes, cudaMemcpyDeviceToHost));
+        ISO_CUDA(cudaMemcpy(band.data() + kGuardBytes, r.d_inter + r.d_inter_bytes, kGuardBytes, cudaMemcpyDeviceToHost));
+        for (unsigned char b : band) bad += b != (unsigned char)kGuardPattern;
+    }
+    *violations = bad;
+    return ISO_SUCCESS;
+    });
+}
+
+int Iso_request_set_wait_limit(Iso_request request, unsigned int polls)
+{
+    if (check_handle(request) || polls == 0) return ISO_ERR_ARG;
+    request->wait_limit = polls;
+    return ISO_SUCCESS;
+}
+
+int Iso_request_test_skew_arrivals(Iso_request request, int extra)
+{
+    if (check_handle(request) || extra < 0 || extra > 1024) return ISO_ERR_ARG;
+    request->skew_next = extra;
+    return ISO_SUCCESS;
+}
+
+int Iso_measure_launch_floor(void *cuda_stream, int launches, int dependent, float *microseconds_per_launch)
+{
+    return guarded([&]() -> int {
+    if (launches < 1 || launches > (1 << 20) || !microseconds_per_launch) return ISO_ERR_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaEvent_t t0 = nullptr, t1 = nullptr;
+    ISO_CUDA(cudaEventCreate(&t0));
+    cudaError_t e = cudaEventCreate(&t1);
+    auto one = [&]() -> cudaError_t {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(1);
+        cfg.blockDim = dim3(32);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = dependent ? 1 : 0;
+        return cudaLaunchKernelEx(&cfg, iso_empty_kernel, 0);
+    };
+    for (int k = 0; k < 16 && e == cudaSuccess; ++k) e = one();
+    if (e == cudaSuccess) e = cudaEventRecord(t0, stream);
+    for (int k = 0; k < launches && e == cudaSuccess; ++k) e = one();
+    if (e == cudaSuccess) e = cudaEventRecord(t1, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    float ms = 0.0f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, t0, t1);
+    cudaEventDestroy(t0);
+    if (t1) cudaEventDestroy(t1);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *microseconds_per_launch = ms * 1e3f / (float)launches;
+    return ISO_SUCCESS;
+    });
 }
 
 int Iso_request_get_stats(Iso_request request, Iso_stats *out)
@@ -1523,15 +1612,15 @@ int scratch_for_current_device(unsigned char **out)
 {
     int device = 0;
     cudaError_t e = cudaGetDevice(&device);
-    if (e != cudaSuccess) return ISO_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_fail(e);
     if (device < 0 || device >= kMaxDevices) return ISO_ERR_ARG;
+    static std::mutex guard;  // two host threads may make their first call at the same time
+    std::lock_guard<std::mutex> lock(guard);
     if (!g_scratch_addr[device]) {
         void *p = nullptr;
         e = cudaGetSymbolAddress(&p, iso_static_scratch);
-        if (e != cudaSuccess || !p) {
-            (void)cudaGetLastError();
-            return ISO_ERR_CUDA;
-        }
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (!p) return ISO_ERR_CUDA;
         g_scratch_addr[device] = static_cast<unsigned char *>(p);
     }
     *out = g_scratch_addr[device];
@@ -1572,6 +1661,7 @@ extern "C" int Iso_neighbor_alltoall_static(int d, const int dims[], int s, cons
     const int64_t m = (int64_t)count * type;
     Request r;
     r.comm = &comm;
+    r.knobs = read_knobs();
     r.kind = ISO_KIND_ALLTOALL;
     r.alg = ISO_ALG_COMBINING;
     r.fusion = 1;
@@ -1620,11 +1710,11 @@ extern "C" int Iso_neighbor_alltoall_static(int d, const int dims[], int s, cons
     for (const LaunchPlan &L : r.launches) fill_units(r, L, reinterpret_cast<UnitDev *>(blob.data() + L.units_off));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     unsigned char *tables = scratch + inter_bytes;
-    if (table_bytes > 0 &&
-        cudaMemcpyAsync(tables, blob.data(), (size_t)table_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return ISO_ERR_CUDA;
-    }
+    // The copy reads `blob`, which dies with this call: outside a stream capture the runtime
+    // has staged a pageable source by the time the call returns, inside one the graph would
+    // keep the dangling host pointer - hence no call of this function inside a capture.
+    if (table_bytes > 0)
+        ISO_CUDA(cudaMemcpyAsync(tables, blob.data(), (size_t)table_bytes, cudaMemcpyHostToDevice, stream));
 
     // the ordinary launch path, pointed at the scratch area (nothing here is owned by `r`)
     r.d_blob = tables;

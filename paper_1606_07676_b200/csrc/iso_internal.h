@@ -81,8 +81,30 @@ struct LaunchPlan {
     size_t parts_off = 0, lookup_off = 0, units_off = 0;
 };
 
+// Experiment knobs, read from the environment ONCE, when a request is created, so that a
+// persistent request keeps one plan however the environment changes between its starts.
+// -1 (or 0 where stated) means "not set": the library's own choice applies.
+struct Knobs {
+    int pack_by_round = -1;   // ISO_PACK_BY_ROUND: intermediate places grouped by reading round (0/1)
+    int lazy_final = -1;      // ISO_LAZY_FINAL: postpone every final hop to the last phase (0/1)
+    int mixed = -1;           // ISO_MIXED: 0 = one launch per unit width instead of one of mixed widths
+    int64_t bulk_chunk = 0;   // ISO_BULK_CHUNK: chunk bytes of the bulk kernel (0: automatic)
+    int vec_threads = 0;      // ISO_VEC_THREADS: 256 or 512 for narrower CTAs (0: up to 1024)
+    int vec_ctas_per_sm = 0;  // ISO_VEC_CTAS_PER_SM: CTAs per SM of the 256-thread shapes (0: automatic)
+    int64_t bulk_tile = 0;    // ISO_BULK_TILE: processes per CTA of the bulk kernel (0: automatic)
+    int host_slabs = -1;      // ISO_HOST_SLABS: slabs of the pipelined host-buffer path (-1: automatic)
+    int graph = -1;           // ISO_GRAPH: graph replay on/off
+    int slabs = -1;           // ISO_SLABS: slab count of Iso_Start
+    int chains = -1;          // ISO_CHAINS
+    bool no_pdl = false;      // ISO_NO_PDL: plain launches instead of programmatic dependent ones
+    bool tune_log = false;    // ISO_TUNE_LOG: the tuner prints every plan it times
+    bool multi_dst = true;    // ISO_MULTI_DST=0: allgather units with one destination each
+};
+Knobs read_knobs();
+
 struct Request {
     Comm *comm = nullptr;
+    Knobs knobs;
     int kind = ISO_KIND_ALLTOALL;
     int alg = ISO_ALG_COMBINING;
     int fusion = 1;
@@ -101,7 +123,8 @@ struct Request {
     // device side (owned by iso_api.cu)
     bool dirty = true;
     void *d_blob = nullptr;
-    unsigned char *d_inter = nullptr;
+    unsigned char *d_inter = nullptr;        // first usable byte (behind the leading guard band)
+    unsigned char *d_inter_alloc = nullptr;  // the allocation: guard band, buffer, guard band
     int64_t d_inter_bytes = 0;
     int *d_err = nullptr;
     unsigned long long *d_counter = nullptr;  // grid-barrier arrivals (one-launch execution)
@@ -116,7 +139,7 @@ struct Request {
     void *copy_stream = nullptr;       // download stream of the pipelined host-buffer path
     void *up_stream = nullptr;         // its upload stream
     std::vector<void *> slab_events;   // its events
-    int sm_count = 148;  // replaced by the device's count when the request is materialised
+    int sm_count = 148;  // a B200's; replaced by the current device's count before the first start
     int chains_request = 1;     // slabs to run side by side, as asked for
     bool graph_request = false; // graph replay, as asked for
     int chains = 1;             // slabs that run side by side (each on its share of the SMs)
@@ -131,6 +154,8 @@ struct Request {
     size_t wave_smem = 0, wave_launches_off = 0, wave_items_off = 0;
     unsigned long long wave_run = 0;  // starts since the counters were last zeroed
     int wave_counters = 0;      // counters allocated in d_counter
+    uint32_t wait_limit = 1u << 22;  // polls before a device-side wait on other CTAs gives up
+    int skew_next = 0;          // testing: extra arrivals the next cooperative start waits for (one shot)
 };
 
 // Builds r.parts, r.inter_stride and the schedule statistics from r.comm, r.kind, r.alg,

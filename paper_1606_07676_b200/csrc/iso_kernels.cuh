@@ -397,9 +397,11 @@ struct MultiDev {
     unsigned long long *counter;  // arrivals at the grid barrier, never reset
     unsigned long long epoch;     // value of the counter when this launch began
     int *err;                     // set to 2 when a barrier wait gives up
+    uint32_t max_polls;           // polls of one wait before it gives up
+    uint32_t arrivals;            // arrivals that complete one barrier (the grid size, unless a test skews it)
 };
 
-constexpr uint32_t kBarrierPolls = 1u << 22;
+constexpr uint32_t kBarrierPolls = 1u << 22;  // default poll limit of the waits on other CTAs
 
 // Grid-wide barrier for a cooperative launch (all CTAs are resident).  One thread per CTA
 // publishes the CTA's writes, counts itself in and polls the counter a bounded number of
@@ -416,7 +418,7 @@ __device__ __forceinline__ bool grid_barrier(const MultiDev &M, unsigned long lo
             unsigned long long seen;
             asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(M.counter) : "memory");
             if (seen >= target) break;
-            if (++polls >= kBarrierPolls) {
+            if (++polls >= M.max_polls) {
                 ok = false;
                 break;
             }
@@ -449,7 +451,7 @@ __global__ void __launch_bounds__(1024, 1) iso_gather_rows_multi(const __grid_co
         case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
         default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
         }
-        if (ph + 1 < M.n && !grid_barrier(M, M.epoch + (unsigned long long)(ph + 1) * gridDim.x, &s_ok)) return;
+        if (ph + 1 < M.n && !grid_barrier(M, M.epoch + (unsigned long long)(ph + 1) * M.arrivals, &s_ok)) return;
     }
 }
 
@@ -475,6 +477,7 @@ struct WaveDev {
     unsigned long long *done;   // per item: arrivals of CTAs, never reset
     unsigned long long target;  // arrivals that mean "complete" for this start
     int *err;                   // set to 2 when a wait gives up
+    uint32_t max_polls;         // polls of one wait before it gives up
 };
 
 template <int DEPTH>
@@ -500,7 +503,7 @@ __global__ void __launch_bounds__(1024, 1) iso_gather_rows_wave(const __grid_con
                     unsigned long long seen;
                     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(seen) : "l"(flag) : "memory");
                     if (seen >= M.target) break;
-                    if (++polls >= kBarrierPolls) {
+                    if (++polls >= M.max_polls) {
                         ok = false;
                         break;
                     }
@@ -584,6 +587,14 @@ __global__ void __launch_bounds__(256) iso_gather_rows_reg(const __grid_constant
                 if (dst[k]) *dst[k] = val[k];
         }
     }
+}
+
+// Does nothing: a chain of these measures what a kernel launch costs on the stream
+// (with and without programmatic dependent launch), the floor under every short phase.
+__global__ void iso_empty_kernel(int)
+{
+    grid_dependency_wait();
+    grid_launch_dependents();
 }
 
 // ---- asynchronous bulk copies (TMA, untiled form) ------------------------------------

@@ -39,6 +39,30 @@ FastDiv make_fastdiv(uint32_t d)
     return f;
 }
 
+Knobs read_knobs()
+{
+    Knobs k;
+    auto num = [](const char *name, long long unset) -> long long {
+        const char *v = std::getenv(name);
+        return v ? std::atoll(v) : unset;
+    };
+    k.pack_by_round = (int)num("ISO_PACK_BY_ROUND", -1);
+    k.lazy_final = (int)num("ISO_LAZY_FINAL", -1);
+    k.mixed = (int)num("ISO_MIXED", -1);
+    k.bulk_chunk = num("ISO_BULK_CHUNK", 0);
+    k.vec_threads = (int)num("ISO_VEC_THREADS", 0);
+    k.vec_ctas_per_sm = (int)num("ISO_VEC_CTAS_PER_SM", 0);
+    k.bulk_tile = num("ISO_BULK_TILE", 0);
+    k.host_slabs = (int)num("ISO_HOST_SLABS", -1);
+    k.graph = (int)num("ISO_GRAPH", -1);
+    k.slabs = (int)num("ISO_SLABS", -1);
+    k.chains = (int)num("ISO_CHAINS", -1);
+    k.no_pdl = num("ISO_NO_PDL", 0) != 0;
+    k.tune_log = std::getenv("ISO_TUNE_LOG") != nullptr;
+    k.multi_dst = num("ISO_MULTI_DST", 1) != 0;
+    return k;
+}
+
 namespace {
 
 int reduce_mod(int c, int p)
@@ -218,7 +242,7 @@ void pack_intermediates(Request &r, int s, bool final_by_dst)
     for (int i = 0; i < s; ++i)
         if (r.len[i] > 0) min_len = std::min(min_len, r.len[i]);
     bool by_round = min_len >= 32;
-    if (const char *env = std::getenv("ISO_PACK_BY_ROUND")) by_round = std::atoi(env) != 0;
+    if (r.knobs.pack_by_round >= 0) by_round = r.knobs.pack_by_round != 0;
     for (int i = 0; i < s; ++i)
         for (size_t j = 0; j + 1 < chain[i].size(); ++j)
             places.push_back(Place{r.parts[chain[i][j]].phase, r.parts[chain[i][j + 1]].phase,
@@ -351,8 +375,8 @@ int build_combining_alltoall(Request &r, const Geometry &g)
     bool lazy_final = r.layout == ISO_LAYOUT_PACKED && r.fusion != 0 && phase > 1;
     for (int i = 0; i < g.s; ++i)
         if (r.len[i] > 16) lazy_final = false;
-    if (const char *env = std::getenv("ISO_LAZY_FINAL"))
-        lazy_final = r.layout == ISO_LAYOUT_PACKED && r.fusion != 0 && phase > 1 && std::atoi(env) != 0;
+    if (r.knobs.lazy_final >= 0)
+        lazy_final = r.layout == ISO_LAYOUT_PACKED && r.fusion != 0 && phase > 1 && r.knobs.lazy_final != 0;
     if (lazy_final) {
         std::vector<int> last_hop(g.s, -1);
         for (size_t k = 0; k < r.parts.size(); ++k) last_hop[r.parts[k].slot] = (int)k;
@@ -437,9 +461,21 @@ int build_combining_allgather(Request &r, const Geometry &g)
     const Groups gr = make_groups(g.d, r.fusion);
     const int64_t m = g.s ? r.len[0] : 0;
     struct Store { int buf; int64_t off; };
+    // Non-periodic dimensions (Section VII): the node of prefix Q exists at process x only if
+    // the process x - (Q, 0, ..., 0) does, so a part that produces it carries, for every mesh
+    // dimension already visited, the prefix's coordinate as its check value.  A node kept in
+    // a receive slot is then written exactly where that slot's block is deliverable, and
+    // elsewhere the slot keeps its contents.  A neighbour whose coordinate reaches across
+    // the whole mesh can never be served and takes no part.
+    bool mesh = false;
+    for (int j = 0; j < g.d; ++j) mesh |= !c.periodic[j];
+    std::vector<char> dead(g.s, 0);
+    for (int i = 0; i < g.s; ++i)
+        for (int j = 0; j < g.d; ++j)
+            if (!c.periodic[j] && std::abs((int64_t)g.at(i)[j]) >= c.dims[j]) dead[i] = 1;
     std::map<std::vector<int>, int> first_with_vector;  // full vector -> smallest slot
     for (int i = g.s - 1; i >= 0; --i)
-        first_with_vector[std::vector<int>(g.at(i), g.at(i) + g.d)] = i;
+        if (!dead[i]) first_with_vector[std::vector<int>(g.at(i), g.at(i) + g.d)] = i;
 
     std::map<std::vector<int>, Store> storage;  // prefix -> where that block lives
     storage[std::vector<int>()] = Store{ISO_BUF_SEND, 0};
@@ -450,18 +486,19 @@ int build_combining_allgather(Request &r, const Geometry &g)
 
     if (m > 0)
         for (int i = 0; i < g.s; ++i)
-            if (!group_nonzero(g.at(i), 0, g.d)) { add_local_copy(r, i, locals_parts); served[i] = 1; ++locals; }
+            if (!dead[i] && !group_nonzero(g.at(i), 0, g.d)) { add_local_copy(r, i, locals_parts); served[i] = 1; ++locals; }
 
     for (int k = 0; k < gr.n && m > 0; ++k) {
         const int j0 = gr.begin[k], j1 = gr.begin[k + 1];
         // rounds of this group: distinct non-zero coordinate keys
         std::map<std::vector<int>, int, RoundOrder> round_of(RoundOrder{c.dims, c.periodic, j0, j1});
         for (int i = 0; i < g.s; ++i)
-            if (group_nonzero(g.at(i), j0, j1)) round_of[std::vector<int>(g.at(i) + j0, g.at(i) + j1)] = 0;
+            if (!dead[i] && group_nonzero(g.at(i), j0, j1)) round_of[std::vector<int>(g.at(i) + j0, g.at(i) + j1)] = 0;
         nmax = std::max<int>(nmax, (int)round_of.size());
         for (auto &kv : round_of) kv.second = round++;
         const size_t group_begin = r.parts.size();
         for (int i = 0; i < g.s; ++i) {
+            if (dead[i]) continue;
             std::vector<int> prefix(g.at(i), g.at(i) + j1), parent(g.at(i), g.at(i) + j0);
             const Store src = storage.at(parent);
             if (!group_nonzero(g.at(i), j0, j1)) {
@@ -482,6 +519,9 @@ int build_combining_allgather(Request &r, const Geometry &g)
                 p.dst_off = dst.off;
                 p.len = m;
                 std::memcpy(p.shift, shift, sizeof(shift));
+                if (mesh)
+                    for (int j = 0; j < j1; ++j)
+                        if (!c.periodic[j]) p.check[j] = g.at(i)[j];
                 r.parts.push_back(p);
                 ++parts;
             };
@@ -553,8 +593,10 @@ int build_schedule(Request &r)
             int v = c.coords[(size_t)i * c.d + j];
             g.red[(size_t)i * c.d + j] = c.periodic[j] ? reduce_mod(v, c.dims[j]) : v;
         }
-    // meshes: the direct schedule, and the combining schedule of the all-to-all
-    if (mesh && !(r.alg == ISO_ALG_DIRECT || (r.alg == ISO_ALG_COMBINING && r.kind != ISO_KIND_ALLGATHER))) return ISO_ERR_ARG;
+    // meshes: the direct and the combining schedules; Algorithm 1 as printed alternates a
+    // block between its receive slot and the intermediate buffer, which an undelivered
+    // slot that must keep its contents does not allow
+    if (mesh && r.alg == ISO_ALG_TORUS) return ISO_ERR_ARG;
     const bool gather = r.kind == ISO_KIND_ALLGATHER;
     if (r.alg == ISO_ALG_TORUS && gather) return ISO_ERR_ARG;
     if (r.alg != ISO_ALG_COMBINING && r.alg != ISO_ALG_DIRECT && r.alg != ISO_ALG_TORUS) return ISO_ERR_ARG;
@@ -664,7 +706,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
 
         // whether this phase may run as one launch of mixed unit widths
         bool allow_mixed = r.wave_request == 0 && !r.persistent;
-        if (const char *env = std::getenv("ISO_MIXED")) allow_mixed = allow_mixed && std::atoi(env) != 0;
+        if (r.knobs.mixed >= 0) allow_mixed = allow_mixed && r.knobs.mixed != 0;
         // split every part into pieces that share one alignment class
         // cls: width class of the launch (0: mixed widths); base: alignment of the rows it touches
         struct Piece { Part p; int kernel; int width; int cls; int base; };
@@ -806,9 +848,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         for (size_t k = lo; k < hi; ++k) min_len = std::min(min_len, cls[k].p.len);
                         unit = 256;
                         while (unit * 2 <= min_len && unit < 2048) unit *= 2;
-                        const char *env = std::getenv("ISO_BULK_CHUNK");
-                        if (env) {
-                            int64_t v = std::atoll(env);
+                        if (r.knobs.bulk_chunk) {
+                            const int64_t v = r.knobs.bulk_chunk;
                             if (v >= 16 && v <= 16384 && v % 16 == 0) unit = v;
                         }
                     }
@@ -871,8 +912,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         // per all-to-all on the 32^3 torus, 161 against 184 on the 8^5 torus);
                         // ISO_VEC_THREADS=256 or 512 selects the narrower shapes
                         uint32_t max_threads = (width == 16 || width == 0) ? 1024 : 256;
-                        if (const char *env = std::getenv("ISO_VEC_THREADS")) {
-                            const int v = std::atoi(env);
+                        if (r.knobs.vec_threads) {
+                            const int v = r.knobs.vec_threads;
                             if ((v == 256 || v == 512) && max_threads == 1024) max_threads = units > 256 ? 1024 : (uint32_t)v;
                         }
                         L.chunk_units = (uint32_t)std::min<uint64_t>(units, max_threads);
@@ -880,8 +921,8 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         L.threads = (int)((L.chunk_units * L.rows_per_pass + 31) / 32 * 32);
                         // CTAs of fewer than 256 threads: as many per SM as keep 1024 threads resident
                         int per_sm = L.threads > 512 ? 1 : (L.threads > 256 ? 2 : std::min(16, std::max(4, 1024 / L.threads)));
-                        if (const char *env = std::getenv("ISO_VEC_CTAS_PER_SM")) {
-                            int v = std::atoi(env);
+                        if (r.knobs.vec_ctas_per_sm) {
+                            const int v = r.knobs.vec_ctas_per_sm;
                             if (v >= 1 && v <= 8 && L.threads <= 256) per_sm = v;
                         }
                         // persistent grid: CTA b takes the row groups b, b + grid, ...
@@ -894,10 +935,10 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         L.threads = std::max(32, std::min(256, threads));
                         tp = std::max<int64_t>(1, (8 * (int64_t)L.threads + (int64_t)units - 1) / (int64_t)units);
                         tp = std::min<int64_t>(tp, 512);
-                        tp = std::min<int64_t>(tp, std::max<int64_t>(1, c.P / (148 * 2)));
+                        tp = std::min<int64_t>(tp, std::max<int64_t>(1, c.P / ((int64_t)r.sm_count * 2)));
                         while (tp > 1 && (uint64_t)tp * units > 0x7fffffffull) tp /= 2;
-                        if (const char *env_tp = std::getenv("ISO_BULK_TILE")) {
-                            int64_t v = std::atoll(env_tp);
+                        if (r.knobs.bulk_tile) {
+                            const int64_t v = r.knobs.bulk_tile;
                             if (v >= 1 && v <= 512 && (uint64_t)v * units <= 0x7fffffffull) tp = v;
                         }
                         grid = (c.P + tp - 1) / tp;

@@ -59,14 +59,15 @@ layout = wl.layout
 send_buffer_np = wl.send_buffer_np
 
 
-def oracle_result(w, send, r0=0, r1=None, fill=POISON):
-    """Expected receive buffers of ranks [r0, r1) from the CPU oracle."""
+def oracle_result(w, send, r0=0, r1=None, fill=POISON, periodic=None):
+    """Expected receive buffers of ranks [r0, r1) from the CPU oracle; with non-periodic
+    dimensions, slots that are not delivered hold `fill`."""
     lens, sd, rd, ss, rs = layout(w)
     if w.collective == "alltoall":
-        return oracle.alltoall(w.dims, w.offsets, w.block_bytes, send, r0, r1)
+        return oracle.alltoall(w.dims, w.offsets, w.block_bytes, send, r0, r1, periodic=periodic, fill=fill)
     if w.collective == "allgather":
-        return oracle.allgather(w.dims, w.offsets, w.block_bytes, send, r0, r1)
-    return oracle.alltoallv(w.dims, w.offsets, lens, sd, rd, ss, rs, send, r0, r1, fill=fill)
+        return oracle.allgather(w.dims, w.offsets, w.block_bytes, send, r0, r1, periodic=periodic, fill=fill)
+    return oracle.alltoallv(w.dims, w.offsets, lens, sd, rd, ss, rs, send, r0, r1, fill=fill, periodic=periodic)
 
 
 def make_request(w, sendbuf=None, recvbuf=None, periodic=None):

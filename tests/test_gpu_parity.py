@@ -248,6 +248,7 @@ def test_cfg3_4096_sampled(torch_cuda):
     comm, req = make_request(w, send, recv)
     rng = np.random.default_rng(5)
     ranks = sorted({0, 1, 255, 256, 257, 511, P - 1, P - 256, P - 257, *rng.integers(0, P, 24).tolist()})
+    host_send = None
     try:
         for alg, fusion in (COMB1, DIRECT):
             iso.Iso_request_set_algorithm(req, alg, fusion)
@@ -262,6 +263,20 @@ def test_cfg3_4096_sampled(torch_cuda):
                     q = oracle.source_rank(w.dims, r, w.offsets[i])
                     want = wl.payload_np(w.kind, w.seed, 0, q * stride + i * m, m)
                     assert np.array_equal(got[i], want), (alg, r, i)
+            # whole planes of dimension 0 at both wrap-around edges, from the oracle run on
+            # their rank ranges: the host send buffer is reserved in full but only the eight
+            # planes those ranks read from (252..255, 0..3) are generated
+            if host_send is None:
+                host_send = np.empty((P, stride), dtype=np.uint8)
+                plane = w.dims[1]
+                for x in (252, 253, 254, 255, 0, 1, 2, 3):
+                    host_send[x * plane:(x + 1) * plane] = wl.payload_np(
+                        w.kind, w.seed, 0, x * plane * stride, plane * stride).reshape(plane, stride)
+            for x in (0, 1, 254, 255):
+                r0, r1 = x * w.dims[1], (x + 1) * w.dims[1]
+                want = oracle.alltoall(w.dims, w.offsets, m, host_send, r0, r1)
+                got = recv[r0 * stride:r1 * stride].cpu().numpy().reshape(r1 - r0, stride)
+                assert np.array_equal(got, want), (alg, "plane", x)
             # a property that holds at any size: the result is a permutation of the send
             # blocks, so per-slot byte sums over all processes are preserved
             a = send.view(P, s, m)[:, 3].to(torch.int64).sum().item()
@@ -427,23 +442,16 @@ def test_mesh(torch_cuda):
     """Non-periodic dimensions: blocks whose source lies outside are not delivered."""
     torch = torch_cuda
     for dims, periodic, offs, m in [((9, 11), [0, 0], wl.moore(2, 2), 16), ((6, 7, 5), [0, 1, 0], wl.moore(3, 1), 64),
-                                    ((12, 9), [1, 0], wl.moore(2, 1), 1024)]:
-        w = wl.Workload("mesh", "alltoall", dims, offs, m, seed=4)
-        run = Run(torch, w, periodic=periodic)
-        full = oracle_result(w, run.send_host).reshape(w.P, w.s, m)
-        want = np.full_like(full, POISON)
-        coords = np.stack(np.unravel_index(np.arange(w.P), dims), axis=1)
-        for i, C in enumerate(offs):
-            inside = np.ones(w.P, bool)
-            for j, per in enumerate(periodic):
-                if not per:
-                    y = coords[:, j] - int(C[j])
-                    inside &= (y >= 0) & (y < dims[j])
-            want[inside, i] = full[inside, i]
-        for alg, fusion in (DIRECT, COMB1, COMB0, COMB2, ALT1):
-            got = run.result(alg, fusion).reshape(w.P, w.s, m)
-            assert np.array_equal(got, want), (dims, alg, fusion)
-        run.close()
+                                    ((12, 9), [1, 0], wl.moore(2, 1), 1024), ((7, 6, 5), [0, 0, 1], wl.positive_octant(3, 3), 16)]:
+        for coll in ("alltoall", "allgather"):
+            w = wl.Workload("mesh", coll, dims, offs, m, seed=4)
+            run = Run(torch, w, periodic=periodic)
+            want = oracle_result(w, run.send_host, periodic=periodic)
+            algs = (DIRECT, COMB1, COMB0, COMB2, ALT1) if coll == "alltoall" else (DIRECT, COMB1, COMB0, COMB2)
+            for alg, fusion in algs:
+                got = run.result(alg, fusion)
+                assert np.array_equal(got, want), (dims, coll, alg, fusion)
+            run.close()
 
 
 def test_persistent_request_streams_and_host_buffers(torch_cuda):

@@ -195,7 +195,93 @@ def pin_chunks(lib):
     assert np.array_equal(np.concatenate(parts), full)
 
 
-PINS = [pin_golden, pin_golden_allgather, pin_push_equals_pull, pin_numpy_special_cases, pin_rank_helpers, pin_chunks]
+def _padded(rows, width, dtype=np.uint8, rng=None):
+    """`rows` x `width` array that is a view into a larger allocation, so that a planted
+    off-by-one in a mesh bound reads defined memory instead of running off the array."""
+    backing = np.zeros((rows + 16, width), dtype=dtype) if rng is None else \
+        rng.integers(0, 256, size=(rows + 16, width)).astype(dtype)
+    return backing[:rows]
+
+
+def pin_golden_mesh(lib):
+    dims, periodic, offs = (3, 4), (0, 0), moore_list(2, 1)
+    P, s = 12, 8
+    send = _padded(P, s, np.int32)
+    send[:] = [[100 * q + i for i in range(s)] for q in range(P)]
+    KEEP = 0x77
+    recv = oracle.alltoall(dims, offs, 4, send, lib=lib, periodic=periodic, fill=KEEP).view(np.int32).reshape(P, s)
+    kept = int(np.array([KEEP] * 4, np.uint8).view(np.int32)[0])
+    n = 0
+    for line in open(os.path.join(GOLDEN, "mesh_3x4_alltoall.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        rank, vals = line.split(":")
+        want = [kept if v == "-" else int(v) for v in vals.split()]
+        assert recv[int(rank)].tolist() == want, "rank " + rank
+        n += 1
+    assert n == 4
+    # the same geometry as an allgather: slot i holds the source's single value or is kept
+    blk = _padded(P, 1, np.int32)
+    blk[:, 0] = [100 * q for q in range(P)]
+    got = oracle.allgather(dims, offs, 4, blk, lib=lib, periodic=periodic, fill=KEEP).view(np.int32).reshape(P, s)
+    assert got[0].tolist() == [500, 400, kept, 100, kept, kept, kept, kept]
+    assert got[11].tolist() == [kept, kept, kept, kept, 1000, kept, 700, 600]
+
+
+def push_mesh(dims, periodic, offsets, lens, sdispls, rdispls, sstride, rstride, send, fill):
+    """Sender's side on a mesh: q sends block i to q + C^i if that process exists."""
+    P = int(np.prod(dims))
+    recv = np.full((P, rstride), fill, dtype=np.uint8)
+    for q in range(P):
+        Q = coords_of(q, dims)
+        for i, C in enumerate(offsets):
+            T = []
+            for a, c, p, per in zip(Q, C, dims, periodic):
+                t = a + int(c)
+                if per:
+                    t %= p
+                elif not 0 <= t < p:
+                    T = None
+                    break
+                T.append(t)
+            if T is None:
+                continue
+            t = rank_of(T, dims)
+            recv[t, rdispls[i]:rdispls[i] + lens[i]] = send[q, sdispls[i]:sdispls[i] + lens[i]]
+    return recv
+
+
+def pin_mesh_push_equals_pull(lib):
+    rng = np.random.default_rng(19)
+    for dims, periodic in [((5,), (0,)), ((3, 4), (0, 1)), ((3, 4), (1, 0)), ((2, 3, 4), (0, 1, 0)), ((4, 1, 3), (0, 0, 0)),
+                           ((3, 3), (1, 1))]:
+        d, P = len(dims), int(np.prod(dims))
+        s = 9
+        offs = rng.integers(-4, 5, size=(s, d)).astype(np.int32)
+        offs[0] = 0
+        offs[3] = offs[2]
+        m = 3
+        ld, dd = np.full(s, m, np.int64), np.arange(s, dtype=np.int64) * m
+        send = _padded(P, s * m, rng=rng)
+        want = push_mesh(dims, periodic, offs, ld, dd, dd, s * m, s * m, send, 0xA5)
+        assert np.array_equal(oracle.alltoall(dims, offs, m, send, lib=lib, periodic=periodic, fill=0xA5), want), (dims, periodic)
+        got = oracle.alltoallv(dims, offs, ld, dd, dd[::-1].copy(), s * m, s * m, send, fill=0xA5, lib=lib, periodic=periodic)
+        assert np.array_equal(got, push_mesh(dims, periodic, offs, ld, dd, dd[::-1], s * m, s * m, send, 0xA5)), (dims, periodic)
+        blk = _padded(P, m, rng=rng)
+        want = push_mesh(dims, periodic, offs, ld, np.zeros(s, np.int64), dd, m, s * m, blk, 0xA5)
+        assert np.array_equal(oracle.allgather(dims, offs, m, blk, lib=lib, periodic=periodic, fill=0xA5), want), (dims, periodic)
+        for r in range(P):
+            R = coords_of(r, dims)
+            for C in offs:
+                src = [a - int(c) for a, c in zip(R, C)]
+                inside = all(per or 0 <= y < p for y, p, per in zip(src, dims, periodic))
+                q = oracle.source_rank_mesh(dims, periodic, r, C, lib=lib)
+                assert (q >= 0) == inside
+                if inside:
+                    assert q == rank_of([y % p for y, p in zip(src, dims)], dims)
+
+
+PINS = [pin_golden_mesh, pin_mesh_push_equals_pull, pin_golden, pin_golden_allgather, pin_push_equals_pull, pin_numpy_special_cases, pin_rank_helpers, pin_chunks]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -217,6 +303,11 @@ MUTANTS = {
     "alltoallv_swaps_displacements": ("recv + (r - r0) * recv_stride + rdispl[i],\n                   send + q * send_stride + sdispl[i]",
                                       "recv + (r - r0) * recv_stride + sdispl[i],\n                   send + q * send_stride + rdispl[i]"),
     "alltoallv_wrong_stride": ("send + q * send_stride + sdispl[i]", "send + q * recv_stride + sdispl[i]"),
+    "mesh_checks_the_receiver_side": ("int64_t y = coord[j] - (int64_t)C[j];", "int64_t y = coord[j] + (int64_t)C[j];"),
+    "mesh_upper_edge_inclusive": ("} else if (y < 0 || y >= p) {", "} else if (y < 0 || y > p) {"),
+    "mesh_flags_ignored": ("        if (periodic[j]) {\n            y = y % p;", "        if (1) {\n            y = y % p;"),
+    "mesh_allgather_reads_own_block": ("            memcpy(recv + ((r - r0) * s + i) * m, send + q * m, (size_t)m);\n        }\n    }\n    return 0;\n}\n\n/* Irregular all-to-all on a mesh",
+                                       "            memcpy(recv + ((r - r0) * s + i) * m, send + r * m, (size_t)m);\n        }\n    }\n    return 0;\n}\n\n/* Irregular all-to-all on a mesh"),
     "offset_row_ignored": ("offsets + (int64_t)i * d);\n            memcpy(recv + ((r - r0) * s + i) * m, send + (q * s + i) * m",
                            "offsets + (int64_t)0 * d);\n            memcpy(recv + ((r - r0) * s + i) * m, send + (q * s + i) * m"),
 }

@@ -323,23 +323,6 @@ def test_ragged_phases_lower_to_one_launch_of_mixed_widths(monkeypatch):
         iso.Iso_comm_free(comm)
 
 
-def _mesh_expected(w, send, periodic):
-    """Oracle result with the blocks whose source lies outside a non-periodic dimension left
-    at the poison value (the receive slot keeps its previous contents)."""
-    m = w.block_bytes
-    full = oracle_result(w, send).reshape(w.P, w.s, m)
-    want = np.full_like(full, POISON)
-    coords = np.stack(np.unravel_index(np.arange(w.P), w.dims), axis=1)
-    for i, C in enumerate(w.offsets):
-        inside = np.ones(w.P, bool)
-        for j, per in enumerate(periodic):
-            if not per:
-                y = coords[:, j] - int(C[j])
-                inside &= (y >= 0) & (y < w.dims[j])
-        want[inside, i] = full[inside, i]
-    return want.reshape(w.P, w.s * m)
-
-
 @pytest.mark.parametrize("dims,periodic,nbh", [((4, 5), [0, 1], "moore2"), ((5, 4, 3), [0, 0, 0], "moore1"),
                                                ((3, 6, 4), [1, 0, 1], "moore1"), ((7, 2), [0, 0], "far")])
 def test_mesh_schedules(dims, periodic, nbh):
@@ -354,21 +337,23 @@ def test_mesh_schedules(dims, periodic, nbh):
         st = iso.Iso_request_get_stats(req)
         send = send_buffer_np(w, st["send_stride"])
         got = simulate(iso.Iso_request_get_parts(req), w.dims, st, send, periodic=periodic)
-        assert np.array_equal(got, _mesh_expected(w, send, periodic)), (alg, fusion)
+        assert np.array_equal(got, oracle_result(w, send, periodic=periodic)), (alg, fusion)
     with pytest.raises(iso.IsoError):
         iso.Iso_request_set_algorithm(req, iso.ISO_ALG_TORUS, 1)
     iso.Iso_request_free(req)
     iso.Iso_comm_free(comm)
-    # allgather on a mesh: the direct schedule only
+    # allgather on a mesh: direct and combining (a trie node exists only where its source does)
     wg = wl.Workload("mesh", "allgather", dims, offs, 4)
     comm, req = make_request(wg, periodic=periodic)
-    assert iso.Iso_request_get_stats(req)["algorithm"] == iso.ISO_ALG_DIRECT
-    st = iso.Iso_request_get_stats(req)
-    send = send_buffer_np(wg, st["send_stride"])
-    got = simulate(iso.Iso_request_get_parts(req), wg.dims, st, send, periodic=periodic)
-    assert np.array_equal(got, _mesh_expected(wg, send, periodic))
+    assert iso.Iso_request_get_stats(req)["algorithm"] == iso.ISO_ALG_COMBINING
+    for alg, fusion in [(iso.ISO_ALG_COMBINING, 1), (iso.ISO_ALG_COMBINING, 0), (iso.ISO_ALG_COMBINING, 2), (iso.ISO_ALG_DIRECT, 1)]:
+        set_alg(req, alg, fusion)
+        st = iso.Iso_request_get_stats(req)
+        send = send_buffer_np(wg, st["send_stride"])
+        got = simulate(iso.Iso_request_get_parts(req), wg.dims, st, send, periodic=periodic)
+        assert np.array_equal(got, oracle_result(wg, send, periodic=periodic)), (alg, fusion)
     with pytest.raises(iso.IsoError):
-        iso.Iso_request_set_algorithm(req, iso.ISO_ALG_COMBINING, 1)
+        iso.Iso_request_set_algorithm(req, iso.ISO_ALG_TORUS, 1)
     iso.Iso_request_free(req)
     iso.Iso_comm_free(comm)
 

@@ -1,4 +1,4 @@
-"""The allocation-free all-to-all entry point against the ordinary one.
+"""The allocation-free all-to-all entry point against the CPU oracle and the ordinary path.
 
 `Iso_neighbor_alltoall_static` serves callers that may not allocate device memory where
 they need the collective (a fixed memory budget handed out at start-up, a host framework
@@ -10,13 +10,14 @@ result of any other test in a run that stops at the first failure.
 import numpy as np
 import pytest
 
+import oracle
 from paper_1606_07676_b200 import binding as iso
 from paper_1606_07676_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
 
-def _reference(torch, dims, offs, m, send):
+def _allocating(torch, dims, offs, m, send):
     """The existing entry points: init + start + wait (allocates tables and buffer)."""
     P, s = int(np.prod(dims)), len(offs)
     recv = torch.full((P, s * m), 0xA5, dtype=torch.uint8, device="cuda")
@@ -29,29 +30,55 @@ def _reference(torch, dims, offs, m, send):
     return recv
 
 
-def test_static_entry_point_matches_the_allocating_one_twice_in_a_row():
+def _cases():
+    odd = np.array([[0, 0, 0], [1, 0, -1], [1, 0, -1], [-5, 3, 2], [0, 1, 0], [2, 2, 2]], np.int32)  # zero vector, a repeat, |c| >= p
+    return [((8, 8, 8), wl.moore(3, 1), 64, 11), ((12, 10), wl.moore(2, 2), 24, 12),
+            ((7, 5), wl.moore(2, 1), 1, 13), ((6, 4, 3), wl.moore(3, 1), 2, 14), ((9, 11), wl.moore(2, 2), 20, 15),
+            ((3, 1, 2), odd, 16, 16), ((2, 2), wl.moore(2, 1), 48, 17), ((5, 4, 3, 2), wl.moore(4, 1), 8, 18)]
+
+
+def test_static_entry_point_matches_the_oracle_twice_in_a_row():
     import torch
     if not torch.cuda.is_available():
         pytest.fail("needs a CUDA device")
     torch.cuda.set_device(0)
-    # two different problems back to back: the second call finds the scratch area full of
-    # the first call's tables and intermediate blocks
-    cases = [((8, 8, 8), wl.moore(3, 1), 64, 11), ((12, 10), wl.moore(2, 2), 24, 12)]
-    for dims, offs, m, seed in cases:
+    # different problems back to back: every call finds the scratch area full of the previous
+    # call's tables and intermediate blocks
+    for dims, offs, m, seed in _cases():
         P, s = int(np.prod(dims)), len(offs)
-        send = wl.payload_torch("uint8", seed, 0, P * s * m, "cuda").view(P, s * m)
-        want = _reference(torch, dims, offs, m, send)
         got = torch.full((P, s * m), 0x5A, dtype=torch.uint8, device="cuda")
-        iso.Iso_neighbor_alltoall_static(dims, offs, send, got, m, iso.ISO_BYTE, torch.cuda.current_stream())
-        torch.cuda.synchronize()
-        assert torch.equal(got, want), "first call differs (dims %s)" % (dims,)
-        # same problem again with new payload: same scratch contents layout, new data
-        send2 = wl.payload_torch("uint8", seed + 100, 0, P * s * m, "cuda").view(P, s * m)
-        want2 = _reference(torch, dims, offs, m, send2)
-        got.fill_(0x5A)
-        iso.Iso_neighbor_alltoall_static(dims, offs, send2, got, m, iso.ISO_BYTE, torch.cuda.current_stream())
-        torch.cuda.synchronize()
-        assert torch.equal(got, want2), "second call differs (dims %s)" % (dims,)
+        for call in range(2):       # the same problem twice, with new contents the second time
+            send_h = wl.payload_np("uint8", seed + 100 * call, 0, 0, P * s * m).reshape(P, s * m).copy()
+            send = torch.from_numpy(send_h).cuda()
+            want = oracle.alltoall(dims, offs, m, send_h)
+            got.fill_(0x5A)
+            iso.Iso_neighbor_alltoall_static(dims, offs, send, got, m, iso.ISO_BYTE, torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            assert np.array_equal(got.cpu().numpy(), want), "call %d differs from the oracle (dims %s, m %d)" % (call, dims, m)
+            # and the ordinary entry points give the same bytes
+            assert torch.equal(got, _allocating(torch, dims, offs, m, send)), (dims, m, call)
+
+
+def test_static_entry_point_allocates_no_device_memory():
+    """What the entry point exists for: once the device has loaded the library's kernels
+    (first call), a call leaves the amount of free device memory exactly as it found it."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("needs a CUDA device")
+    torch.cuda.set_device(0)
+    dims, offs, m = (8, 8, 8), wl.moore(3, 1), 64
+    P, s = 512, 26
+    send = wl.payload_torch("uint8", 3, 0, P * s * m, "cuda").view(P, s * m)
+    recv = torch.empty((P, s * m), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    iso.Iso_neighbor_alltoall_static(dims, offs, send, recv, m, iso.ISO_BYTE, stream)      # warm-up: kernels get loaded
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        iso.Iso_neighbor_alltoall_static(dims, offs, send, recv, m, iso.ISO_BYTE, stream)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
 
 
 def test_static_entry_point_rejects_what_does_not_fit():
