@@ -2,14 +2,17 @@
 """Benchmark of the isomorphic neighbourhood all-to-all on one B200 (or N independent
 replicas, one per GPU).
 
-A step is one `Iso_Start` of the whole schedule on the workload (default: all-to-all on a
-32x32x32 torus, Moore neighbourhood of radius 1, 64-byte fp32 blocks).  The headline value
-is the effective bandwidth over the bytes the message-combining schedule actually moves
-(read + written), device timed with CUDA events; the same line carries the payload rate,
-the one-pass direct kernel for comparison, the roofline fraction, the end-to-end rate with
-host buffers and the CPU oracle timed on the host cores.
+A step is one `Iso_Start` of the whole schedule on the workload (default: the largest of the
+configurations, all-to-all on a 256x256 torus, Moore neighbourhood of radius 2, 4 KB blocks:
+6.4 GB per buffer).  The headline value is the effective bandwidth over the bytes the
+message-combining schedule moves (read + written), device timed with CUDA events over
+repeated runs of K steps; the same line carries the payload rate, the roofline fraction of
+the dominant kernel with its DRAM traffic, the end-to-end rate with host buffers, the CPU
+oracle timed on the host cores, and a table (`detail.configs`) with every configuration
+under the combining, the direct and the hop-by-hop schedule, each checked against the
+oracle on sampled ranks after it was timed.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--sweep]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--sweep paper]
     python bench.py --impl reference ...      # times the CPU oracle instead
 """
 from __future__ import annotations
@@ -31,12 +34,42 @@ import numpy as np
 
 METRIC = "neighbor-alltoall effective GB/s (device-timed) and % of B200 HBM peak, combining vs direct"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + written) per launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (iso_gather_rows_wide on cfg2_alltoall); only valid for that kernel build
-# and workload, so it is reported for the default workload and schedule only.
-TRAFFIC_BYTES_PER_LAUNCH = {"cfg2_alltoall": 44.56e6}
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 512 << 20
+L2_BYTES = 126 << 20
+HEADLINE = "cfg3_m4096"
+# ncu counters of the dominant kernels (DRAM bytes per launch), each stamped with a hash of
+# the kernel sources it was taken on; an entry whose stamp is not the present sources' is
+# ignored (traffic: null)
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+KERNEL_SOURCES = ("iso_kernels.cuh", "iso_api.cu", "iso_schedule.cpp", "iso_internal.h")
+
+
+def sources_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_1606_07676_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, schedule: str):
+    """DRAM bytes per step of `workload` under `schedule` from the tracked ncu summary, as
+    {"bytes_per_step", "launches", "mode", "scaled_from"}, or None when there is no entry or
+    the kernels have changed since it was captured."""
+    try:
+        lines = open(TRAFFIC_FILE).read().splitlines()
+    except OSError:
+        return None
+    now = sources_hash()
+    for ln in lines:
+        f = ln.split()
+        if len(f) < 7 or f[0].startswith("#"):
+            continue
+        if f[0] == workload and f[1] == schedule and f[6] == now:
+            return {"bytes_per_step": float(f[3]), "launches": int(f[2]), "mode": f[4], "scaled_from": f[5]}
+    return None
 
 
 def measured_peak():
@@ -135,46 +168,154 @@ def max_over_ranks(dist, value: float, device) -> float:
     return float(t.item())
 
 
-# ------------------------------------------------------------------------ reference arm
-def oracle_run(w, send):
-    """One pass of the CPU oracle over the whole workload (only the CPU-baseline leg and the
-    reference arm call this)."""
-    import oracle
+# ------------------------------------------------------------ what both arms agree on
+def replica_count(w) -> int:
+    """Independent instances of a workload that the timed steps rotate over, so that an
+    instance's send and receive buffers have left the L2 before it comes round again."""
     from paper_1606_07676_b200 import workloads as wl
     lens, sd, rd, ss, rs = wl.layout(w)
-    if w.collective == "alltoall":
-        return oracle.alltoall(w.dims, w.offsets, w.block_bytes, send)
-    if w.collective == "allgather":
-        return oracle.allgather(w.dims, w.offsets, w.block_bytes, send)
-    return oracle.alltoallv(w.dims, w.offsets, lens, sd, rd, ss, rs, send)
+    foot = max(1, w.P * (ss + rs))
+    return max(1, min(16, -(-4 * L2_BYTES // foot)))
+
+
+def config_dict(w, fusion: int, n_gpus: int) -> dict:
+    """The `config` object of the JSON line; the same in both arms."""
+    from paper_1606_07676_b200 import workloads as wl
+    lens, sd, rd, ss, rs = wl.layout(w)
+    foot = w.P * (ss + rs)
+    n = replica_count(w)
+    if n == 1:
+        l2 = "inputs larger than L2: %.0f MB of send and receive buffers per step" % (foot / 1e6)
+    else:
+        l2 = ("inputs larger than L2: steps rotate over %d independent instances of the workload "
+              "(%.1f MB of send and receive buffers each)" % (n, foot / 1e6))
+    return {"workload": w.name, "collective": w.collective, "dims": list(w.dims), "s": w.s, "P": w.P,
+            "block_bytes": w.block_bytes or None,
+            "schedule": "combining (Section V), fusion level %d" % fusion,
+            "parallelism": "replicas only" if n_gpus > 1 else "single GPU",
+            "l2": l2,
+            "bytes": "value = bytes the message-combining schedule reads + writes (2 x P x sum_i m_i x hops_i) / time, "
+                     "the same byte count in both arms; payload = one read + one write of every delivered block"}
+
+
+# ------------------------------------------------------------------------ the CPU oracle
+class OracleSample:
+    """A bounded sample of a workload for the CPU oracle: the receive buffers of the ranks of
+    the first planes of dimension 0 (the whole workload when that is small).  The host send
+    buffer is reserved in full, but only the planes those ranks read from are generated, so a
+    6 GB workload costs a few hundred MB of host memory.  Only the CPU-baseline leg and the
+    reference arm use this."""
+
+    def __init__(self, w, max_out_bytes=192 << 20):
+        from paper_1606_07676_b200 import workloads as wl
+        self.w = w
+        self.lens, self.sd, self.rd, self.ss, self.rs = wl.layout(w)
+        P, p0 = w.P, w.dims[0]
+        plane = P // p0
+        planes = max(1, min(p0, max_out_bytes // max(1, plane * self.rs)))
+        if planes >= p0 or P * self.ss <= (512 << 20):
+            self.r0, self.r1 = 0, P
+            self.send = wl.send_buffer_np(w, self.ss)
+            self.what = "the whole workload (%d processes x %d blocks)" % (P, w.s)
+        else:
+            self.r0, self.r1 = 0, planes * plane
+            need = sorted({(x - int(c0)) % p0 for x in range(planes) for c0 in list(w.offsets[:, 0]) + [0]})
+            self.send = np.empty((P, self.ss), dtype=np.uint8)
+            for x in need:
+                self.send[x * plane:(x + 1) * plane] = wl.payload_np(
+                    w.kind, w.seed, 0, x * plane * self.ss, plane * self.ss).reshape(plane, self.ss)
+            self.what = ("the receive buffers of %d of %d processes (planes 0..%d of dimension 0; %d source planes "
+                         "generated)" % (self.r1, P, planes - 1, len(need)))
+        self.ranks = self.r1 - self.r0
+        self.bytes_min = 2 * self.ranks * int(self.lens.sum())
+
+    def nominal_moved(self) -> int:
+        """Bytes the message-combining schedule moves for the sampled ranks, by the paper's
+        count (Section V: a block hops once per non-zero coordinate)."""
+        from oracle import counters
+        w = self.w
+        if w.collective == "allgather":
+            zeros = sum(1 for v in counters.residues(w.offsets, w.dims) if not any(v))
+            parts = counters.allgather_direct_volume(w.offsets, w.d, w.dims) + zeros
+            return 2 * self.ranks * w.block_bytes * parts
+        hops = counters.direct_hops(w.offsets, w.d, w.dims)
+        return 2 * self.ranks * sum(int(n) * max(h, 1) for n, h in zip(self.lens, hops))
+
+    def run(self, lo=None, hi=None):
+        import oracle
+        w = self.w
+        lo = self.r0 if lo is None else lo
+        hi = self.r1 if hi is None else hi
+        if w.collective == "alltoall":
+            return oracle.alltoall(w.dims, w.offsets, w.block_bytes, self.send, lo, hi)
+        if w.collective == "allgather":
+            return oracle.allgather(w.dims, w.offsets, w.block_bytes, self.send, lo, hi)
+        return oracle.alltoallv(w.dims, w.offsets, self.lens, self.sd, self.rd, self.ss, self.rs, self.send, lo, hi)
+
+
+def cpu_baseline(w, seconds=10.0):
+    """The oracle, as it stands, on this host: repeated passes over a bounded sample of the
+    workload; GB/s over one read + one write of every delivered block."""
+    sample = OracleSample(w)
+    sample.run()
+    times = []
+    t_end = time.perf_counter() + seconds
+    while len(times) < 3 or (time.perf_counter() < t_end and len(times) < 50):
+        t0 = time.perf_counter()
+        sample.run()
+        times.append(time.perf_counter() - t0)
+    dt = statistics.median(times)
+    out = {"value": sample.bytes_min / dt / 1e9, "unit": "GB/s (payload: one read + one write of every delivered block)",
+           "cores": 1, "kind": "oracle", "sample": "%s, median of %d passes" % (sample.what, len(times)),
+           "ms_per_pass": dt * 1e3, "ms_whole_workload_extrapolated": dt * 1e3 * w.P / sample.ranks}
+    # The same oracle over all host cores: the sampled ranks are cut into one contiguous range
+    # per thread (the C call releases the interpreter lock).
+    cores = len(os.sched_getaffinity(0))
+    if cores > 1:
+        from concurrent.futures import ThreadPoolExecutor
+        cuts = [sample.r0 + sample.ranks * k // cores for k in range(cores + 1)]
+        with ThreadPoolExecutor(cores) as pool:
+            def whole():
+                list(pool.map(lambda k: sample.run(cuts[k], cuts[k + 1]), range(cores)))
+            whole()
+            par = []
+            t_end = time.perf_counter() + seconds / 2
+            while len(par) < 3 or (time.perf_counter() < t_end and len(par) < 50):
+                t0 = time.perf_counter()
+                whole()
+                par.append(time.perf_counter() - t0)
+        pdt = statistics.median(par)
+        out["all_cores"] = {"value": sample.bytes_min / pdt / 1e9, "unit": "GB/s", "cores": cores, "ms_per_pass": pdt * 1e3,
+                            "sample": "same sample, one contiguous rank range per thread, median of %d passes" % len(par)}
+    return out
 
 
 def run_reference(args):
-    """Times the CPU oracle, as it stands, on the same workload and metric."""
+    """Times the CPU oracle, as it stands, on a bounded sample of the same workload, in the
+    same unit and over the same byte count as the GPU arm."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
     from paper_1606_07676_b200 import workloads as wl
 
     w = wl.config(args.workload)
-    lens, sd, rd, ss, rs = wl.layout(w)
-    send = wl.send_buffer_np(w, ss)
-    bytes_min = 2 * w.P * int(lens.sum())
+    sample = OracleSample(w)
     for _ in range(max(1, args.warmup)):
-        oracle_run(w, send)
+        sample.run()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle_run(w, send)
+        sample.run()
     dt = (time.perf_counter() - t0) / args.steps
-    value = bytes_min / dt / 1e9
+    value = sample.nominal_moved() / dt / 1e9
+    what = "%s per step, %d steps, one host thread" % (sample.what, args.steps)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": args.workload, "P": w.P, "s": w.s, "note": "CPU oracle (direct definition), "
-                   "one host thread, whole workload per step; bytes = one read + one write of every block"},
-        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle",
-                         "sample": "the whole workload, %d steps" % args.steps},
+        "config": config_dict(w, args.fusion, args.gpus),
+        "payload": {"gbs": sample.bytes_min / dt / 1e9},
+        "ms_whole_workload_extrapolated": dt * 1e3 * w.P / sample.ranks,
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": what},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -273,7 +414,7 @@ def time_steps(torch, fn, steps, warmup, flush):
 
 def time_run(torch, fn, steps, warmup):
     """Device time (ms) per step of `steps` back-to-back calls fn(0..steps-1), one CUDA event
-    pair around the whole run on the current stream."""
+    pair around the whole run on the current stream (the stream the kernels are launched on)."""
     for k in range(warmup):
         fn(k)
     torch.cuda.synchronize()
@@ -286,19 +427,38 @@ def time_run(torch, fn, steps, warmup):
     return a.elapsed_time(b) / steps
 
 
+def time_repeats(torch, fn, steps, warmup, dist=None, min_total_ms=500.0, max_repeats=400):
+    """Runs of exactly `steps` back-to-back steps, each between a synchronisation (and a
+    barrier over the ranks) and one CUDA event pair, repeated until at least `min_total_ms`
+    of device time has been timed.  Returns the per-step times (ms) of the runs; with several
+    ranks every entry is the slowest rank's."""
+    first = max_over_ranks(dist, time_run(torch, fn, steps, warmup), "cuda")      # calibration, not reported
+    repeats = int(max(1, min(max_repeats, -(-min_total_ms // max(first * steps, 1e-6)))))
+    out = []
+    for _ in range(repeats):
+        if dist is not None:
+            dist.barrier()
+        out.append(max_over_ranks(dist, time_run(torch, fn, steps, 0), "cuda"))
+    return out
+
+
+def spread(times):
+    return {"ms": statistics.median(times), "ms_min": min(times), "ms_max": max(times), "repeats": len(times)}
+
+
 class Replicas:
     """Independent instances of one workload (different seeds, own buffers and requests),
     enough of them that a round-robin over the instances touches far more memory than the
     L2 holds before an instance comes round again."""
 
-    def __init__(self, torch, iso, wl, name, min_bytes=4 * 126 * (1 << 20), max_replicas=16):
+    def __init__(self, torch, iso, wl, name):
         first = Bound(torch, iso, wl, name)
         st = iso.Iso_request_get_stats(first.req)
-        foot = st["P"] * (st["send_stride"] + st["recv_stride"] + st["inter_stride"])
-        n = max(1, min(max_replicas, -(-min_bytes // max(1, foot))))
+        n = replica_count(first.w)
         self.items = [first] + [Bound(torch, iso, wl, name, seed=first.w.seed + 1000 * k) for k in range(1, n)]
-        self.footprint = foot
+        self.footprint = st["P"] * (st["send_stride"] + st["recv_stride"])
         self.iso, self.torch = iso, torch
+        self.k = 0
 
     def set(self, alg, fusion):
         st = self.items[0].set(alg, fusion)
@@ -319,68 +479,103 @@ class Replicas:
             b.close()
 
 
-def end_to_end(torch, iso, b, moved, minimum, args, dist, world):
+def parity_check(torch, b, n_random=40):
+    """The receive buffers of sampled ranks of instance `b`, as its last start left them,
+    against the CPU oracle: the oracle names the source process of every block and the
+    block's bytes are regenerated on the host.  Outside every timed region."""
+    import oracle
+    from paper_1606_07676_b200 import workloads as wl
+    w = b.w
+    torch.cuda.synchronize()
+    P, last = w.P, w.dims[-1]
+    plane = P // w.dims[0]
+    rng = np.random.default_rng(2016)
+    ranks = sorted({0, 1, last - 1, last % P, plane - 1, plane % P, P - plane, P - last, P - 1,
+                    *rng.integers(0, P, n_random).tolist()})
+    for r in ranks:
+        got = b.recv[r * b.rs:(r + 1) * b.rs].cpu().numpy()
+        for i in range(w.s):
+            n = int(b.lens[i])
+            q = oracle.source_rank(w.dims, r, w.offsets[i])
+            want = wl.payload_np(w.kind, w.seed, 0, q * b.ss + int(b.sd[i]), n)
+            if not np.array_equal(got[int(b.rd[i]):int(b.rd[i]) + n], want):
+                return False
+    return True
+
+
+def end_to_end(torch, iso, b, moved, minimum, steps, dist, world):
     """The same step through Iso_Start_host: pinned host buffers in and out, copies inside the
     timed region; with several ranks the slowest one counts and the rate is the aggregate."""
-    hs = torch.empty(b.w.P * b.ss, dtype=torch.uint8).pin_memory()
-    hs.copy_(b.send.cpu())
-    hr = torch.empty(b.w.P * b.rs, dtype=torch.uint8).pin_memory()
+    hs = torch.empty(b.w.P * b.ss, dtype=torch.uint8, pin_memory=True)
+    hs.copy_(b.send)
+    hr = torch.empty(b.w.P * b.rs, dtype=torch.uint8, pin_memory=True)
     stream = torch.cuda.current_stream()
 
     def start_host(k):
         iso.Iso_Start_host(b.req, hs, hr, stream)
 
-    e2e_steps = max(3, min(args.steps, 20))
     if dist is not None:
         dist.barrier()
-    me = time_run(torch, start_host, e2e_steps, 3)
+    me = time_run(torch, start_host, steps, 2)
     me = max_over_ranks(dist, me, "cuda")
-    return {"value": world * moved / (me * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": me,
-            "h2d_bytes_per_step": world * int(hs.numel()), "d2h_bytes_per_step": world * int(hr.numel()),
-            "payload_gbs": world * minimum / (me * 1e-3) / 1e9}
+    # the result that travelled back, against the device's own receive buffers
+    same = bool(torch.equal(hr, b.recv.cpu()))
+    try:
+        link = iso.Iso_request_get_host_transfer_ms(b.req)    # of the last step: first copy begins .. last copy ends
+    except iso.IsoError:
+        link = None
+    del hs, hr
+    return {"link_busy": link,"value": world * moved / (me * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": me, "steps": steps,
+            "h2d_bytes_per_step": world * int(b.w.P * b.ss), "d2h_bytes_per_step": world * int(b.w.P * b.rs),
+            "payload_gbs": world * minimum / (me * 1e-3) / 1e9,
+            "link_gbs_per_direction": b.w.P * b.ss / (me * 1e-3) / 1e9,
+            "host_result_equals_device_result": same}
 
 
-def cpu_baseline(w, seconds=10.0):
-    """The oracle, as it stands, on this host: repeated runs of the whole workload for a
-    bounded time; returns GB/s over one read + one write of every delivered block."""
-    from paper_1606_07676_b200 import workloads as wl
-    lens, sd, rd, ss, rs = wl.layout(w)
-    send = wl.send_buffer_np(w, ss)
-    bytes_min = 2 * w.P * int(lens.sum())
-    oracle_run(w, send)
-    times = []
-    t_end = time.perf_counter() + seconds
-    while len(times) < 3 or (time.perf_counter() < t_end and len(times) < 50):
-        t0 = time.perf_counter()
-        oracle_run(w, send)
-        times.append(time.perf_counter() - t0)
-    dt = statistics.median(times)
-    out = {"value": bytes_min / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
-           "sample": "the whole workload (%d processes x %d blocks), median of %d runs" % (w.P, w.s, len(times)),
-           "ms": dt * 1e3}
-    # The same oracle over all host cores: the destination ranks are cut into one contiguous
-    # range per thread (the C call releases the interpreter lock); regular collectives only.
-    cores = len(os.sched_getaffinity(0))
-    if cores > 1 and w.collective in ("alltoall", "allgather"):
-        import oracle
-        from concurrent.futures import ThreadPoolExecutor
-        fn = oracle.alltoall if w.collective == "alltoall" else oracle.allgather
-        cuts = [w.P * k // cores for k in range(cores + 1)]
-        with ThreadPoolExecutor(cores) as pool:
-            def whole():
-                list(pool.map(lambda k: fn(w.dims, w.offsets, w.block_bytes, send, cuts[k], cuts[k + 1]),
-                              range(cores)))
-            whole()
-            par = []
-            t_end = time.perf_counter() + seconds / 2
-            while len(par) < 3 or (time.perf_counter() < t_end and len(par) < 50):
-                t0 = time.perf_counter()
-                whole()
-                par.append(time.perf_counter() - t0)
-        pdt = statistics.median(par)
-        out["all_cores"] = {"value": bytes_min / pdt / 1e9, "unit": "GB/s", "cores": cores, "ms": pdt * 1e3,
-                            "sample": "same workload, one contiguous rank range per thread, median of %d runs"
-                                      % len(par)}
+SCHEDULES = (("combining", "ISO_ALG_COMBINING", 1), ("direct", "ISO_ALG_DIRECT", 1), ("torus", "ISO_ALG_TORUS", 1))
+
+
+def row(st, times, peak, ok):
+    ms = statistics.median(times)
+    moved, minimum = st["bytes_moved"], st["bytes_min"]
+    return dict(spread(times), rounds=st["rounds"], launches=st["launches"], bytes_moved=moved, bytes_min=minimum,
+                gbs_moved=moved / ms / 1e6, gbs_payload=minimum / ms / 1e6,
+                frac_of_measured=moved / ms / 1e6 / peak, frac_of_nominal_8TBs=moved / ms / 1e6 / NOMINAL_HBM_GBS,
+                payload_frac_of_measured=minimum / ms / 1e6 / peak, parity_checked=ok)
+
+
+def steps_for(est_ms, floor_steps):
+    """Steps per timed run of a table row: at least `floor_steps`, and enough that a run
+    lasts about 20 ms."""
+    return int(max(floor_steps, min(20000, -(-20.0 // max(est_ms, 1e-4)))))
+
+
+def config_table(torch, iso, wl, peak, args, names, have=None):
+    """Every configuration under the combining schedule (one launch per dimension), the
+    one-pass direct schedule and the hop-by-hop schedule of Algorithm 1, each timed as
+    repeated runs until `--detail-ms` of device time and then checked against the oracle.
+    `have` holds rows measured elsewhere (the headline workload)."""
+    out = dict(have or {})
+    for name in names:
+        if name in out:
+            continue
+        reps = Replicas(torch, iso, wl, name)
+        rows = {}
+        for key, alg_name, fusion in SCHEDULES:
+            if key == "torus" and reps.items[0].w.collective == "allgather":
+                rows[key] = None        # Algorithm 1 is an all-to-all schedule
+                continue
+            st = reps.set(getattr(iso, alg_name), fusion)
+            est = time_run(torch, reps.start, 8, 3)
+            k = steps_for(est, args.steps)
+            times = time_repeats(torch, reps.start, k, 0, None, args.detail_ms)
+            ok = all(parity_check(torch, b, 12) for b in reps.items[:2])
+            rows[key] = dict(row(st, times, peak, ok), steps_per_run=k, replicas=len(reps.items),
+                             execution=reps.execution())
+        out[name] = rows
+        reps.close()
+        del reps
+        torch.cuda.empty_cache()
     return out
 
 
@@ -401,47 +596,38 @@ def run_ours(args):
     Bound.pipeline = args.pipeline
     reps = Replicas(torch, iso, wl, args.workload)
     b = reps.items[0]
+    alg = {"combining": iso.ISO_ALG_COMBINING, "direct": iso.ISO_ALG_DIRECT, "torus": iso.ISO_ALG_TORUS}[args.alg]
 
     # ---- headline: message-combining schedule, one launch per dimension ----------------
-    st = reps.set(iso.ISO_ALG_COMBINING, args.fusion)
+    st = reps.set(alg, args.fusion)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(local) if rank == 0 else None
     t0 = time.time()
-    ms = time_run(torch, reps.start, args.steps, args.warmup)
+    if args.headline_only:
+        times = [max_over_ranks(dist, time_run(torch, reps.start, args.steps, args.warmup), "cuda")]
+    else:
+        times = time_repeats(torch, reps.start, args.steps, args.warmup, dist, args.min_ms)
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
-    t1 = time.time()
-    clocks = None
-    if sampler is not None and (world > 1 or args.headline_only):
-        clocks = sampler.stop(t0, t1)
-        sampler = None
-    ms = max_over_ranks(dist, ms, "cuda")
+    ms = statistics.median(times)
     moved, minimum = st["bytes_moved"], st["bytes_min"]
     value = world * moved / (ms * 1e-3) / 1e9
     per_gpu = moved / (ms * 1e-3) / 1e9
-
-    detail = {"combining": {"fusion_level": args.fusion, "rounds": st["rounds"], "launches": st["launches"],
-                            "execution": dict(reps.execution(), tuned=bool(args.tune)),
-                            "bytes_moved": moved, "bytes_min": minimum, "ms": ms, "gbs_moved": per_gpu,
-                            "gbs_payload": minimum / (ms * 1e-3) / 1e9, "replicas": len(reps.items),
-                            "footprint_bytes_per_replica": reps.footprint}}
+    launches = iso.Iso_request_get_stats(b.req)["launches"]
+    # the output of the timed request, as the last timed step left it, against the oracle
+    parity = all(parity_check(torch, x) for x in reps.items[:2]) if not args.headline_only else None
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_min": min(times), "ms_per_step_max": max(times),
+        "repeats": len(times), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": args.workload, "collective": b.w.collective, "dims": list(b.w.dims), "s": b.w.s,
-                   "P": b.w.P, "block_bytes": b.w.block_bytes or None,
-                   "schedule": "combining (Section V), fusion level %d" % args.fusion,
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": "inputs larger than L2: steps rotate over %d independent instances of the workload "
-                         "(%.0f MB each, %.0f MB in all), timed back to back between one event pair"
-                         % (len(reps.items), reps.footprint / 1e6, reps.footprint * len(reps.items) / 1e6),
-                   "bytes": "value = bytes read + written by the schedule / device time"},
-        "gpu_launches": iso.Iso_request_get_stats(b.req)["launches"] * args.steps,
+        "config": config_dict(b.w, args.fusion, world),
+        "gpu_launches": launches * args.steps * len(times),
+        "parity_checked": parity,
         "frac_of_nominal_8TBs": per_gpu / NOMINAL_HBM_GBS,
         "frac_of_measured": per_gpu / peak,
         # the same time over the minimum one-read-one-write payload instead of the bytes moved
@@ -449,63 +635,119 @@ def run_ours(args):
                     "frac_of_measured": minimum / (ms * 1e-3) / 1e9 / peak,
                     "frac_of_nominal_8TBs": minimum / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
     }
+    if args.alg != "combining":
+        line["config"]["schedule"] = args.alg
 
-    if rank == 0 and world == 1 and args.headline_only:
-        line["e2e"] = None
-        line["roofline"] = {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s",
-                            "frac": per_gpu / peak, "traffic": args.traffic, "peak_kind": "%s copy bandwidth" % peak_kind}
-    elif rank == 0 and world == 1:
-        flush = Flush(torch)
-        one = lambda k: reps.start(0)
-        # the same schedule on ONE instance: per-step events with an L2 flush in between
-        # (includes the event and launch latency of a lone step), and back to back (warm)
-        cold = time_steps(torch, one, min(args.steps, 50), 3, flush)
-        detail["combining"]["ms_single_flushed_median"] = tukey_median(cold)
-        detail["combining"]["ms_single_warm"] = time_run(torch, one, args.steps, 3)
-        # per-round launches (the paper's schedule, one launch per round) and the direct kernel
-        for key, alg, fusion in (("combining_per_round", iso.ISO_ALG_COMBINING, 0), ("direct", iso.ISO_ALG_DIRECT, 1)):
-            s2 = reps.set(alg, fusion)
-            m2 = time_run(torch, reps.start, args.steps, args.warmup)
-            detail[key] = {"launches": s2["launches"], "bytes_moved": s2["bytes_moved"], "ms": m2,
-                           "gbs_moved": s2["bytes_moved"] / (m2 * 1e-3) / 1e9,
-                           "gbs_payload": s2["bytes_min"] / (m2 * 1e-3) / 1e9,
-                           "frac_of_peak_moved": s2["bytes_moved"] / (m2 * 1e-3) / 1e9 / peak}
-        st = reps.set(iso.ISO_ALG_COMBINING, args.fusion)
-        # clocks were sampled over all device-timed legs above (the headline leg alone
-        # lasts only steps x 40 microseconds)
+    # ---- roofline of the dominant kernel ----------------------------------------------
+    kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_rows_wide"
+    rec = recorded_traffic(args.workload, args.alg) if (
+        args.fusion == 1 and not args.single_launch and args.bulk_threshold is None and not args.tune
+        and args.slabs is None and args.pipeline is None) else None
+    roofline = {
+        "bound": "hbm", "kernel": kernel, "achieved": per_gpu, "peak": peak, "unit": "GB/s",
+        "frac": per_gpu / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
+        "frac_note": "rate over the bytes the schedule reads + writes; intermediate blocks that one phase "
+                     "writes and the next reads may be served by L2, dram_frac counts device-memory bytes only",
+        "launches_per_step": launches, "bytes_per_launch": moved // max(1, launches),
+        "avg_launch_ms": ms / max(1, launches),
+        "traffic": None, "dram_frac": None,
+        "note": "achieved = bytes read+written per launch / (step time / launches per step), "
+                "timed live with CUDA events on the launching stream; launch gaps are inside the step time",
+    }
+    if args.traffic is not None:
+        roofline["traffic"] = args.traffic
+        roofline["dram_frac"] = args.traffic * launches / (ms * 1e-3) / 1e9 / peak
+    elif rec is not None:
+        roofline["traffic"] = rec["bytes_per_step"] / max(1, launches)
+        roofline["dram_frac"] = rec["bytes_per_step"] / (ms * 1e-3) / 1e9 / peak
+        roofline["traffic_note"] = ("dram__bytes_read.sum + dram__bytes_write.sum per launch (ncu, %s; %s), from "
+                                    "profiles/dram_traffic.txt, taken on the present kernel sources"
+                                    % (rec["mode"].replace("_", " "), rec["scaled_from"].replace("_", " ")))
+    else:
+        roofline["traffic_note"] = "no ncu capture of the present kernel sources for this workload and schedule"
+    line["roofline"] = roofline
+
+    detail = {"headline": {"fusion_level": args.fusion, "rounds": st["rounds"], "launches": launches,
+                           "execution": dict(reps.execution(), tuned=bool(args.tune)),
+                           "bytes_moved": moved, "bytes_min": minimum, "replicas": len(reps.items),
+                           "footprint_bytes_per_replica": reps.footprint}}
+    clocks = None
+    full = rank == 0 and world == 1 and not args.headline_only
+    if full:
+        # the headline workload under the other schedules, while its buffers are there
+        have = {args.workload: {"combining": dict(row(st, times, peak, parity), steps_per_run=args.steps,
+                                                  replicas=len(reps.items), execution=reps.execution())}}
+        if args.alg == "combining" and not args.no_detail:
+            for key, alg_name, fusion in SCHEDULES[1:]:
+                if key == "torus" and b.w.collective == "allgather":
+                    have[args.workload][key] = None
+                    continue
+                s2 = reps.set(getattr(iso, alg_name), fusion)
+                est = time_run(torch, reps.start, 3, 2)
+                k = steps_for(est, min(args.steps, 20))
+                t2 = time_repeats(torch, reps.start, k, 0, None, args.detail_ms)
+                have[args.workload][key] = dict(row(s2, t2, peak, all(parity_check(torch, x, 12) for x in reps.items[:2])),
+                                                steps_per_run=k, replicas=len(reps.items), execution=reps.execution())
+            st = reps.set(alg, args.fusion)
+        try:
+            line["e2e"] = end_to_end(torch, iso, b, moved, minimum, max(3, min(args.steps, 5 if moved > (1 << 30) else 20)), dist, world)
+        except RuntimeError as err:      # page-locking two host copies of the buffers failed
+            line["e2e"] = None
+            detail["e2e_error"] = str(err)[:200]
+        reps.close()
+        del reps, b
+        torch.cuda.empty_cache()
+        if not args.no_detail:
+            detail["launch_floor_us"] = {
+                "dependent_launches": iso.Iso_measure_launch_floor(torch.cuda.current_stream(), 4000, True),
+                "plain_launches": iso.Iso_measure_launch_floor(torch.cuda.current_stream(), 4000, False),
+                "note": "device time per launch of an empty kernel, back to back on one stream: a phase of a "
+                        "schedule cannot be shorter; cfg1 and cfg3_m4 are bound by it"}
+            names = wl.CONFIG_NAMES if args.workload == HEADLINE else ()
+            detail["configs"] = config_table(torch, iso, wl, peak, args, names, have)
+            for name in ("cfg1", "cfg3_m4"):
+                for key, r_ in (detail["configs"].get(name) or {}).items():
+                    if r_:
+                        r_["launch_floor_ms"] = r_["launches"] * detail["launch_floor_us"]["dependent_launches"] * 1e-3
+            # DRAM traffic of the small configuration whose intermediate blocks stay in L2
+            for name in ("cfg2_alltoall", "cfg3_m64"):
+                rec2 = recorded_traffic(name, "combining")
+                r_ = (detail["configs"].get(name) or {}).get("combining")
+                if rec2 and r_:
+                    r_["dram_bytes_per_step"] = rec2["bytes_per_step"]
+                    r_["dram_frac_of_measured"] = rec2["bytes_per_step"] / r_["ms"] / 1e6 / peak
+                    r_["l2_served_share"] = 1.0 - rec2["bytes_per_step"] / r_["bytes_moved"]
+            # end to end on the small configuration too (54.5 MB each way: latency of the pipeline shows)
+            if "cfg2_alltoall" in detail["configs"] and args.workload != "cfg2_alltoall":
+                small = Bound(torch, iso, wl, "cfg2_alltoall")
+                s2 = small.set(iso.ISO_ALG_COMBINING, 1)
+                detail["configs"]["cfg2_alltoall"]["combining"]["e2e"] = end_to_end(
+                    torch, iso, small, s2["bytes_moved"], s2["bytes_min"], 20, None, 1)
+                small.close()
+                del small
+        else:
+            detail["configs"] = have
         clocks = sampler.stop(t0, time.time())
         sampler = None
-
-        line["e2e"] = end_to_end(torch, iso, b, moved, minimum, args, dist, world)
-
-        # ---- roofline of the dominant kernel ------------------------------------------
-        launches = max(1, st["launches"])
-        kernel = "iso_gather_bulk" if st["bulk_bytes"] * 2 > moved else "iso_gather_rows_wide<16,12>"
-        line["roofline"] = {
-            "bound": "hbm", "kernel": kernel, "achieved": per_gpu, "peak": peak, "unit": "GB/s",
-            "frac": per_gpu / peak, "peak_kind": "%s copy bandwidth" % peak_kind,
-            "bytes_per_launch": moved // launches, "avg_launch_ms": ms / launches,
-            "traffic": args.traffic if args.traffic is not None else (
-                TRAFFIC_BYTES_PER_LAUNCH.get(args.workload) if args.fusion == 1 and not args.single_launch
-                and args.bulk_threshold is None else None),
-            "traffic_note": "DRAM read+write bytes per launch (ncu, caches flushed before each launch); "
-                            "writes still held in L2 when the kernel ends are not in it",
-            "note": "achieved = bytes read+written per launch / (step time / launches per step); "
-                    "launch gaps are inside the step time",
-        }
-        line["cpu_baseline"] = cpu_baseline(b.w, args.cpu_seconds)
-    elif world > 1:
-        # every rank runs its replica through the host-buffer entry point; slowest rank counts
-        e2e = end_to_end(torch, iso, b, moved, minimum, args, dist, world)
-        line["e2e"] = e2e
-        line["roofline"] = {"bound": "hbm", "achieved": per_gpu, "peak": peak, "unit": "GB/s",
-                            "frac": per_gpu / peak, "traffic": None, "peak_kind": "%s copy bandwidth" % peak_kind}
-
-    reps.close()
-    del reps, b
-    torch.cuda.empty_cache()
-    if rank == 0 and world == 1 and args.sweep and not args.headline_only:
-        detail["sweep"] = sweep(torch, iso, wl, peak, args)
+        if args.sweep:
+            detail["sweep"] = sweep(torch, iso, wl, peak, args)
+        line["cpu_baseline"] = cpu_baseline(wl.config(args.workload), args.cpu_seconds)
+    else:
+        if sampler is not None:
+            clocks = sampler.stop(t0, time.time())
+            sampler = None
+        if world > 1:
+            # every rank runs its replica through the host-buffer entry point; slowest rank counts
+            try:
+                line["e2e"] = end_to_end(torch, iso, b, moved, minimum, 3, dist, world)
+            except RuntimeError as err:
+                line["e2e"] = None
+                detail["e2e_error"] = str(err)[:200]
+        else:
+            line["e2e"] = None
+        reps.close()
+        del reps, b
+        torch.cuda.empty_cache()
     line["clocks"] = clocks
     line["detail"] = detail
     if rank == 0:
@@ -516,12 +758,13 @@ def run_ours(args):
 
 
 def sweep(torch, iso, wl, peak, args):
-    """Every named workload, combining (one launch per dimension, and per round) and direct:
-    the results table.  Same protocol as the headline (rotation over instances, back to back)."""
+    """The paper's larger neighbourhoods: combining (one launch per dimension, and per round),
+    direct, and the combining schedule after Iso_request_tune.  Same protocol as the table of
+    configurations (rotation over instances, back to back)."""
     out = {}
-    for name in (wl.PAPER_NAMES if args.sweep == "paper" else wl.CONFIG_NAMES):
+    for name in wl.PAPER_NAMES:
         reps = Replicas(torch, iso, wl, name)
-        row = {}
+        rows = {}
         for key, alg, fusion in (("combining", iso.ISO_ALG_COMBINING, 1), ("combining_per_round", iso.ISO_ALG_COMBINING, 0),
                                  ("direct", iso.ISO_ALG_DIRECT, 1), ("combining_tuned", iso.ISO_ALG_COMBINING, 1)):
             # the last row: the same schedule after Iso_request_tune has timed slabs x chains x
@@ -530,16 +773,13 @@ def sweep(torch, iso, wl, peak, args):
             Bound.tune = was or key == "combining_tuned"
             st = reps.set(alg, fusion)
             Bound.tune = was
-            steps = 40 if st["bytes_moved"] < (4 << 30) else 6
-            ms = time_run(torch, reps.start, steps, 4)
-            row[key] = {"rounds": st["rounds"], "launches": st["launches"], "execution": reps.execution(),
-                        "bytes_moved": st["bytes_moved"],
-                        "bytes_min": st["bytes_min"], "bulk_bytes": st["bulk_bytes"], "ms": ms,
-                        "replicas": len(reps.items),
-                        "gbs_moved": st["bytes_moved"] / ms / 1e6, "gbs_payload": st["bytes_min"] / ms / 1e6,
-                        "frac_moved_of_peak": st["bytes_moved"] / ms / 1e6 / peak,
-                        "frac_moved_of_8TBs": st["bytes_moved"] / ms / 1e6 / NOMINAL_HBM_GBS}
-        out[name] = row
+            est = time_run(torch, reps.start, 8, 3)
+            k = steps_for(est, 20)
+            times = time_repeats(torch, reps.start, k, 0, None, args.detail_ms)
+            rows[key] = dict(row(st, times, peak, all(parity_check(torch, b, 8) for b in reps.items[:1])),
+                             steps_per_run=k, replicas=len(reps.items), execution=reps.execution(),
+                             bulk_bytes=st["bulk_bytes"])
+        out[name] = rows
         reps.close()
         del reps
         torch.cuda.empty_cache()
@@ -577,17 +817,22 @@ def run_init_times(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2_alltoall")
+    ap.add_argument("--workload", default=HEADLINE)
+    ap.add_argument("--alg", default="combining", choices=["combining", "direct", "torus"],
+                    help="schedule of the headline run (the table always has all three)")
     ap.add_argument("--fusion", type=int, default=1)
-    ap.add_argument("--sweep", nargs="?", const="configs", default=None, choices=["configs", "paper"],
-                    help="also time every named workload (configs: the five configurations; "
-                         "paper: the paper's larger neighbourhoods)")
+    ap.add_argument("--min-ms", type=float, default=500.0,
+                    help="the K-step run is repeated until this much device time has been timed")
+    ap.add_argument("--detail-ms", type=float, default=500.0, help="the same for every row of the table")
+    ap.add_argument("--sweep", nargs="?", const="paper", default=None, choices=["paper"],
+                    help="also time the paper's larger neighbourhoods")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--headline-only", action="store_true",
-                    help="time the headline schedule only (short runs under a profiler)")
+                    help="one K-step run of the headline schedule and nothing else (short runs under a profiler)")
+    ap.add_argument("--no-detail", action="store_true", help="skip the table of configurations")
     ap.add_argument("--single-launch", action="store_true",
                     help="run all phases in one cooperative launch instead of one launch per phase")
     ap.add_argument("--bulk-threshold", type=int, default=None,
@@ -604,7 +849,12 @@ def main():
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture, if one is current")
     ap.add_argument("--init-times", action="store_true",
                     help="print host-side set-up times on the grid of the paper's Table II and exit")
+    ap.add_argument("--sources-hash", action="store_true",
+                    help="print the stamp of the present kernel sources (for profiles/dram_traffic.txt) and exit")
     args = ap.parse_args()
+    if args.sources_hash:
+        print(sources_hash())
+        return 0
     if args.init_times:
         return run_init_times(args)
     args.warmup = max(args.warmup, 3)

@@ -106,7 +106,9 @@ typedef struct Iso_stats {
     int64_t recv_stride;
     int64_t inter_stride; /* same for the library's intermediate buffer (0: none needed) */
     int64_t bytes_min;    /* 2 * P * sum_i m_i: every delivered block read once, written once */
-    int64_t bytes_moved;  /* bytes read + written by one Iso_Start with this schedule */
+    int64_t bytes_moved;  /* bytes read + written by one Iso_Start with this schedule as it is
+                             lowered (an allgather phase in sender-side form reads a block once for
+                             up to four copies) */
     int64_t bulk_bytes;   /* part of bytes_moved handled by the bulk-copy kernel */
 } Iso_stats;
 
@@ -120,7 +122,9 @@ typedef struct Iso_part {
     int slot;
     int src_buf;          /* ISO_BUF_* */
     int dst_buf;
-    int kernel;           /* 0: vector copy kernel, 1: bulk copy kernel */
+    int kernel;           /* 0: vector copy kernel, 1: bulk copy kernel, 2: vector copy kernel in its
+                             sender-side form (allgather phases: a block is loaded once and stored
+                             to every place it is copied to) */
     int width;            /* bytes per vector unit (vector kernel) */
     int reserved;
     int64_t src_off;
@@ -288,20 +292,41 @@ int Iso_request_set_graph(Iso_request request, int enable);
  * persistent requests, which are set up once and started many times): runs the request
  * with 1, 2, 4, ... slabs, with 1, 2 and 4 chains, with and without graph replay, timing a
  * few starts of each on `cuda_stream` with events, and leaves the request on the fastest
- * combination (a less plain plan has to win by 2 %).  `cold` = 0 times the starts back to
- * back, as in a loop over the same buffers; `cold` != 0 overwrites a scratch buffer of twice
- * the L2 size before every timed start (allocated for the duration of the call), as when
- * other work runs between the starts.  The collective is executed many times meanwhile:
+ * combination (a less plain plan has to win by 2 %).  `flags` is a sum of ISO_TUNE_* values.
+ * Without ISO_TUNE_COLD the starts are timed back to back, as in a loop over the same
+ * buffers; with it a scratch buffer of twice the L2 size is overwritten before every timed
+ * start (allocated for the duration of the call), as when other work runs between the
+ * starts.  With ISO_TUNE_SCHEDULE the schedule is chosen as well: the message-combining
+ * schedule with one and with two dimensions per phase and the direct schedule are all timed,
+ * each under every execution plan, and the request is left on the fastest (on one device
+ * the direct schedule usually wins: it moves the fewest bytes); Iso_request_get_stats then
+ * reports the algorithm and fusion level in use, Iso_request_get_execution the plan.
+ * Without it the request keeps its schedule.  The collective is executed many times meanwhile:
  * the send buffers must hold readable data and the receive buffers are overwritten (with
  * the collective's result).  Blocks the host until done.  Does nothing in single-launch
  * mode.  On error the settings from before the call are restored.
  */
-int Iso_request_tune(Iso_request request, void *cuda_stream, int cold);
+enum { ISO_TUNE_COLD = 1, ISO_TUNE_SCHEDULE = 2 };
+int Iso_request_tune(Iso_request request, void *cuda_stream, int flags);
 
 /* What Iso_Start does at present: slabs (1: none), chains (1: none), graph replay (0/1).
  * Before the first Iso_Start after a change these are the values asked for (slabs 0:
  * automatic); any of the pointers may be NULL. */
 int Iso_request_get_execution(Iso_request request, int *slabs, int *chains, int *graph);
+
+/*
+ * Sender-side form of allgather phases (Section III-B: a block travels once per trie edge).
+ * A phase of the allgather schedules copies one block to several places; run as a gather,
+ * every copy loads the block again.  In sender-side form a thread loads a 16-byte unit of
+ * the block once, from the process that holds it, and stores it to up to four of its
+ * destinations (a block with more copies is loaded once per four).  mode 0: never;
+ * 1 (default): in the phases where it measured faster (no block with more than four copies,
+ * at least 64 MiB written); 2: in every phase that allows it - blocks that are multiples of
+ * 16 bytes and below the bulk threshold, one shifted dimension per phase, periodic, no slab,
+ * chain or one-launch execution asked for.  The result never depends on it;
+ * Iso_request_get_stats counts a block read once per load in bytes_moved.
+ */
+int Iso_request_set_sender_side(Iso_request request, int mode);
 
 /* Parts of at least `bytes` bytes whose addresses and length are multiples of 16 are moved
  * by the bulk-copy kernel (asynchronous bulk copies staged through shared memory), the rest
@@ -339,7 +364,7 @@ int Iso_Start(Iso_request request, void *cuda_stream);
  * above: copies `host_sendbuf` to the request's device send buffer, runs the schedule and
  * copies the device receive buffer to `host_recvbuf`.  When only blocks read from the send
  * buffer move along dimension 0 (true for the combining and direct schedules on periodic
- * tori with at least four planes) the work is pipelined over up to eight slabs of
+ * tori with at least four planes) the work is pipelined over up to 32 slabs of
  * dimension 0: a slab's schedule runs as soon as the slabs it reads from have arrived and
  * its receive buffers travel back while later slabs are still being uploaded (uploads and
  * downloads on two internal streams created by the first such call, kernels on
@@ -348,6 +373,16 @@ int Iso_Start(Iso_request request, void *cuda_stream);
  * memory is page-locked.  Complete after Iso_wait or a synchronisation of `cuda_stream`. */
 int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_recvbuf,
                    void *cuda_stream);
+
+/*
+ * Link-busy times of the last pipelined Iso_Start_host of this request (measurement aid):
+ * milliseconds between the first upload starting and the last one ending, the same for the
+ * downloads, and for the whole call on `cuda_stream`; `slabs` = slabs it was pipelined over.
+ * Any pointer may be NULL.  Waits for the request first.  ISO_ERR_STATE when the last start
+ * was not a pipelined Iso_Start_host.
+ */
+int Iso_request_get_host_transfer_ms(Iso_request request, float *upload_ms, float *download_ms, float *total_ms,
+                                     int *slabs);
 
 /* Local completion (Section VII): blocks until the last start has finished and returns
  * ISO_ERR_TIMEOUT if a kernel gave up a bounded wait, ISO_ERR_CUDA on a CUDA error.

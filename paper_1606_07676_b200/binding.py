@@ -31,7 +31,7 @@ EXPORTS = (
     "Iso_neighborhood_create", "Iso_comm_free", "Iso_comm_set_periodic",
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
     "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_pipeline", "Iso_request_set_chains", "Iso_request_set_graph", "Iso_request_tune", "Iso_request_get_execution", "Iso_request_set_bulk_threshold",
-    "Iso_request_check_guards", "Iso_request_set_wait_limit", "Iso_request_test_skew_arrivals", "Iso_measure_launch_floor",
+    "Iso_request_set_sender_side", "Iso_request_check_guards", "Iso_request_get_host_transfer_ms", "Iso_request_set_wait_limit", "Iso_request_test_skew_arrivals", "Iso_measure_launch_floor",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
     "Iso_neighbor_alltoall_static", "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
@@ -101,7 +101,10 @@ def load_library() -> ctypes.CDLL:
         "Iso_request_tune": [vp, vp, ci],
         "Iso_request_get_execution": [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)],
         "Iso_request_set_bulk_threshold": [vp, i64],
+        "Iso_request_set_sender_side": [vp, ci],
         "Iso_request_check_guards": [vp, ctypes.POINTER(i64)],
+        "Iso_request_get_host_transfer_ms": [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                             ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ci)],
         "Iso_request_set_wait_limit": [vp, ctypes.c_uint],
         "Iso_request_test_skew_arrivals": [vp, ci],
         "Iso_measure_launch_floor": [vp, ci, ci, ctypes.POINTER(ctypes.c_float)],
@@ -265,9 +268,14 @@ def Iso_request_set_graph(request: int, enable: bool) -> None:
     _check(load_library().Iso_request_set_graph(request, 1 if enable else 0), "Iso_request_set_graph")
 
 
-def Iso_request_tune(request: int, cuda_stream=None, cold: bool = False) -> dict:
-    """Times the execution variants on the device and keeps the fastest; returns it."""
-    _check(load_library().Iso_request_tune(request, _stream(cuda_stream), 1 if cold else 0), "Iso_request_tune")
+ISO_TUNE_COLD, ISO_TUNE_SCHEDULE = 1, 2
+
+
+def Iso_request_tune(request: int, cuda_stream=None, cold: bool = False, schedule: bool = False) -> dict:
+    """Times the execution variants (and, with `schedule`, the schedules) on the device and
+    keeps the fastest; returns the execution plan."""
+    flags = (ISO_TUNE_COLD if cold else 0) | (ISO_TUNE_SCHEDULE if schedule else 0)
+    _check(load_library().Iso_request_tune(request, _stream(cuda_stream), flags), "Iso_request_tune")
     return Iso_request_get_execution(request)
 
 
@@ -280,6 +288,19 @@ def Iso_request_get_execution(request: int) -> dict:
 
 def Iso_request_set_bulk_threshold(request: int, nbytes: int) -> None:
     _check(load_library().Iso_request_set_bulk_threshold(request, nbytes), "Iso_request_set_bulk_threshold")
+
+
+def Iso_request_get_host_transfer_ms(request: int) -> dict:
+    """Link-busy times of the last pipelined Iso_Start_host (milliseconds) and its slab count."""
+    up, down, total, slabs = ctypes.c_float(0), ctypes.c_float(0), ctypes.c_float(0), ctypes.c_int(0)
+    _check(load_library().Iso_request_get_host_transfer_ms(request, ctypes.byref(up), ctypes.byref(down),
+                                                           ctypes.byref(total), ctypes.byref(slabs)),
+           "Iso_request_get_host_transfer_ms")
+    return {"upload_ms": up.value, "download_ms": down.value, "total_ms": total.value, "slabs": slabs.value}
+
+
+def Iso_request_set_sender_side(request: int, mode: int) -> None:
+    _check(load_library().Iso_request_set_sender_side(request, mode), "Iso_request_set_sender_side")
 
 
 def Iso_request_check_guards(request: int) -> int:

@@ -40,6 +40,11 @@ void release_device(Request &r)
 {
     if (r.graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.graph_exec));
     r.graph_exec = nullptr;
+    if (r.host_graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.host_graph_exec));
+    r.host_graph_exec = nullptr;
+    r.host_last_hs = r.host_last_hr = nullptr;
+    if (r.host_main_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.host_main_stream));
+    r.host_main_stream = nullptr;
     if (r.d_blob) cudaFree(r.d_blob);
     if (r.d_inter_alloc) cudaFree(r.d_inter_alloc);
     r.d_inter_alloc = nullptr;
@@ -48,6 +53,9 @@ void release_device(Request &r)
     if (r.up_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.up_stream));
     r.up_stream = nullptr;
     for (void *e : r.slab_events) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+    for (void *e : r.host_timing) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+    r.host_timing.clear();
+    r.host_timed = false;
     r.copy_stream = nullptr;
     r.slab_events.clear();
     if (r.d_counter) cudaFree(r.d_counter);
@@ -126,6 +134,7 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
     comm->refcount++;
     r->kind = kind;
     r->knobs = read_knobs();
+    if (r->knobs.sender_side >= 0 && r->knobs.sender_side <= 2) r->sender_side = r->knobs.sender_side;
     r->send = static_cast<const unsigned char *>(sendbuf);
     r->recv = static_cast<unsigned char *>(recvbuf);
     r->s = comm->s;
@@ -187,6 +196,29 @@ void fill_units(const Request &r, const LaunchPlan &L, UnitDev *ud)
     std::copy(units.begin(), units.end(), ud);
 }
 
+// Descriptors of a sender-side launch: one per 16-byte unit of every parent block.
+void fill_fans(const Request &r, const LaunchPlan &L, FanDev *fd)
+{
+    const Comm &c = *r.comm;
+    const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
+    const int64_t rank_stride = L.n_used ? c.rank_stride[L.used_dim[0]] : 0;
+    size_t at = 0;
+    for (const FanParent &f : L.fans) {
+        FanDev d{};
+        d.src_buf = (uint8_t)f.src_buf;
+        d.n_dst = (uint8_t)f.dsts.size();
+        for (int64_t k = 0; k < f.len / 16; ++k) {
+            d.src_term = f.src_off + 16 * k;
+            for (size_t e = 0; e < f.dsts.size(); ++e) {
+                d.dst_buf[e] = (uint8_t)f.dsts[e].buf;
+                d.c[e] = f.dsts[e].c;
+                d.dst_term[e] = f.dsts[e].off + 16 * k + (int64_t)f.dsts[e].c * rank_stride * stride[f.dsts[e].buf];
+            }
+            fd[at++] = d;
+        }
+    }
+}
+
 // Uploads the lowered schedule and allocates the intermediate buffer.
 int materialise(Request &r)
 {
@@ -194,12 +226,16 @@ int materialise(Request &r)
     // a captured graph holds the addresses of the tables and buffers that are replaced below
     if (r.graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.graph_exec));
     r.graph_exec = nullptr;
+    if (r.host_graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.host_graph_exec));
+    r.host_graph_exec = nullptr;
+    r.host_last_hs = r.host_last_hr = nullptr;
     // grids are sized for the device that runs them (the host-only lowering at init assumed a B200)
     int device = 0, sms = 0;
     ISO_CUDA(cudaGetDevice(&device));
     ISO_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    if (sms > 0 && sms != r.sm_count) {
-        r.sm_count = sms;
+    if (sms > 0) r.sm_count = sms;
+    {
+        // lowered afresh with the request's present settings: the slab plan below reads it
         int rc0 = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
         if (rc0 != ISO_SUCCESS) return rc0;
     }
@@ -248,6 +284,7 @@ int materialise(Request &r)
         bytes += (L.lookup.size() * sizeof(uint16_t) + 15) / 16 * 16;
         L.units_off = bytes;
         if (L.kernel == KERNEL_VEC) bytes += (size_t)L.units_per_proc * sizeof(UnitDev);
+        if (L.kernel == KERNEL_FAN) bytes += (size_t)L.units_per_proc * sizeof(FanDev);
     }
     // one-launch execution: every launch is a 16-byte vector launch on periodic dimensions
     bool single = r.persistent && !r.wave_ok && r.launches.size() >= 2;
@@ -302,6 +339,7 @@ int materialise(Request &r)
         if (!L.lookup.empty())
             std::memcpy(blob.data() + L.lookup_off, L.lookup.data(), L.lookup.size() * sizeof(uint16_t));
         if (L.kernel == KERNEL_VEC) fill_units(r, L, reinterpret_cast<UnitDev *>(blob.data() + L.units_off));
+        if (L.kernel == KERNEL_FAN) fill_fans(r, L, reinterpret_cast<FanDev *>(blob.data() + L.units_off));
     }
     if (r.d_blob) cudaFree(r.d_blob);
     r.d_blob = nullptr;
@@ -497,13 +535,18 @@ unsigned grid_for_rows(const LaunchPlan &L, const LaunchDev &a, int share = 1)
     return (unsigned)g;
 }
 
+constexpr int kMaxDynamicSmem = 227 * 1024;  // dynamic shared memory a CTA can opt in to on sm_100
+
+// Shared memory of a wide launch that keeps a coordinate table behind the cp.async ring.
+size_t table_bytes(const LaunchDev &a) { return (size_t)a.tab_iters * a.rows_per_pass * a.tab_stride * sizeof(uint32_t); }
+
 template <typename Kernel>
 cudaError_t launch_kernel(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, cudaStream_t stream, bool dependent)
 {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(grid_for_rows(L, a, a.grid_share));
     cfg.blockDim = dim3((unsigned)L.threads);
-    cfg.dynamicSmemBytes = L.smem;
+    cfg.dynamicSmemBytes = L.smem + table_bytes(a);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     // programmatic dependent launch: the kernel may start while its predecessor in the stream
@@ -529,12 +572,23 @@ cudaError_t launch_wide(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, 
     {
         std::lock_guard<std::mutex> lock(guard);
         if (std::find(opted_in.begin(), opted_in.end(), key) == opted_in.end()) {
-            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWideDepth * 1024 * 16);
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
             if (e != cudaSuccess) return e;
             opted_in.push_back(key);
         }
     }
     return launch_kernel(kernel, L, a, stream, dependent);
+}
+
+// The wide vector kernel with or without the coordinate table; the table variants exist for
+// the cases launch_one uses them in.
+template <int W, int NU, bool MESH, bool COMPACT>
+cudaError_t launch_rows_wide(bool tab, const LaunchPlan &L, const LaunchDev &a, cudaStream_t stream, bool dependent)
+{
+    if constexpr (!MESH && (COMPACT || NU <= 2)) {
+        if (tab) return launch_wide(iso_gather_rows_wide<W, kWideDepth, NU, MESH, COMPACT, true>, L, a, stream, dependent);
+    }
+    return launch_wide(iso_gather_rows_wide<W, kWideDepth, NU, MESH, COMPACT, false>, L, a, stream, dependent);
 }
 
 int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool dependent, long long row_lo = 0,
@@ -554,6 +608,8 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
     cudaError_t e;
     if (L.kernel == KERNEL_BULK) {
         e = launch_kernel(iso_gather_bulk, L, a, stream, dependent);
+    } else if (L.kernel == KERNEL_FAN) {
+        e = launch_wide(iso_fan_rows<kWideDepth>, L, a, stream, dependent);
     } else if (L.width > 0 && L.width < 4) {
         e = L.width == 2 ? launch_kernel(iso_gather_rows_reg<2, 4>, L, a, stream, dependent)
                          : launch_kernel(iso_gather_rows_reg<1, 4>, L, a, stream, dependent);
@@ -562,9 +618,24 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
         // (with compact unit descriptors: on the dimensions one unit is shifted along)
         const int count = L.compact ? L.max_nnz : L.n_used;
         const int nu = count <= 3 ? count : ISO_MAX_DIMS;
+        // wide CTAs: a table of the coordinates of the rows a CTA visits, if it fits behind the ring
+        bool tab = false;
+        // (measured: +2 to +5 % on the phases of the combining schedules, which shift along one
+        // dimension, and on the compact last phase of 16-byte blocks; the one-pass direct
+        // schedules, three or more wrap tests per row, are bound by the latency of their
+        // scattered loads and gain nothing, so they keep the divisions)
+        if ((L.width == 16 || L.width == 0) && L.threads > 256 && L.n_used > 0 && r.knobs.coord_table &&
+            (L.compact || nu <= 2) && !a.mesh_mask) {
+            const long long groups = (a.row_hi - a.row_lo + L.rows_per_pass - 1) / L.rows_per_pass;
+            const long long grid = grid_for_rows(L, a, a.grid_share);
+            a.tab_iters = (uint32_t)((groups + grid - 1) / grid);
+            a.tab_stride = L.n_used <= 4 ? 4 : 8;
+            tab = L.smem + table_bytes(a) <= (size_t)kMaxDynamicSmem;
+            if (!tab) a.tab_iters = 0;
+        }
 #define ISO_ROWS(W, NU, MESH, COMPACT)                                                                          \
     e = ((W == 16 || W == 0) && L.threads > 256)                                                                \
-            ? launch_wide(iso_gather_rows_wide<(W == 0 ? 0 : 16), kWideDepth, NU, MESH, COMPACT>, L, a, stream, dependent) \
+            ? launch_rows_wide<(W == 0 ? 0 : 16), NU, MESH, COMPACT>(tab, L, a, stream, dependent)             \
             : launch_kernel(iso_gather_rows<W, kVecDepth, NU, MESH, COMPACT>, L, a, stream, dependent)
 #define ISO_ROWS_W(W)                                                            \
     do {                                                                         \
@@ -611,13 +682,18 @@ void plan_slabs(const Request &r, std::vector<SlabPlan> &slabs, int want = 0)
     std::vector<int> shifts;  // distinct shifts along dimension 0 (0 included)
     shifts.push_back(0);
     for (const LaunchPlan &L : r.launches)
+        if (L.kernel == KERNEL_FAN) return;  // a sender-side launch writes outside the rows it is given
+    for (const LaunchPlan &L : r.launches)
         for (const LoweredPart &lp : L.parts) {
             const int s0 = lp.p.shift[0];
             if (s0 == 0) continue;
             if (lp.p.src_buf != ISO_BUF_SEND) return;
             if (std::find(shifts.begin(), shifts.end(), s0) == shifts.end()) shifts.push_back(s0);
         }
-    int n = std::min(p0, 8);
+    // default: up to 32 slabs.  The last slabs to arrive (a slab and the neighbours it reads
+    // from) can only run and travel back after the final upload, so the tail of the pipeline
+    // is about three slabs long: a quarter of the transfer time with 8 slabs, a tenth with 32.
+    int n = std::min(p0, 32);
     if (want > 0) {
         n = std::min(p0, want);
     } else if (r.knobs.host_slabs >= 0) {
@@ -638,6 +714,117 @@ void plan_slabs(const Request &r, std::vector<SlabPlan> &slabs, int want = 0)
             slabs[slab_of[x]].last_needed = std::max(slabs[slab_of[x]].last_needed, slab_of[src]);
             if (slab_of[src] < 64) slabs[slab_of[x]].needs |= 1ULL << slab_of[src];
         }
+}
+
+// Whether `p` is page-locked host memory (only such copies are recorded into a graph).
+bool page_locked(const void *p)
+{
+    cudaPointerAttributes at{};
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    return at.type == cudaMemoryTypeHost;
+}
+
+// Streams and events of the pipelined host-buffer path.
+int prepare_host_pipeline(Request &r, size_t S)
+{
+    if (!r.copy_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.copy_stream), cudaStreamNonBlocking));
+    if (!r.up_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.up_stream), cudaStreamNonBlocking));
+    while (r.slab_events.size() < 2 * S + 2) {
+        cudaEvent_t e;
+        ISO_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        r.slab_events.push_back(e);
+    }
+    // timing events for Iso_request_get_host_transfer_ms: begin and end of the uploads, of the
+    // downloads and of the whole call
+    while (r.host_timing.size() < 6) {
+        cudaEvent_t e;
+        ISO_CUDA(cudaEventCreate(&e));
+        r.host_timing.push_back(e);
+    }
+    return ISO_SUCCESS;
+}
+
+// Enqueues one pipelined host-buffer start.  Only blocks read from the send buffer cross
+// slabs, so a slab's whole schedule can run as soon as the send buffers of the slabs it reads
+// have arrived, and its receive buffers can travel back while later slabs are still on their
+// way in.  Three streams: uploads back to back on one, kernels on `stream`, downloads on a
+// third, so that both directions of the link are busy at the same time and no copy waits
+// behind a kernel.  With `capturing` the calls are being recorded into a graph (`stream` is
+// the capture's origin): the timing events then become external event nodes.
+int enqueue_host_pipeline(Request &r, const std::vector<SlabPlan> &slabs, const unsigned char *hs, unsigned char *hr,
+                          cudaStream_t stream, bool capturing)
+{
+    const Comm &c = *r.comm;
+    const size_t S = slabs.size();
+    cudaStream_t down = static_cast<cudaStream_t>(r.copy_stream), up = static_cast<cudaStream_t>(r.up_stream);
+    auto stamp = [&](void *event, cudaStream_t on) -> cudaError_t {
+        return cudaEventRecordWithFlags(static_cast<cudaEvent_t>(event), on, capturing ? cudaEventRecordExternal : cudaEventRecordDefault);
+    };
+    // copies of this call must not overtake earlier work on the caller's stream
+    cudaEvent_t fence = static_cast<cudaEvent_t>(r.slab_events[2 * S]);
+    ISO_CUDA(cudaEventRecord(fence, stream));
+    ISO_CUDA(cudaStreamWaitEvent(up, fence, 0));
+    ISO_CUDA(cudaStreamWaitEvent(down, fence, 0));
+    ISO_CUDA(stamp(r.host_timing[4], stream));
+    ISO_CUDA(stamp(r.host_timing[0], up));
+    bool first_download = true;
+    const bool use_pdl = !r.knobs.no_pdl;
+    // Upload order: the last slab first, then 0, 1, ...: on a torus slab 0 reads the last slab,
+    // so in natural order it (and its download) would have to wait for the very last upload.
+    std::vector<size_t> order(S), pos(S);
+    for (size_t i = 0; i < S; ++i) order[i] = S <= 64 ? (i + S - 1) % S : i;
+    for (size_t i = 0; i < S; ++i) pos[order[i]] = i;
+    std::vector<size_t> ready_at(S, 0);  // position in the upload order after which a slab can run
+    for (size_t k = 0; k < S; ++k) {
+        if (S <= 64) {
+            for (size_t j = 0; j < S; ++j)
+                if (slabs[k].needs >> j & 1ULL) ready_at[k] = std::max(ready_at[k], pos[j]);
+            ready_at[k] = std::max(ready_at[k], pos[k]);
+        } else {
+            ready_at[k] = (size_t)std::max(slabs[k].last_needed, (int)k);
+        }
+    }
+    std::vector<char> done(S, 0);
+    for (size_t upi = 0; upi < S; ++upi) {
+        const SlabPlan &u = slabs[order[upi]];
+        const size_t off = (size_t)(u.row_lo * r.send_stride), n = (size_t)((u.row_hi - u.row_lo) * r.send_stride);
+        if (n) ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send) + off, hs + off, n, cudaMemcpyHostToDevice, up));
+        cudaEvent_t arrived = static_cast<cudaEvent_t>(r.slab_events[S + upi]);
+        ISO_CUDA(cudaEventRecord(arrived, up));
+        // every slab whose last needed upload this was
+        for (size_t k = 0; k < S; ++k) {
+            if (done[k] || ready_at[k] > upi) continue;
+            const SlabPlan &w = slabs[k];
+            ISO_CUDA(cudaStreamWaitEvent(stream, arrived, 0));
+            for (const LaunchPlan &L : r.launches) {
+                int rc = launch_one(r, L, stream, use_pdl, w.row_lo, w.row_hi, r.inter_rows < c.P ? w.row_lo : 0);
+                if (rc != ISO_SUCCESS) return rc;
+            }
+            cudaEvent_t ev = static_cast<cudaEvent_t>(r.slab_events[k]);
+            ISO_CUDA(cudaEventRecord(ev, stream));
+            ISO_CUDA(cudaStreamWaitEvent(down, ev, 0));
+            if (first_download) ISO_CUDA(stamp(r.host_timing[2], down));
+            first_download = false;
+            const size_t roff = (size_t)(w.row_lo * r.recv_stride), rn = (size_t)((w.row_hi - w.row_lo) * r.recv_stride);
+            if (rn) ISO_CUDA(cudaMemcpyAsync(hr + roff, r.recv + roff, rn, cudaMemcpyDeviceToHost, down));
+            done[k] = 1;
+        }
+    }
+    ISO_CUDA(stamp(r.host_timing[1], up));
+    ISO_CUDA(stamp(r.host_timing[3], down));
+    // join: the caller's stream is complete only when the downloads are
+    ISO_CUDA(cudaEventRecord(fence, down));
+    ISO_CUDA(cudaStreamWaitEvent(stream, fence, 0));
+    // the upload stream ends with its time stamp: join it as well (a capture must end with
+    // every forked stream joined)
+    cudaEvent_t up_done = static_cast<cudaEvent_t>(r.slab_events[2 * S + 1]);
+    ISO_CUDA(cudaEventRecord(up_done, up));
+    ISO_CUDA(cudaStreamWaitEvent(stream, up_done, 0));
+    ISO_CUDA(stamp(r.host_timing[5], stream));
+    return ISO_SUCCESS;
 }
 
 // No exception may cross the C boundary: allocation failures become ISO_ERR_NOMEM.
@@ -718,7 +905,7 @@ void choose_slab_plan(Request &r)
         r.use_graph = true;
         rows *= chains;
     }
-    // the pipelined host-buffer path cuts dimension 0 into up to eight slabs of its own
+    // the pipelined host-buffer path cuts dimension 0 into slabs of its own (plan_slabs)
     std::vector<SlabPlan> host;
     plan_slabs(r, host);
     for (const SlabPlan &w : host) rows = std::max(rows, w.row_hi - w.row_lo);
@@ -1064,10 +1251,11 @@ int Iso_request_get_execution(Iso_request request, int *slabs, int *chains, int 
     return ISO_SUCCESS;
 }
 
-int Iso_request_tune(Iso_request request, void *cuda_stream, int cold)
+int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
 {
     return guarded([&]() -> int {
-    if (check_handle(request)) return ISO_ERR_ARG;
+    if (check_handle(request) || (flags & ~(ISO_TUNE_COLD | ISO_TUNE_SCHEDULE))) return ISO_ERR_ARG;
+    const bool cold = (flags & ISO_TUNE_COLD) != 0;
     Request &r = *request;
     if (!r.send || !r.recv) return ISO_ERR_STATE;
     if (r.persistent || r.wave_request > 0) return ISO_SUCCESS;
@@ -1094,18 +1282,28 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int cold)
         }
     }
     const bool log = r.knobs.tune_log;
-    struct Choice { int slabs, chains, graph; };
-    const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0};
+    struct Choice { int slabs, chains, graph, alg, fusion; };
+    const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0, r.alg, r.fusion};
     Choice best = before;
     float best_ms = -1.0f;
     int rc = ISO_SUCCESS;
     const int p0 = r.comm->dims[0];
-    auto apply = [&](const Choice &c) {
+    auto apply = [&](const Choice &c) -> int {
         r.slab_request = c.slabs;
         r.chains_request = c.chains;
         r.graph_request = c.graph != 0;
         r.dirty = true;
+        if (c.alg != r.alg || c.fusion != r.fusion) return Iso_request_set_algorithm(request, c.alg, c.fusion);
+        return ISO_SUCCESS;
     };
+    // the schedules to try: the present one, or - when asked - the message-combining schedule
+    // with the hops of 1 and of 2 consecutive dimensions per phase, and the direct schedule
+    std::vector<std::pair<int, int>> schedules(1, std::make_pair(r.alg, r.fusion));
+    if (flags & ISO_TUNE_SCHEDULE) {
+        schedules.assign(1, std::make_pair((int)ISO_ALG_COMBINING, 1));
+        if (r.comm->d >= 3) schedules.push_back(std::make_pair((int)ISO_ALG_COMBINING, 2));
+        schedules.push_back(std::make_pair((int)ISO_ALG_DIRECT, 1));
+    }
     // time `reps` starts back to back (the collective only reads the send buffers, so
     // repeating it leaves the same result)
     auto measure = [&](int reps, float &ms) -> int {
@@ -1127,18 +1325,19 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int cold)
         ms /= (float)reps;
         return ISO_SUCCESS;
     };
+    for (const auto &sched : schedules) {
     std::vector<Choice> tried;
     for (int graph = 0; graph <= 1 && rc == ISO_SUCCESS; ++graph)
         for (int chains = 1; chains <= 4 && rc == ISO_SUCCESS; chains *= 2) {
             if (chains > 1 && !graph) continue;  // chains only exist inside a graph
             for (int slabs = 1; slabs <= 64 && slabs <= std::max(1, p0) && rc == ISO_SUCCESS; slabs *= 2) {
                 if (chains > 1 && slabs < chains) continue;
-                apply(Choice{slabs, chains, graph});
                 if (r.started) rc = Iso_wait(request);
+                if (rc == ISO_SUCCESS) rc = apply(Choice{slabs, chains, graph, sched.first, sched.second});
                 if (rc == ISO_SUCCESS) rc = materialise(r);
                 if (rc != ISO_SUCCESS) break;
                 // what the schedule allowed may differ from what was asked for: skip repeats
-                const Choice got{(int)std::max<size_t>(1, r.slab_plan.size()), r.chains, r.use_graph ? 1 : 0};
+                const Choice got{(int)std::max<size_t>(1, r.slab_plan.size()), r.chains, r.use_graph ? 1 : 0, r.alg, r.fusion};
                 bool seen = false;
                 for (const Choice &c : tried) seen = seen || (c.slabs == got.slabs && c.chains == got.chains && c.graph == got.graph);
                 if (seen) continue;
@@ -1149,24 +1348,42 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int cold)
                 const int reps = (int)std::max(5.0f, std::min(200.0f, 2.0f / std::max(ms, 1e-3f)));
                 rc = measure(reps, ms);
                 if (rc != ISO_SUCCESS) break;
-                if (log) std::fprintf(stderr, "iso tune: slabs %d chains %d graph %d: %.4f ms\n", got.slabs, got.chains, got.graph, ms);
+                if (log)
+                    std::fprintf(stderr, "iso tune: alg %d fusion %d slabs %d chains %d graph %d: %.4f ms\n", got.alg, got.fusion,
+                                 got.slabs, got.chains, got.graph, ms);
                 // the plainer plans come first; a later one must win by 2 % to replace them
                 if (best_ms < 0.0f || ms < 0.98f * best_ms) {
                     best_ms = ms;
-                    best = Choice{slabs, chains, graph};
+                    best = Choice{slabs, chains, graph, sched.first, sched.second};
                 }
             }
         }
+    }
     cudaEventDestroy(t0);
     cudaEventDestroy(t1);
     if (scratch) cudaFree(scratch);
-    apply(rc == ISO_SUCCESS ? best : before);
     if (r.started) {
         int e = Iso_wait(request);
         if (rc == ISO_SUCCESS) rc = e;
     }
-    int e = materialise(r);
+    int e = apply(rc == ISO_SUCCESS ? best : before);
+    if (e == ISO_SUCCESS) e = materialise(r);
     return rc != ISO_SUCCESS ? rc : e;
+    });
+}
+
+int Iso_request_set_sender_side(Iso_request request, int mode)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request) || mode < 0 || mode > 2) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    request->sender_side = mode;
+    int rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
+    request->dirty = true;
+    return rc;
     });
 }
 
@@ -1322,72 +1539,49 @@ int Iso_Start_host(Iso_request request, const void *host_sendbuf, void *host_rec
         int rc = Iso_Start(request, cuda_stream);
         if (rc != ISO_SUCCESS) return rc;
         if (rbytes) ISO_CUDA(cudaMemcpyAsync(hr, r.recv, rbytes, cudaMemcpyDeviceToHost, stream));
+        r.host_timed = false;
         return ISO_SUCCESS;
     }
 
-    // Pipelined over slabs of the leading dimension.  Only blocks read from the send buffer
-    // cross slabs, so a slab's whole schedule can run as soon as the send buffers of the
-    // slabs it reads have arrived, and its receive buffers can travel back while later
-    // slabs are still on their way in.  Three streams: uploads back to back on one, kernels
-    // on the caller's stream, downloads on a third, so that both directions of the link are
-    // busy at the same time and no copy waits behind a kernel.
-    const size_t S = slabs.size();
-    if (!r.copy_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.copy_stream), cudaStreamNonBlocking));
-    if (!r.up_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.up_stream), cudaStreamNonBlocking));
-    cudaStream_t down = static_cast<cudaStream_t>(r.copy_stream), up = static_cast<cudaStream_t>(r.up_stream);
-    while (r.slab_events.size() < 2 * S + 1) {
-        cudaEvent_t e;
-        ISO_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-        r.slab_events.push_back(e);
+    // Pipelined over slabs of the leading dimension (enqueue_host_pipeline).  The same call
+    // with the same host buffers is a fixed sequence of a few hundred copies, launches and
+    // event operations: the first such call enqueues them one by one, the second captures
+    // them into a graph, and from then on a start is one graph launch (submitting the
+    // sequence one call at a time took longer than the 54 MB transfers of the 32^3 torus).
+    const unsigned char *hs_b = hs;
+    unsigned char *hr_b = hr;
+    if (r.host_graph_exec && r.host_graph_hs == hs_b && r.host_graph_hr == hr_b) {
+        ISO_CUDA(cudaGraphLaunch(static_cast<cudaGraphExec_t>(r.host_graph_exec), stream));
+    } else if (r.knobs.host_graph && r.host_last_hs == hs_b && r.host_last_hr == hr_b && page_locked(hs_b) && page_locked(hr_b)) {
+        if (r.host_graph_exec) cudaGraphExecDestroy(static_cast<cudaGraphExec_t>(r.host_graph_exec));
+        r.host_graph_exec = nullptr;
+        if (!r.host_main_stream)
+            ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.host_main_stream), cudaStreamNonBlocking));
+        int rc = prepare_host_pipeline(r, slabs.size());
+        if (rc != ISO_SUCCESS) return rc;
+        cudaStream_t origin = static_cast<cudaStream_t>(r.host_main_stream);
+        cudaGraph_t graph = nullptr;
+        ISO_CUDA(cudaStreamBeginCapture(origin, cudaStreamCaptureModeThreadLocal));
+        rc = enqueue_host_pipeline(r, slabs, hs_b, hr_b, origin, true);
+        cudaError_t e = cudaStreamEndCapture(origin, &graph);
+        cudaGraphExec_t exec = nullptr;
+        if (rc == ISO_SUCCESS && e == cudaSuccess) e = cudaGraphInstantiate(&exec, graph, 0);
+        if (graph) cudaGraphDestroy(graph);
+        if (rc != ISO_SUCCESS) return rc;
+        if (e != cudaSuccess) return cuda_fail(e);
+        r.host_graph_exec = exec;
+        r.host_graph_hs = hs_b;
+        r.host_graph_hr = hr_b;
+        ISO_CUDA(cudaGraphLaunch(exec, stream));
+    } else {
+        int rc = prepare_host_pipeline(r, slabs.size());
+        if (rc == ISO_SUCCESS) rc = enqueue_host_pipeline(r, slabs, hs_b, hr_b, stream, false);
+        if (rc != ISO_SUCCESS) return rc;
     }
-    // copies of this call must not overtake earlier work on the caller's stream
-    cudaEvent_t fence = static_cast<cudaEvent_t>(r.slab_events[2 * S]);
-    ISO_CUDA(cudaEventRecord(fence, stream));
-    ISO_CUDA(cudaStreamWaitEvent(up, fence, 0));
-    ISO_CUDA(cudaStreamWaitEvent(down, fence, 0));
-    const bool use_pdl = !r.knobs.no_pdl;
-    // Upload order: the last slab first, then 0, 1, ...: on a torus slab 0 reads the last slab,
-    // so in natural order it (and its download) would have to wait for the very last upload.
-    std::vector<size_t> order(S), pos(S);
-    for (size_t i = 0; i < S; ++i) order[i] = S <= 64 ? (i + S - 1) % S : i;
-    for (size_t i = 0; i < S; ++i) pos[order[i]] = i;
-    std::vector<size_t> ready_at(S, 0);  // position in the upload order after which a slab can run
-    for (size_t k = 0; k < S; ++k) {
-        if (S <= 64) {
-            for (size_t j = 0; j < S; ++j)
-                if (slabs[k].needs >> j & 1ULL) ready_at[k] = std::max(ready_at[k], pos[j]);
-            ready_at[k] = std::max(ready_at[k], pos[k]);
-        } else {
-            ready_at[k] = (size_t)std::max(slabs[k].last_needed, (int)k);
-        }
-    }
-    std::vector<char> done(S, 0);
-    for (size_t upi = 0; upi < S; ++upi) {
-        const SlabPlan &u = slabs[order[upi]];
-        const size_t off = (size_t)(u.row_lo * r.send_stride), n = (size_t)((u.row_hi - u.row_lo) * r.send_stride);
-        if (n) ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send) + off, hs + off, n, cudaMemcpyHostToDevice, up));
-        cudaEvent_t arrived = static_cast<cudaEvent_t>(r.slab_events[S + upi]);
-        ISO_CUDA(cudaEventRecord(arrived, up));
-        // every slab whose last needed upload this was
-        for (size_t k = 0; k < S; ++k) {
-            if (done[k] || ready_at[k] > upi) continue;
-            const SlabPlan &w = slabs[k];
-            ISO_CUDA(cudaStreamWaitEvent(stream, arrived, 0));
-            for (const LaunchPlan &L : r.launches) {
-                int rc = launch_one(r, L, stream, use_pdl, w.row_lo, w.row_hi, r.inter_rows < c.P ? w.row_lo : 0);
-                if (rc != ISO_SUCCESS) return rc;
-            }
-            cudaEvent_t ev = static_cast<cudaEvent_t>(r.slab_events[k]);
-            ISO_CUDA(cudaEventRecord(ev, stream));
-            ISO_CUDA(cudaStreamWaitEvent(down, ev, 0));
-            const size_t roff = (size_t)(w.row_lo * r.recv_stride), rn = (size_t)((w.row_hi - w.row_lo) * r.recv_stride);
-            if (rn) ISO_CUDA(cudaMemcpyAsync(hr + roff, r.recv + roff, rn, cudaMemcpyDeviceToHost, down));
-            done[k] = 1;
-        }
-    }
-    // join: the caller's stream is complete only when the downloads are
-    ISO_CUDA(cudaEventRecord(fence, down));
-    ISO_CUDA(cudaStreamWaitEvent(stream, fence, 0));
+    r.host_last_hs = hs_b;
+    r.host_last_hr = hr_b;
+    r.host_timed = true;
+    r.host_slabs_used = (int)slabs.size();
     r.last_stream = cuda_stream;
     r.started = true;
     return ISO_SUCCESS;
@@ -1417,6 +1611,27 @@ int Iso_wait(Iso_request request)
         ISO_CUDA(cudaStreamSynchronize(stream));
         return ISO_ERR_TIMEOUT;
     }
+    return ISO_SUCCESS;
+    });
+}
+
+int Iso_request_get_host_transfer_ms(Iso_request request, float *upload_ms, float *download_ms, float *total_ms,
+                                     int *slabs)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request)) return ISO_ERR_ARG;
+    Request &r = *request;
+    if (!r.host_timed) return ISO_ERR_STATE;
+    int rc = Iso_wait(request);
+    if (rc != ISO_SUCCESS) return rc;
+    auto span = [&](int a, int b, float *out) -> cudaError_t {
+        if (!out) return cudaSuccess;
+        return cudaEventElapsedTime(out, static_cast<cudaEvent_t>(r.host_timing[a]), static_cast<cudaEvent_t>(r.host_timing[b]));
+    };
+    ISO_CUDA(span(0, 1, upload_ms));
+    ISO_CUDA(span(2, 3, download_ms));
+    ISO_CUDA(span(4, 5, total_ms));
+    if (slabs) *slabs = r.host_slabs_used;
     return ISO_SUCCESS;
     });
 }

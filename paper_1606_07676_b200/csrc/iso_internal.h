@@ -53,7 +53,22 @@ struct LoweredPart {
     int width = 16;    // bytes per unit of this piece (differs between pieces in a launch of mixed widths)
 };
 
-enum { KERNEL_VEC = 0, KERNEL_BULK = 1 };
+enum { KERNEL_VEC = 0, KERNEL_BULK = 1, KERNEL_FAN = 2 };
+
+// Sender-side form of an allgather phase (Section III-B: a trie edge carries one block once):
+// a parent block, read once from the process that holds it, and the places it is copied to.
+struct FanDst {
+    int buf = ISO_BUF_RECV;
+    int64_t off = 0;
+    int c = 0;  // the destination process is the source process shifted by +c along the phase's dimension, c in [0, p)
+};
+struct FanParent {
+    int src_buf = ISO_BUF_SEND;
+    int64_t src_off = 0;
+    int64_t len = 0;
+    std::vector<FanDst> dsts;  // at most kFanDsts
+};
+constexpr int kFanDsts = 4;  // destinations per descriptor; a parent with more is listed several times
 constexpr int kMaxVecUnits = 4096;  // unit positions per process in one vector launch
 constexpr int kVecDepth = 8;        // cp.async ring slots per thread in the vector kernel
 constexpr int kWideDepth = 12;      // the same in CTAs of more than 256 threads (one CTA per SM)
@@ -77,6 +92,7 @@ struct LaunchPlan {
     int used_dim[ISO_MAX_DIMS] = {0};
     int max_nnz = 0;       // most dimensions any one part shifts along
     bool compact = false;  // vector kernel: unit descriptors list only the shifted dimensions
+    std::vector<FanParent> fans;  // KERNEL_FAN: the launch as parents and their destinations (parts: the same copies, one per destination)
     // byte offsets of this launch's tables inside the request's device blob
     size_t parts_off = 0, lookup_off = 0, units_off = 0;
 };
@@ -98,7 +114,9 @@ struct Knobs {
     int chains = -1;          // ISO_CHAINS
     bool no_pdl = false;      // ISO_NO_PDL: plain launches instead of programmatic dependent ones
     bool tune_log = false;    // ISO_TUNE_LOG: the tuner prints every plan it times
-    bool multi_dst = true;    // ISO_MULTI_DST=0: allgather units with one destination each
+    int sender_side = -1;     // ISO_SENDER_SIDE: 0 never, 1 automatic, 2 wherever possible (allgather phases; -1: the request's setting)
+    bool host_graph = true;   // ISO_HOST_GRAPH=0: the pipelined host-buffer path is never replayed from a graph
+    bool coord_table = true;  // ISO_COORD_TABLE=0: row coordinates by division in every thread
 };
 Knobs read_knobs();
 
@@ -139,6 +157,13 @@ struct Request {
     void *copy_stream = nullptr;       // download stream of the pipelined host-buffer path
     void *up_stream = nullptr;         // its upload stream
     std::vector<void *> slab_events;   // its events
+    void *host_main_stream = nullptr;  // origin stream when that path is captured into a graph
+    void *host_graph_exec = nullptr;   // cudaGraphExec_t of one pipelined host-buffer start
+    const void *host_graph_hs = nullptr, *host_graph_hr = nullptr;  // the host buffers that graph copies from / to
+    const void *host_last_hs = nullptr, *host_last_hr = nullptr;    // the host buffers of the last such start
+    std::vector<void *> host_timing;   // timing events of its last call: uploads, downloads, whole call (begin, end each)
+    bool host_timed = false;
+    int host_slabs_used = 0;
     int sm_count = 148;  // a B200's; replaced by the current device's count before the first start
     int chains_request = 1;     // slabs to run side by side, as asked for
     bool graph_request = false; // graph replay, as asked for
@@ -154,6 +179,7 @@ struct Request {
     size_t wave_smem = 0, wave_launches_off = 0, wave_items_off = 0;
     unsigned long long wave_run = 0;  // starts since the counters were last zeroed
     int wave_counters = 0;      // counters allocated in d_counter
+    int sender_side = 1;        // allgather phases in sender-side form: 0 never, 1 where measured faster, 2 wherever possible
     uint32_t wait_limit = 1u << 22;  // polls before a device-side wait on other CTAs gives up
     int skew_next = 0;          // testing: extra arrivals the next cooperative start waits for (one shot)
 };

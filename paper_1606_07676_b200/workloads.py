@@ -225,6 +225,7 @@ def config(name: str, seed: int = DEFAULT_SEED) -> Workload:
     cfg2_alltoall  all-to-all, 32^3, Moore r=1, 64 B of fp32 in [-1,1)
     cfg2_allgather allgather,  same torus and neighbourhood
     cfg3_m<M>      all-to-all, 256^2, Moore r=2, M in {4,64,512,4096} uint8 bytes
+                   (cfg3_m<M>_<a>x<b>: the same on an a x b torus)
     cfg4           all-to-all, 8^5, Moore r=1, 16 B of fp32
     cfg5           irregular all-to-all, 64x64x32, 30 random offsets in [-3,3]^3,
                    lengths uniform over {4,16,64,256,1024} B, packed displacements
@@ -240,8 +241,11 @@ def config(name: str, seed: int = DEFAULT_SEED) -> Workload:
     if name == "cfg2_allgather":
         return Workload(name, "allgather", (32, 32, 32), moore(3, 1), 64, kind="fp32", seed=seed)
     if name.startswith("cfg3_m"):
-        m = int(name[len("cfg3_m"):])
-        return Workload(name, "alltoall", (256, 256), moore(2, 2), m, kind="uint8", seed=seed)
+        # cfg3_m<M>_<a>x<b>: the same neighbourhood and block size on an a x b torus (fewer rows,
+        # same row length: the case profiler captures with many passes are taken on)
+        size, _, shape = name[len("cfg3_m"):].partition("_")
+        dims = tuple(int(x) for x in shape.split("x")) if shape else (256, 256)
+        return Workload(name, "alltoall", dims, moore(2, 2), int(size), kind="uint8", seed=seed)
     if name == "cfg4":
         return Workload(name, "alltoall", (8, 8, 8, 8, 8), moore(5, 1), 16, kind="fp32", seed=seed)
     if name in ("cfg5", "cfg5_32x32x32"):

@@ -114,6 +114,7 @@ def test_random_cases(chunk):
             # applies where the schedule allows and is ignored elsewhere
             pipe = (0, 0, 1, 0, 3)[(c["trial"] + 2 * alg + fusion) % 5]
             iso.Iso_request_set_pipeline(req, pipe)
+            iso.Iso_request_set_sender_side(req, (2, 1, 2, 0)[(c["trial"] + fusion) % 4])
             iso.Iso_request_set_algorithm(req, alg, fusion)
             if rs:
                 recv.fill_(POISON)

@@ -153,6 +153,14 @@ def test_chains_graph_replay_and_tuning(torch_cuda):
             iso.Iso_wait(run.req)
             assert np.array_equal(run.recv.cpu().numpy().reshape(want.shape), want), (name, "tuned", chosen)
             assert iso.Iso_request_get_execution(run.req) == chosen
+        # the tuner may choose the schedule as well: whatever it keeps gives the oracle's bytes
+        chosen = iso.Iso_request_tune(run.req, torch.cuda.current_stream(), cold=False, schedule=True)
+        st = iso.Iso_request_get_stats(run.req)
+        assert (st["algorithm"], st["fusion_level"]) in [(iso.ISO_ALG_COMBINING, 1), (iso.ISO_ALG_COMBINING, 2), (iso.ISO_ALG_DIRECT, 1)]
+        run.recv.fill_(0xA5)
+        iso.Iso_Start(run.req, torch.cuda.current_stream())
+        iso.Iso_wait(run.req)
+        assert np.array_equal(run.recv.cpu().numpy().reshape(want.shape), want), (name, "tuned schedule", chosen, st["algorithm"])
         run.close()
 
 
@@ -213,6 +221,37 @@ def test_narrow_cta_shapes(torch_cuda, monkeypatch):
 
 def test_cfg2_allgather(torch_cuda):
     check(torch_cuda, wl.config("cfg2_allgather"), [COMB0, COMB1, COMB2, COMBD, DIRECT])
+
+
+def test_allgather_phases_in_sender_side_form(torch_cuda):
+    """Allgather phases as one load and up to four stores per 16-byte unit (forced on with
+    mode 2; left to the library, only large phases take this form): same bytes as the oracle
+    on the configuration, the paper's neighbourhoods (blocks with up to fourteen copies, so a
+    block is listed several times), tiny and aliasing tori, repeated vectors, the zero vector,
+    the irregular allgather, and after switching the form off again."""
+    torch = torch_cuda
+    cases = [wl.config("cfg2_allgather"), wl.config("octant_d3r3_allgather"), wl.config("moore_d4r1_allgather"),
+             wl.Workload("sh", "allgather", (16, 15, 17), wl.shells(3, (3, 7)), 16, seed=3),
+             wl.Workload("m33", "allgather", (9, 8, 7), wl.moore(3, 3), 48, seed=4),
+             wl.Workload("rag", "allgather", (37, 53), wl.moore(2, 2), 80, seed=5)]
+    cases += [w for w in _tiny_cases() if w.collective == "allgather" and w.block_bytes % 16 == 0]
+    for w in cases:
+        run = Run(torch, w)
+        want = oracle_result(w, run.send_host)
+        for mode, kernels in ((2, {2}), (0, {0, 1}), (1, {0, 1, 2})):
+            iso.Iso_request_set_sender_side(run.req, mode)
+            for alg, fusion in (COMB1, COMB0):
+                got = run.result(alg, fusion)
+                assert np.array_equal(got, want), (w.name, w.dims, mode, alg, fusion)
+                used = {p["kernel"] for p in iso.Iso_request_get_parts(run.req)}
+                assert used <= kernels, (w.name, mode, used)
+            assert iso.Iso_request_check_guards(run.req) == 0
+        run.close()
+    # left to the library, the large phases of the 80-neighbour allgather take this form
+    run = Run(torch, wl.config("moore_d4r1_allgather"))
+    run.result(*COMB1)
+    assert {p["phase"] for p in iso.Iso_request_get_parts(run.req) if p["kernel"] == 2} == {2, 3}
+    run.close()
 
 
 @pytest.mark.parametrize("m", [4, 64, 512])
@@ -475,6 +514,37 @@ def test_persistent_request_streams_and_host_buffers(torch_cuda):
     iso.Iso_wait(run.req)
     assert np.array_equal(hr.numpy(), want)
     run.close()
+
+
+def test_host_buffer_starts_replayed_from_a_graph(torch_cuda):
+    """Repeated Iso_Start_host calls with the same page-locked buffers: the first is enqueued
+    call by call, the second is captured into a graph, later ones replay it.  New contents in
+    the same host buffer must come through every time, on a side stream as well."""
+    torch = torch_cuda
+    w = wl.config("cfg2_alltoall")
+    side = torch.cuda.Stream()
+    run = Run(torch, w, stream=side)
+    hs = torch.empty((w.P, run.ss), dtype=torch.uint8).pin_memory()
+    hr = torch.empty((w.P, run.rs), dtype=torch.uint8).pin_memory()
+    try:
+        for k in range(5):
+            contents = wl.payload_np(w.kind, 900 + k, 0, 0, w.P * run.ss).reshape(w.P, run.ss)
+            hs.copy_(torch.from_numpy(contents))
+            hr.fill_(0)
+            run.recv.fill_(POISON)
+            torch.cuda.synchronize()
+            iso.Iso_Start_host(run.req, hs, hr, side)
+            iso.Iso_wait(run.req)
+            assert np.array_equal(hr.numpy(), oracle_result(w, contents)), k
+            t = iso.Iso_request_get_host_transfer_ms(run.req)
+            assert t["slabs"] == 32 and 0 < t["upload_ms"] <= t["total_ms"] and 0 < t["download_ms"] <= t["total_ms"], t
+        # a plain start in between, then host buffers again
+        assert np.array_equal(run.result(*COMB1), oracle_result(w, contents))
+        iso.Iso_Start_host(run.req, hs, hr, side)
+        iso.Iso_wait(run.req)
+        assert np.array_equal(hr.numpy(), oracle_result(w, contents))
+    finally:
+        run.close()
 
 
 @pytest.mark.parametrize("name", ["cfg2_alltoall", "cfg2_allgather", "cfg3_m64", "cfg5"])

@@ -239,6 +239,28 @@ def test_allgather_statistics_follow_the_trie():
         assert st["parts"] == counters.allgather_direct_volume(offs, 3, dims)
         assert st["rounds"] == counters.direct_rounds(offs, 3, dims)
         assert st["bytes_moved"] == 2 * w.P * 64 * (st["parts"] + st["local_copies"])
+        # sender-side launches: a parent block is read once for up to four of the places it is
+        # copied to, every copy is written
+        iso.Iso_request_set_sender_side(req, 2)
+        st = iso.Iso_request_get_stats(req)
+        parts = iso.Iso_request_get_parts(req)
+        assert len(parts) == st["parts"] + st["local_copies"] and all(p["kernel"] == 2 for p in parts)
+        children = {}
+        for p in parts:
+            key = (p["phase"], p["src_buf"], p["src_off"])
+            children[key] = children.get(key, 0) + 1
+        reads = sum(-(-n // 4) for n in children.values())
+        assert st["bytes_moved"] == w.P * 64 * (reads + len(parts))
+        # the schedule is the same one: executed on the host it gives the oracle's result
+        send = send_buffer_np(w, st["send_stride"])
+        if w.P <= 4096:
+            assert np.array_equal(simulate(parts, w.dims, st, send), oracle_result(w, send))
+        # the receiver-side form (asked for through a slab count) reads a block once per copy
+        iso.Iso_request_set_slabs(req, 2)
+        iso.Iso_request_set_bulk_threshold(req, 512)
+        st2 = iso.Iso_request_get_stats(req)
+        assert st2["bytes_moved"] == 2 * w.P * 64 * (st["parts"] + st["local_copies"])
+        assert all(p["kernel"] == 0 for p in iso.Iso_request_get_parts(req))
         iso.Iso_request_free(req)
         iso.Iso_comm_free(comm)
     # Moore neighbourhoods need no intermediate storage: every padded prefix is a neighbour
