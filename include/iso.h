@@ -290,7 +290,8 @@ int Iso_request_set_graph(Iso_request request, int enable);
 /*
  * Measures instead of guessing (no counterpart in the paper; in the spirit of its
  * persistent requests, which are set up once and started many times): runs the request
- * with 1, 2, 4, ... slabs, with 1, 2 and 4 chains, with and without graph replay, timing a
+ * with 1, 2, 4, ... slabs, with 1, 2 and 4 chains, with and without graph replay (and, for
+ * ragged rows, with and without the bulk warps of Iso_request_set_hybrid), timing a
  * few starts of each on `cuda_stream` with events, and leaves the request on the fastest
  * combination (a less plain plan has to win by 2 %).  `flags` is a sum of ISO_TUNE_* values.
  * Without ISO_TUNE_COLD the starts are timed back to back, as in a loop over the same
@@ -313,6 +314,18 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags);
  * Before the first Iso_Start after a change these are the values asked for (slabs 0:
  * automatic); any of the pointers may be NULL. */
 int Iso_request_get_execution(Iso_request request, int *slabs, int *chains, int *graph);
+
+/*
+ * Ragged rows of the irregular collectives (no counterpart in the paper).  A launch whose
+ * pieces need several unit widths normally moves everything through the vector kernel.  With
+ * `enable` != 0 the 16-byte-aligned bodies of at least 256 bytes among its pieces are moved
+ * by bulk copies instead, issued by extra warps of the same thread blocks while the other
+ * warps move the short pieces and ragged ends (up to three dimensions, periodic, bulk
+ * threshold not 0).  Measured on irregular sizes from {4, ..., 1024} bytes: 22 % faster for the
+ * one-pass direct schedule on the 64x64x32 torus, 15 % slower for the combining schedule in
+ * slabs, hence off by default; Iso_request_tune tries both.  The result never depends on it.
+ */
+int Iso_request_set_hybrid(Iso_request request, int enable);
 
 /*
  * Sender-side form of allgather phases (Section III-B: a block travels once per trie edge).

@@ -31,7 +31,7 @@ EXPORTS = (
     "Iso_neighborhood_create", "Iso_comm_free", "Iso_comm_set_periodic",
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
     "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_pipeline", "Iso_request_set_chains", "Iso_request_set_graph", "Iso_request_tune", "Iso_request_get_execution", "Iso_request_set_bulk_threshold",
-    "Iso_request_set_sender_side", "Iso_request_check_guards", "Iso_request_get_host_transfer_ms", "Iso_request_set_wait_limit", "Iso_request_test_skew_arrivals", "Iso_measure_launch_floor",
+    "Iso_request_set_hybrid", "Iso_request_set_sender_side", "Iso_request_check_guards", "Iso_request_get_host_transfer_ms", "Iso_request_set_wait_limit", "Iso_request_test_skew_arrivals", "Iso_measure_launch_floor",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
     "Iso_neighbor_alltoall_static", "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
@@ -101,6 +101,7 @@ def load_library() -> ctypes.CDLL:
         "Iso_request_tune": [vp, vp, ci],
         "Iso_request_get_execution": [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)],
         "Iso_request_set_bulk_threshold": [vp, i64],
+        "Iso_request_set_hybrid": [vp, ci],
         "Iso_request_set_sender_side": [vp, ci],
         "Iso_request_check_guards": [vp, ctypes.POINTER(i64)],
         "Iso_request_get_host_transfer_ms": [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
@@ -297,6 +298,10 @@ def Iso_request_get_host_transfer_ms(request: int) -> dict:
                                                            ctypes.byref(total), ctypes.byref(slabs)),
            "Iso_request_get_host_transfer_ms")
     return {"upload_ms": up.value, "download_ms": down.value, "total_ms": total.value, "slabs": slabs.value}
+
+
+def Iso_request_set_hybrid(request: int, enable: bool) -> None:
+    _check(load_library().Iso_request_set_hybrid(request, 1 if enable else 0), "Iso_request_set_hybrid")
 
 
 def Iso_request_set_sender_side(request: int, mode: int) -> None:

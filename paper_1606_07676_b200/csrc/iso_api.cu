@@ -49,14 +49,12 @@ void release_device(Request &r)
     if (r.d_inter_alloc) cudaFree(r.d_inter_alloc);
     r.d_inter_alloc = nullptr;
     if (r.d_err) cudaFree(r.d_err);
-    if (r.copy_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.copy_stream));
-    if (r.up_stream) cudaStreamDestroy(static_cast<cudaStream_t>(r.up_stream));
-    r.up_stream = nullptr;
+    for (void *st : r.host_streams) cudaStreamDestroy(static_cast<cudaStream_t>(st));
+    r.host_streams.clear();
     for (void *e : r.slab_events) cudaEventDestroy(static_cast<cudaEvent_t>(e));
     for (void *e : r.host_timing) cudaEventDestroy(static_cast<cudaEvent_t>(e));
     r.host_timing.clear();
     r.host_timed = false;
-    r.copy_stream = nullptr;
     r.slab_events.clear();
     if (r.d_counter) cudaFree(r.d_counter);
     r.d_counter = nullptr;
@@ -135,6 +133,7 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
     r->kind = kind;
     r->knobs = read_knobs();
     if (r->knobs.sender_side >= 0 && r->knobs.sender_side <= 2) r->sender_side = r->knobs.sender_side;
+    if (r->knobs.hybrid >= 0) r->hybrid = r->knobs.hybrid != 0;
     r->send = static_cast<const unsigned char *>(sendbuf);
     r->recv = static_cast<unsigned char *>(recvbuf);
     r->s = comm->s;
@@ -276,8 +275,15 @@ int materialise(Request &r)
     int rc = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
     if (rc != ISO_SUCCESS) return rc;
 
-    size_t bytes = 0;
+    // every plan that needs tables: the launches and the bulk sides of hybrid launches
+    std::vector<LaunchPlan *> plans;
     for (LaunchPlan &L : r.launches) {
+        plans.push_back(&L);
+        for (LaunchPlan &S : L.side) plans.push_back(&S);
+    }
+    size_t bytes = 0;
+    for (LaunchPlan *plan : plans) {
+        LaunchPlan &L = *plan;
         L.parts_off = bytes;
         bytes += L.parts.size() * sizeof(PartDev);
         L.lookup_off = bytes;
@@ -306,7 +312,8 @@ int materialise(Request &r)
     const size_t wave_items_off = bytes;
     bytes += wave_n * sizeof(WaveItem);
     std::vector<unsigned char> blob(bytes ? bytes : 16, 0);
-    for (const LaunchPlan &L : r.launches) {
+    for (const LaunchPlan *plan : plans) {
+        const LaunchPlan &L = *plan;
         int used_index[ISO_MAX_DIMS];
         for (int j = 0; j < ISO_MAX_DIMS; ++j) used_index[j] = -1;
         for (int k = 0; k < L.n_used; ++k) used_index[L.used_dim[k]] = k;
@@ -580,6 +587,38 @@ cudaError_t launch_wide(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, 
     return launch_kernel(kernel, L, a, stream, dependent);
 }
 
+// The hybrid kernel: the vector side's threads plus one warp for the bulk side.
+template <typename Kernel>
+cudaError_t launch_hybrid(Kernel kernel, const LaunchPlan &L, const LaunchDev &a, const LaunchDev &side, size_t smem,
+                          cudaStream_t stream, bool dependent)
+{
+    static std::vector<std::pair<int, const void *>> opted_in;
+    static std::mutex guard;
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return e;
+    const std::pair<int, const void *> key(device, reinterpret_cast<const void *>(kernel));
+    {
+        std::lock_guard<std::mutex> lock(guard);
+        if (std::find(opted_in.begin(), opted_in.end(), key) == opted_in.end()) {
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+            if (e != cudaSuccess) return e;
+            opted_in.push_back(key);
+        }
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid_for_rows(L, a, a.grid_share));
+    cfg.blockDim = dim3((unsigned)L.threads + side.chunk_units);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, a, side);
+}
+
 // The wide vector kernel with or without the coordinate table; the table variants exist for
 // the cases launch_one uses them in.
 template <int W, int NU, bool MESH, bool COMPACT>
@@ -610,6 +649,30 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
         e = launch_kernel(iso_gather_bulk, L, a, stream, dependent);
     } else if (L.kernel == KERNEL_FAN) {
         e = launch_wide(iso_fan_rows<kWideDepth>, L, a, stream, dependent);
+    } else if (!L.side.empty()) {
+        // mixed-width launch with a bulk side: vector warps + one bulk warp per CTA
+        LaunchDev sd = make_launch_args(r, L.side[0]);
+        sd.row_lo = a.row_lo;
+        sd.row_hi = a.row_hi;
+        if (inter_row_base && sd.buf[ISO_BUF_INTER]) sd.buf[ISO_BUF_INTER] -= inter_row_base * r.inter_stride;
+        const long long groups = (a.row_hi - a.row_lo + L.rows_per_pass - 1) / L.rows_per_pass;
+        const long long grid = grid_for_rows(L, a, a.grid_share);
+        bool tab = false;
+        if (L.n_used > 0 && L.n_used <= 2 && r.knobs.coord_table) {
+            a.tab_iters = (uint32_t)((groups + grid - 1) / grid);
+            a.tab_stride = 4;
+            tab = L.smem + table_bytes(a) + 128 + L.side[0].smem <= (size_t)kMaxDynamicSmem;
+            if (!tab) a.tab_iters = 0;
+        }
+        sd.chunk_units = (uint32_t)L.side[0].threads;
+        sd.side_offset = (uint32_t)((L.smem + table_bytes(a) + 127) / 128 * 128);
+        const size_t smem = sd.side_offset + L.side[0].smem;
+        e = L.n_used == 0   ? launch_hybrid(iso_gather_rows_hybrid<kHybridDepth, 0, false>, L, a, sd, smem, stream, dependent)
+            : L.n_used == 1 ? (tab ? launch_hybrid(iso_gather_rows_hybrid<kHybridDepth, 1, true>, L, a, sd, smem, stream, dependent)
+                                   : launch_hybrid(iso_gather_rows_hybrid<kHybridDepth, 1, false>, L, a, sd, smem, stream, dependent))
+            : L.n_used == 2 ? (tab ? launch_hybrid(iso_gather_rows_hybrid<kHybridDepth, 2, true>, L, a, sd, smem, stream, dependent)
+                                   : launch_hybrid(iso_gather_rows_hybrid<kHybridDepth, 2, false>, L, a, sd, smem, stream, dependent))
+                            : launch_hybrid(iso_gather_rows_hybrid<kHybridDepth, 3, false>, L, a, sd, smem, stream, dependent);
     } else if (L.width > 0 && L.width < 4) {
         e = L.width == 2 ? launch_kernel(iso_gather_rows_reg<2, 4>, L, a, stream, dependent)
                          : launch_kernel(iso_gather_rows_reg<1, 4>, L, a, stream, dependent);
@@ -727,12 +790,17 @@ bool page_locked(const void *p)
     return at.type == cudaMemoryTypeHost;
 }
 
-// Streams and events of the pipelined host-buffer path.
+// Streams and events of the pipelined host-buffer path: two streams per direction (a copy
+// costs about 20 microseconds before its first byte moves; with the copies of a direction
+// dealt to two streams the next copy's set-up runs under the current copy's transfer).
 int prepare_host_pipeline(Request &r, size_t S)
 {
-    if (!r.copy_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.copy_stream), cudaStreamNonBlocking));
-    if (!r.up_stream) ISO_CUDA(cudaStreamCreateWithFlags(reinterpret_cast<cudaStream_t *>(&r.up_stream), cudaStreamNonBlocking));
-    while (r.slab_events.size() < 2 * S + 2) {
+    while (r.host_streams.size() < 4) {
+        cudaStream_t st;
+        ISO_CUDA(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
+        r.host_streams.push_back(st);
+    }
+    while (r.slab_events.size() < 2 * S + 4) {
         cudaEvent_t e;
         ISO_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
         r.slab_events.push_back(e);
@@ -750,27 +818,31 @@ int prepare_host_pipeline(Request &r, size_t S)
 // Enqueues one pipelined host-buffer start.  Only blocks read from the send buffer cross
 // slabs, so a slab's whole schedule can run as soon as the send buffers of the slabs it reads
 // have arrived, and its receive buffers can travel back while later slabs are still on their
-// way in.  Three streams: uploads back to back on one, kernels on `stream`, downloads on a
-// third, so that both directions of the link are busy at the same time and no copy waits
-// behind a kernel.  With `capturing` the calls are being recorded into a graph (`stream` is
-// the capture's origin): the timing events then become external event nodes.
+// way in.  Five streams: uploads alternate between two, kernels run on `stream`, downloads
+// alternate between two more, so that both directions of the link are busy at the same time
+// and no copy waits behind a kernel.  With `capturing` the calls are being recorded into a
+// graph (`stream` is the capture's origin): the timing events then become external event nodes.
 int enqueue_host_pipeline(Request &r, const std::vector<SlabPlan> &slabs, const unsigned char *hs, unsigned char *hr,
                           cudaStream_t stream, bool capturing)
 {
     const Comm &c = *r.comm;
     const size_t S = slabs.size();
-    cudaStream_t down = static_cast<cudaStream_t>(r.copy_stream), up = static_cast<cudaStream_t>(r.up_stream);
+    cudaStream_t up[2] = {static_cast<cudaStream_t>(r.host_streams[0]), static_cast<cudaStream_t>(r.host_streams[1])};
+    cudaStream_t down[2] = {static_cast<cudaStream_t>(r.host_streams[2]), static_cast<cudaStream_t>(r.host_streams[3])};
     auto stamp = [&](void *event, cudaStream_t on) -> cudaError_t {
         return cudaEventRecordWithFlags(static_cast<cudaEvent_t>(event), on, capturing ? cudaEventRecordExternal : cudaEventRecordDefault);
     };
+    auto event = [&](size_t k) { return static_cast<cudaEvent_t>(r.slab_events[k]); };
     // copies of this call must not overtake earlier work on the caller's stream
-    cudaEvent_t fence = static_cast<cudaEvent_t>(r.slab_events[2 * S]);
+    cudaEvent_t fence = event(2 * S);
     ISO_CUDA(cudaEventRecord(fence, stream));
-    ISO_CUDA(cudaStreamWaitEvent(up, fence, 0));
-    ISO_CUDA(cudaStreamWaitEvent(down, fence, 0));
+    for (int k = 0; k < 2; ++k) {
+        ISO_CUDA(cudaStreamWaitEvent(up[k], fence, 0));
+        ISO_CUDA(cudaStreamWaitEvent(down[k], fence, 0));
+    }
     ISO_CUDA(stamp(r.host_timing[4], stream));
-    ISO_CUDA(stamp(r.host_timing[0], up));
-    bool first_download = true;
+    ISO_CUDA(stamp(r.host_timing[0], up[0]));
+    size_t downloads = 0;
     const bool use_pdl = !r.knobs.no_pdl;
     // Upload order: the last slab first, then 0, 1, ...: on a torus slab 0 reads the last slab,
     // so in natural order it (and its download) would have to wait for the very last upload.
@@ -791,38 +863,41 @@ int enqueue_host_pipeline(Request &r, const std::vector<SlabPlan> &slabs, const 
     for (size_t upi = 0; upi < S; ++upi) {
         const SlabPlan &u = slabs[order[upi]];
         const size_t off = (size_t)(u.row_lo * r.send_stride), n = (size_t)((u.row_hi - u.row_lo) * r.send_stride);
-        if (n) ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send) + off, hs + off, n, cudaMemcpyHostToDevice, up));
-        cudaEvent_t arrived = static_cast<cudaEvent_t>(r.slab_events[S + upi]);
-        ISO_CUDA(cudaEventRecord(arrived, up));
-        // every slab whose last needed upload this was
+        if (n) ISO_CUDA(cudaMemcpyAsync(const_cast<unsigned char *>(r.send) + off, hs + off, n, cudaMemcpyHostToDevice, up[upi & 1]));
+        ISO_CUDA(cudaEventRecord(event(S + upi), up[upi & 1]));
+        // every slab whose last needed upload this was: it follows this upload and the one
+        // before it, which is the latest on the other upload stream
         for (size_t k = 0; k < S; ++k) {
             if (done[k] || ready_at[k] > upi) continue;
             const SlabPlan &w = slabs[k];
-            ISO_CUDA(cudaStreamWaitEvent(stream, arrived, 0));
+            ISO_CUDA(cudaStreamWaitEvent(stream, event(S + upi), 0));
+            if (upi > 0) ISO_CUDA(cudaStreamWaitEvent(stream, event(S + upi - 1), 0));
             for (const LaunchPlan &L : r.launches) {
                 int rc = launch_one(r, L, stream, use_pdl, w.row_lo, w.row_hi, r.inter_rows < c.P ? w.row_lo : 0);
                 if (rc != ISO_SUCCESS) return rc;
             }
-            cudaEvent_t ev = static_cast<cudaEvent_t>(r.slab_events[k]);
-            ISO_CUDA(cudaEventRecord(ev, stream));
-            ISO_CUDA(cudaStreamWaitEvent(down, ev, 0));
-            if (first_download) ISO_CUDA(stamp(r.host_timing[2], down));
-            first_download = false;
+            ISO_CUDA(cudaEventRecord(event(k), stream));
+            cudaStream_t dn = down[downloads & 1];
+            ISO_CUDA(cudaStreamWaitEvent(dn, event(k), 0));
+            if (downloads == 0) ISO_CUDA(stamp(r.host_timing[2], dn));
+            ++downloads;
             const size_t roff = (size_t)(w.row_lo * r.recv_stride), rn = (size_t)((w.row_hi - w.row_lo) * r.recv_stride);
-            if (rn) ISO_CUDA(cudaMemcpyAsync(hr + roff, r.recv + roff, rn, cudaMemcpyDeviceToHost, down));
+            if (rn) ISO_CUDA(cudaMemcpyAsync(hr + roff, r.recv + roff, rn, cudaMemcpyDeviceToHost, dn));
             done[k] = 1;
         }
     }
-    ISO_CUDA(stamp(r.host_timing[1], up));
-    ISO_CUDA(stamp(r.host_timing[3], down));
-    // join: the caller's stream is complete only when the downloads are
-    ISO_CUDA(cudaEventRecord(fence, down));
+    // join: the caller's stream is complete only when every copy stream is (a capture must
+    // end with every forked stream joined); the time stamps follow the joins
+    ISO_CUDA(cudaEventRecord(event(2 * S + 1), up[1]));
+    ISO_CUDA(cudaStreamWaitEvent(up[0], event(2 * S + 1), 0));
+    ISO_CUDA(stamp(r.host_timing[1], up[0]));
+    ISO_CUDA(cudaEventRecord(event(2 * S + 2), down[1]));
+    ISO_CUDA(cudaStreamWaitEvent(down[0], event(2 * S + 2), 0));
+    ISO_CUDA(stamp(r.host_timing[3], down[0]));
+    ISO_CUDA(cudaEventRecord(fence, down[0]));
     ISO_CUDA(cudaStreamWaitEvent(stream, fence, 0));
-    // the upload stream ends with its time stamp: join it as well (a capture must end with
-    // every forked stream joined)
-    cudaEvent_t up_done = static_cast<cudaEvent_t>(r.slab_events[2 * S + 1]);
-    ISO_CUDA(cudaEventRecord(up_done, up));
-    ISO_CUDA(cudaStreamWaitEvent(stream, up_done, 0));
+    ISO_CUDA(cudaEventRecord(event(2 * S + 3), up[0]));
+    ISO_CUDA(cudaStreamWaitEvent(stream, event(2 * S + 3), 0));
     ISO_CUDA(stamp(r.host_timing[5], stream));
     return ISO_SUCCESS;
 }
@@ -1282,8 +1357,8 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
         }
     }
     const bool log = r.knobs.tune_log;
-    struct Choice { int slabs, chains, graph, alg, fusion; };
-    const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0, r.alg, r.fusion};
+    struct Choice { int slabs, chains, graph, alg, fusion, hybrid; };
+    const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0, r.alg, r.fusion, r.hybrid ? 1 : 0};
     Choice best = before;
     float best_ms = -1.0f;
     int rc = ISO_SUCCESS;
@@ -1292,6 +1367,7 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
         r.slab_request = c.slabs;
         r.chains_request = c.chains;
         r.graph_request = c.graph != 0;
+        r.hybrid = c.hybrid != 0;
         r.dirty = true;
         if (c.alg != r.alg || c.fusion != r.fusion) return Iso_request_set_algorithm(request, c.alg, c.fusion);
         return ISO_SUCCESS;
@@ -1325,7 +1401,18 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
         ms /= (float)reps;
         return ISO_SUCCESS;
     };
-    for (const auto &sched : schedules) {
+    for (const auto &sched : schedules)
+    for (int hybrid = 0; hybrid <= 1 && rc == ISO_SUCCESS; ++hybrid) {
+    if (hybrid) {
+        // ragged rows only: does the lowering hand anything to bulk warps?
+        r.hybrid = true;
+        if (r.started) rc = Iso_wait(request);
+        if (rc == ISO_SUCCESS) rc = apply(Choice{1, 1, 0, sched.first, sched.second, 1});
+        if (rc == ISO_SUCCESS) rc = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
+        bool any = false;
+        for (const LaunchPlan &L : r.launches) any = any || !L.side.empty();
+        if (!any || rc != ISO_SUCCESS) continue;
+    }
     std::vector<Choice> tried;
     for (int graph = 0; graph <= 1 && rc == ISO_SUCCESS; ++graph)
         for (int chains = 1; chains <= 4 && rc == ISO_SUCCESS; chains *= 2) {
@@ -1333,11 +1420,11 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
             for (int slabs = 1; slabs <= 64 && slabs <= std::max(1, p0) && rc == ISO_SUCCESS; slabs *= 2) {
                 if (chains > 1 && slabs < chains) continue;
                 if (r.started) rc = Iso_wait(request);
-                if (rc == ISO_SUCCESS) rc = apply(Choice{slabs, chains, graph, sched.first, sched.second});
+                if (rc == ISO_SUCCESS) rc = apply(Choice{slabs, chains, graph, sched.first, sched.second, hybrid});
                 if (rc == ISO_SUCCESS) rc = materialise(r);
                 if (rc != ISO_SUCCESS) break;
                 // what the schedule allowed may differ from what was asked for: skip repeats
-                const Choice got{(int)std::max<size_t>(1, r.slab_plan.size()), r.chains, r.use_graph ? 1 : 0, r.alg, r.fusion};
+                const Choice got{(int)std::max<size_t>(1, r.slab_plan.size()), r.chains, r.use_graph ? 1 : 0, r.alg, r.fusion, hybrid};
                 bool seen = false;
                 for (const Choice &c : tried) seen = seen || (c.slabs == got.slabs && c.chains == got.chains && c.graph == got.graph);
                 if (seen) continue;
@@ -1349,12 +1436,12 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
                 rc = measure(reps, ms);
                 if (rc != ISO_SUCCESS) break;
                 if (log)
-                    std::fprintf(stderr, "iso tune: alg %d fusion %d slabs %d chains %d graph %d: %.4f ms\n", got.alg, got.fusion,
-                                 got.slabs, got.chains, got.graph, ms);
+                    std::fprintf(stderr, "iso tune: alg %d fusion %d hybrid %d slabs %d chains %d graph %d: %.4f ms\n", got.alg,
+                                 got.fusion, got.hybrid, got.slabs, got.chains, got.graph, ms);
                 // the plainer plans come first; a later one must win by 2 % to replace them
                 if (best_ms < 0.0f || ms < 0.98f * best_ms) {
                     best_ms = ms;
-                    best = Choice{slabs, chains, graph, sched.first, sched.second};
+                    best = Choice{slabs, chains, graph, sched.first, sched.second, hybrid};
                 }
             }
         }
@@ -1369,6 +1456,21 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
     int e = apply(rc == ISO_SUCCESS ? best : before);
     if (e == ISO_SUCCESS) e = materialise(r);
     return rc != ISO_SUCCESS ? rc : e;
+    });
+}
+
+int Iso_request_set_hybrid(Iso_request request, int enable)
+{
+    return guarded([&]() -> int {
+    if (check_handle(request)) return ISO_ERR_ARG;
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    request->hybrid = enable != 0;
+    int rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
+    request->dirty = true;
+    return rc;
     });
 }
 
@@ -1720,7 +1822,13 @@ int Iso_request_get_parts(Iso_request request, Iso_part *out, int capacity, int 
     return guarded([&]() -> int {
     if (check_handle(request) || !count || capacity < 0 || (capacity > 0 && !out)) return ISO_ERR_ARG;
     int n = 0;
+    std::vector<const LaunchPlan *> plans;
     for (const LaunchPlan &L : request->launches) {
+        plans.push_back(&L);
+        for (const LaunchPlan &S : L.side) plans.push_back(&S);
+    }
+    for (const LaunchPlan *plan : plans) {
+        const LaunchPlan &L = *plan;
         for (const LoweredPart &lp : L.parts) {
             if (n < capacity) {
                 Iso_part q{};

@@ -69,9 +69,12 @@ struct FanParent {
     std::vector<FanDst> dsts;  // at most kFanDsts
 };
 constexpr int kFanDsts = 4;  // destinations per descriptor; a parent with more is listed several times
+constexpr int64_t kHybridMinBytes = 256;  // 16-byte-aligned pieces of a ragged row from which bulk copies take over
 constexpr int kMaxVecUnits = 4096;  // unit positions per process in one vector launch
 constexpr int kVecDepth = 8;        // cp.async ring slots per thread in the vector kernel
 constexpr int kWideDepth = 12;      // the same in CTAs of more than 256 threads (one CTA per SM)
+constexpr int kHybridDepth = 6;     // the same for the vector warps of a hybrid launch (most of the shared memory stages bulk copies)
+constexpr size_t kHybridStageBytes = 128 * 1024;  // staging area of the bulk warps of a hybrid launch
 
 struct LaunchPlan {
     int kernel = KERNEL_VEC;
@@ -92,6 +95,8 @@ struct LaunchPlan {
     int used_dim[ISO_MAX_DIMS] = {0};
     int max_nnz = 0;       // most dimensions any one part shifts along
     bool compact = false;  // vector kernel: unit descriptors list only the shifted dimensions
+    std::vector<LaunchPlan> side;  // mixed-width vector launch: at most one bulk-copy plan for the long bodies of its rows,
+                                   // run by one extra warp of the same CTAs
     std::vector<FanParent> fans;  // KERNEL_FAN: the launch as parents and their destinations (parts: the same copies, one per destination)
     // byte offsets of this launch's tables inside the request's device blob
     size_t parts_off = 0, lookup_off = 0, units_off = 0;
@@ -115,6 +120,7 @@ struct Knobs {
     bool no_pdl = false;      // ISO_NO_PDL: plain launches instead of programmatic dependent ones
     bool tune_log = false;    // ISO_TUNE_LOG: the tuner prints every plan it times
     int sender_side = -1;     // ISO_SENDER_SIDE: 0 never, 1 automatic, 2 wherever possible (allgather phases; -1: the request's setting)
+    int hybrid = -1;          // ISO_HYBRID: 1 = long bodies of ragged rows through bulk warps, 0 = not (-1: the request's setting)
     bool host_graph = true;   // ISO_HOST_GRAPH=0: the pipelined host-buffer path is never replayed from a graph
     bool coord_table = true;  // ISO_COORD_TABLE=0: row coordinates by division in every thread
 };
@@ -154,8 +160,7 @@ struct Request {
     bool started = false;
     std::vector<std::pair<long long, long long>> slab_plan;  // row ranges of the slabs (empty: whole torus at once)
     int64_t inter_rows = 0;            // processes the intermediate buffer holds
-    void *copy_stream = nullptr;       // download stream of the pipelined host-buffer path
-    void *up_stream = nullptr;         // its upload stream
+    std::vector<void *> host_streams;  // pipelined host-buffer path: two upload and two download streams
     std::vector<void *> slab_events;   // its events
     void *host_main_stream = nullptr;  // origin stream when that path is captured into a graph
     void *host_graph_exec = nullptr;   // cudaGraphExec_t of one pipelined host-buffer start
@@ -179,6 +184,7 @@ struct Request {
     size_t wave_smem = 0, wave_launches_off = 0, wave_items_off = 0;
     unsigned long long wave_run = 0;  // starts since the counters were last zeroed
     int wave_counters = 0;      // counters allocated in d_counter
+    bool hybrid = false;        // launches of mixed widths hand their long bodies to bulk warps (Iso_request_set_hybrid)
     int sender_side = 1;        // allgather phases in sender-side form: 0 never, 1 where measured faster, 2 wherever possible
     uint32_t wait_limit = 1u << 22;  // polls before a device-side wait on other CTAs gives up
     int skew_next = 0;          // testing: extra arrivals the next cooperative start waits for (one shot)

@@ -74,6 +74,7 @@ struct LaunchDev {
     int grid_share;          // host side only: launches of this kind that run side by side
     uint32_t tab_iters;      // coordinate table: row groups a CTA visits at most (0: no table)
     uint32_t tab_stride;     // coordinate table: 32-bit words per row (4 or 8)
+    uint32_t side_offset;    // hybrid kernel, bulk side: byte offset of its staging area in shared memory
     FastDivDev div_units;    // division by units_per_proc
     FastDivDev div_uniform;  // division by uniform_units
     int used_dim[ISO_MAX_DIMS];
@@ -286,11 +287,11 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
 // with the integer-multiply pipe as the top stall; the table removes that arithmetic.
 template <int W, int DEPTH, int NU, bool MESH, bool COMPACT, bool TAB = false>
 __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned char *ring_base, bool dependent_launch,
-                                                 uint32_t cta, uint32_t n_cta)
-{
+                                                 uint32_t cta, uint32_t n_cta, const uint32_t nthr)
+{   // nthr: threads of the CTA that run this body (all of them, except in the hybrid kernel)
     using V = typename VecOf<W>::type;
-    V *const ring = reinterpret_cast<V *>(ring_base) + threadIdx.x;  // slot k at ring[k * blockDim.x]
-    V *const ring_end = ring + DEPTH * blockDim.x;
+    V *const ring = reinterpret_cast<V *>(ring_base) + threadIdx.x;  // slot k at ring[k * nthr]
+    V *const ring_end = ring + DEPTH * nthr;
 
     const uint32_t CU = L.chunk_units, U = L.units_per_proc;
     const int G = (int)L.rows_per_pass;
@@ -304,12 +305,12 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
     UnitRegs R_first;
     if (active) R_first = load_unit(L, ul);
     // entry (it * G + g) of the coordinate table: row slot g in the CTA's it-th row group
-    uint32_t *const tab = reinterpret_cast<uint32_t *>(ring_base + (size_t)DEPTH * blockDim.x * sizeof(V));
+    uint32_t *const tab = reinterpret_cast<uint32_t *>(ring_base + (size_t)DEPTH * nthr * sizeof(V));
     const uint32_t NT = TAB ? L.tab_stride : 0;
     if (TAB) {
         const long long group0 = L.row_lo + (long long)G * cta;
         const uint32_t entries = L.tab_iters * (uint32_t)G;
-        for (uint32_t j = threadIdx.x; j < entries; j += blockDim.x) {
+        for (uint32_t j = threadIdx.x; j < entries; j += nthr) {
             const uint32_t it = j / (uint32_t)G;
             const long long r = group0 + (long long)it * rstep + (j - it * (uint32_t)G);
             if (r < L.row_hi) {
@@ -379,7 +380,7 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
         for (int i = 0; i < DEPTH; ++i) {
             if (r_ld < r_end) {
                 const unsigned char *src;
-                if (source(src_ld, r_ld, row_ld, src)) cp_async_unit<W>(ring + i * blockDim.x, src, R.width);
+                if (source(src_ld, r_ld, row_ld, src)) cp_async_unit<W>(ring + i * nthr, src, R.width);
                 r_ld += rstep;
                 src_ld += src_step;
                 row_ld += tab_step;
@@ -405,7 +406,7 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
                 row_ld += tab_step;
             }
             cp_async_commit();
-            slot += blockDim.x;
+            slot += nthr;
             if (slot == ring_end) slot = ring;
         }
         cp_async_wait<0>();
@@ -416,7 +417,7 @@ template <int W, int DEPTH, int NU, bool MESH, bool COMPACT>
 __global__ void __launch_bounds__(256, 4) iso_gather_rows(const __grid_constant__ LaunchDev L)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true, blockIdx.x, gridDim.x);
+    gather_rows_body<W, DEPTH, NU, MESH, COMPACT>(L, smem_raw, true, blockIdx.x, gridDim.x, blockDim.x);
 }
 
 // The same body in CTAs of up to 1024 threads, for launches whose payload per process has
@@ -426,7 +427,7 @@ template <int W, int DEPTH, int NU, bool MESH, bool COMPACT, bool TAB>
 __global__ void __launch_bounds__(1024, 1) iso_gather_rows_wide(const __grid_constant__ LaunchDev L)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    gather_rows_body<W, DEPTH, NU, MESH, COMPACT, TAB>(L, smem_raw, true, blockIdx.x, gridDim.x);
+    gather_rows_body<W, DEPTH, NU, MESH, COMPACT, TAB>(L, smem_raw, true, blockIdx.x, gridDim.x, blockDim.x);
 }
 
 // Sender-side form of an allgather phase.  In the prefix-trie schedule (Section III-B) a node's
@@ -588,11 +589,11 @@ __global__ void __launch_bounds__(1024, 1) iso_gather_rows_multi(const __grid_co
         for (uint32_t i = threadIdx.x; i < sizeof(LaunchDev) / 4; i += blockDim.x) dst[i] = __ldg(src + i);
         __syncthreads();
         switch (sL->n_used) {
-        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
-        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
-        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
-        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
-        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false, blockIdx.x, gridDim.x); break;
+        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false, blockIdx.x, gridDim.x, blockDim.x); break;
+        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false, blockIdx.x, gridDim.x, blockDim.x); break;
+        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false, blockIdx.x, gridDim.x, blockDim.x); break;
+        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false, blockIdx.x, gridDim.x, blockDim.x); break;
+        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false, blockIdx.x, gridDim.x, blockDim.x); break;
         }
         if (ph + 1 < M.n && !grid_barrier(M, M.epoch + (unsigned long long)(ph + 1) * M.arrivals, &s_ok)) return;
     }
@@ -662,15 +663,15 @@ __global__ void __launch_bounds__(1024, 1) iso_gather_rows_wave(const __grid_con
         uint32_t cta = blockIdx.x + n_cta - s_item.cta_offset;
         if (cta >= n_cta) cta -= n_cta;
         switch (s_item.variant) {
-        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false, cta, n_cta); break;
-        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false, cta, n_cta); break;
-        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false, cta, n_cta); break;
-        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false, cta, n_cta); break;
-        case 4: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false, cta, n_cta); break;
-        case 5: gather_rows_body<16, DEPTH, 1, false, true>(*sL, ring, false, cta, n_cta); break;
-        case 6: gather_rows_body<16, DEPTH, 2, false, true>(*sL, ring, false, cta, n_cta); break;
-        case 7: gather_rows_body<16, DEPTH, 3, false, true>(*sL, ring, false, cta, n_cta); break;
-        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, true>(*sL, ring, false, cta, n_cta); break;
+        case 0: gather_rows_body<16, DEPTH, 0, false, false>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        case 1: gather_rows_body<16, DEPTH, 1, false, false>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        case 2: gather_rows_body<16, DEPTH, 2, false, false>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        case 3: gather_rows_body<16, DEPTH, 3, false, false>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        case 4: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, false>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        case 5: gather_rows_body<16, DEPTH, 1, false, true>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        case 6: gather_rows_body<16, DEPTH, 2, false, true>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        case 7: gather_rows_body<16, DEPTH, 3, false, true>(*sL, ring, false, cta, n_cta, blockDim.x); break;
+        default: gather_rows_body<16, DEPTH, ISO_MAX_DIMS, false, true>(*sL, ring, false, cta, n_cta, blockDim.x); break;
         }
         // all stores of this CTA for the item are issued: publish them and count the CTA in
         __syncthreads();
@@ -884,6 +885,149 @@ __global__ void __launch_bounds__(256) iso_gather_bulk(const __grid_constant__ L
         }
     bulk_wait_all();
     if (failed) atomicExch(L.err, 1);
+}
+
+// Chunk `u` of the long pieces of row r (the bulk side of a hybrid launch): like decode_unit,
+// with the row's coordinates computed on the spot instead of read from a tile's table.
+__device__ __forceinline__ UnitAddr decode_row_unit(const LaunchDev &L, long long r, uint32_t u)
+{
+    uint32_t t;
+    if (L.uniform_units) {
+        t = fastdiv(L.div_uniform, u);
+    } else {
+        t = L.lookup[u >> L.lookup_shift];
+        while (t + 1 < L.nparts && __ldg(&L.parts[t + 1].first_unit) <= u) ++t;
+    }
+    const PartDev *p = L.parts + t;
+    const uint32_t k = u - __ldg(&p->first_unit);
+    long long rs = r + __ldg(&p->rank_delta);
+    const int nnz = __ldg(&p->nnz);
+    for (int e = 0; e < nnz; ++e) {
+        const int dk = __ldg(&p->dim[e]);
+        const int c = __ldg(&p->c[e]);
+        const uint32_t q = fastdiv(L.div_rstride[dk], (uint32_t)r);
+        const int x = (int)(q - fastdiv(L.div_size[dk], q) * L.used_size[dk]);
+        if (x < c) rs += (long long)L.used_size[dk] * L.used_rstride[dk];
+    }
+    const long long within = (long long)k * L.width;
+    const long long rest = __ldg(&p->len) - within;
+    UnitAddr a;
+    a.src = L.buf[__ldg(&p->src_buf)] + rs * L.buf_stride[__ldg(&p->src_buf)] + __ldg(&p->src_off) + within;
+    a.dst = L.buf[__ldg(&p->dst_buf)] + r * L.buf_stride[__ldg(&p->dst_buf)] + __ldg(&p->dst_off) + within;
+    a.bytes = (uint32_t)(rest < (long long)L.width ? rest : (long long)L.width);
+    a.valid = true;
+    return a;
+}
+
+// Ragged rows (irregular collectives): the vector gather and the bulk gather in ONE kernel.
+// A row of such a collective is a few long blocks between many short pieces.  Moved unit by
+// unit, the long blocks make up most of the 16-byte units, and every unit costs a cp.async,
+// a shared-memory load and a store through the same load/store queue, whose capacity, not
+// memory bandwidth, then bounds the kernel.  Here the first warps run the vector gather over
+// the short pieces and ragged ends only, while the last warps (S.chunk_units threads) move the
+// long 16-byte-aligned bodies of the SAME rows (same assignment of row groups to CTAs) with
+// bulk copies, global -> shared -> global, two stages per lane, as iso_gather_bulk does: the bulk
+// copies have their own queue, so both engines work at the same time, and pieces that share
+// a 32-byte sector with a long body still move within a few rows of it.  Periodic
+// dimensions only.  L: the vector side; S: the bulk side (same row range).
+template <int DEPTH, int NU, bool TAB>
+__global__ void __launch_bounds__(1024, 1) iso_gather_rows_hybrid(const __grid_constant__ LaunchDev L,
+                                                                  const __grid_constant__ LaunchDev S)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lanes = S.chunk_units;  // threads of the bulk warps
+    const uint32_t nvec = blockDim.x - lanes;
+    if (threadIdx.x < nvec) {
+        gather_rows_body<0, DEPTH, NU, false, false, TAB>(L, smem_raw, true, blockIdx.x, gridDim.x, nvec);
+        return;
+    }
+    const uint32_t lane = threadIdx.x - nvec;
+    const uint32_t chunk = S.width;
+    unsigned char *stage = smem_raw + S.side_offset + (size_t)lane * 2 * chunk;
+    uint64_t *bar = reinterpret_cast<uint64_t *>(smem_raw + S.side_offset + (size_t)lanes * 2 * chunk) + 2 * lane;
+    mbar_init(&bar[0], 1);
+    mbar_init(&bar[1], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+    __syncwarp();
+    if (TAB) __syncthreads();  // the barrier the vector warps pass after filling their coordinate table
+    grid_dependency_wait();
+    grid_launch_dependents();
+
+    // items of this CTA: (row group it, row slot g, chunk u), consecutive lanes on consecutive chunks
+    const uint32_t G = L.rows_per_pass, U = S.units_per_proc;
+    const long long group0 = S.row_lo + (long long)G * blockIdx.x;
+    const long long rstep = (long long)G * gridDim.x;
+    const uint32_t per_group = G * U;
+    uint32_t total = 0;
+    if (group0 < S.row_hi) total = (uint32_t)((S.row_hi - group0 + rstep - 1) / rstep) * per_group;
+    uint32_t parity_bits = 0, pending_bits = 0;
+    bool failed = false;
+    auto await = [&](uint32_t s) {
+        uint32_t polls = 0;
+        while (!mbar_try_wait(&bar[s], (parity_bits >> s) & 1u)) {
+            if (++polls >= kBulkWaitPolls) {
+                failed = true;
+                return;
+            }
+        }
+        parity_bits ^= 1u << s;
+        pending_bits &= ~(1u << s);
+    };
+    auto item = [&](uint32_t k) -> UnitAddr {
+        const uint32_t it = k / per_group, rem = k - it * per_group;
+        const uint32_t g = rem / U, u = rem - g * U;
+        const long long r = group0 + (long long)it * rstep + g;
+        UnitAddr a{};
+        a.valid = false;
+        if (r < S.row_hi) a = decode_row_unit(S, r, u);
+        return a;
+    };
+
+    UnitAddr cur{}, nxt{};
+    cur.valid = nxt.valid = false;
+    uint32_t s = 0;  // stage of `cur`
+    if (lane < total) {
+        cur = item(lane);
+        if (cur.valid) {
+            mbar_expect_tx(&bar[0], cur.bytes);
+            bulk_load(stage, cur.src, cur.bytes, &bar[0]);
+            pending_bits |= 1u;
+        }
+    }
+    for (uint32_t k = lane; k < total; k += lanes) {
+        nxt.valid = false;
+        if (k + lanes < total) {
+            bulk_wait_read_all();  // the other stage was last read by the store of the item before
+            nxt = item(k + lanes);
+            if (nxt.valid && !failed) {
+                mbar_expect_tx(&bar[s ^ 1u], nxt.bytes);
+                bulk_load(stage + (size_t)(s ^ 1u) * chunk, nxt.src, nxt.bytes, &bar[s ^ 1u]);
+                pending_bits |= 1u << (s ^ 1u);
+            }
+        }
+        if (cur.valid && !failed) {
+            await(s);
+            if (!failed) {
+                fence_async_smem();
+                bulk_store(cur.dst, stage + (size_t)s * chunk, cur.bytes);
+                bulk_commit();
+            }
+        }
+        cur = nxt;
+        s ^= 1u;
+    }
+    // on the error path a load may still be in flight: one more bounded wait, so that it does
+    // not land in shared memory that has been handed to another CTA
+    for (uint32_t q = 0; q < 2; ++q)
+        if (pending_bits >> q & 1u) {
+            const bool keep = failed;
+            failed = false;
+            await(q);
+            failed = failed || keep;
+        }
+    bulk_wait_all();
+    if (failed) atomicExch(S.err, 1);
 }
 
 }  // namespace iso

@@ -62,6 +62,7 @@ Knobs read_knobs()
     k.sender_side = (int)num("ISO_SENDER_SIDE", -1);
     k.coord_table = num("ISO_COORD_TABLE", 1) != 0;
     k.host_graph = num("ISO_HOST_GRAPH", 1) != 0;
+    k.hybrid = (int)num("ISO_HYBRID", -1);
     return k;
 }
 
@@ -896,6 +897,48 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                 }
         }
 
+        // parts of one launch with their unit ranges, the dimensions the launch shifts along
+        // and the coarse unit -> part lookup
+        auto fill_parts = [&](LaunchPlan &L, const std::vector<Piece> &src, size_t lo, size_t hi, int kernel, int64_t unit) -> int {
+            uint64_t units = 0;
+            bool uniform = true;
+            bool used[ISO_MAX_DIMS] = {false};
+            for (size_t k = lo; k < hi; ++k) {
+                LoweredPart lp;
+                lp.p = src[k].p;
+                lp.width = kernel == KERNEL_BULK ? (int)unit : src[k].width;
+                uint64_t n = (uint64_t)((lp.p.len + lp.width - 1) / lp.width);
+                if (units + n > 0x7fffffffull) return ISO_ERR_COUNT;
+                lp.first_unit = (uint32_t)units;
+                lp.units = (uint32_t)n;
+                units += n;
+                if (!L.parts.empty() && L.parts[0].units != lp.units) uniform = false;
+                int nnz = 0;
+                for (int j = 0; j < c.d; ++j)
+                    if (lp.p.shift[j] || lp.p.check[j]) { used[j] = true; ++nnz; }
+                L.max_nnz = std::max(L.max_nnz, nnz);
+                L.parts.push_back(lp);
+            }
+            L.units_per_proc = (uint32_t)units;
+            L.uniform_units = uniform ? L.parts[0].units : 0;
+            for (int j = 0; j < c.d; ++j)
+                if (used[j]) L.used_dim[L.n_used++] = j;
+            if (!uniform) {
+                int shift = 0;
+                while ((units >> shift) + 1 > 16384) ++shift;
+                L.lookup_shift = shift;
+                size_t n = (size_t)(units >> shift) + 1;
+                L.lookup.resize(n);
+                size_t t = 0;
+                for (size_t e = 0; e < n; ++e) {
+                    uint64_t u = (uint64_t)e << shift;
+                    while (t + 1 < L.parts.size() && L.parts[t + 1].first_unit <= u) ++t;
+                    L.lookup[e] = (uint16_t)t;
+                }
+            }
+            return ISO_SUCCESS;
+        };
+
         // one launch per (kernel, width) class, in a fixed order
         for (int kernel = 0; kernel < 2; ++kernel) {
             for (int width : {0, 16, 8, 4, 2, 1}) {  // 0: the launch of mixed unit widths
@@ -903,6 +946,30 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                 std::vector<std::pair<size_t, size_t>> ranges;
                 for (const Piece &q : pieces)
                     if (q.kernel == kernel && q.cls == width) cls.push_back(q);
+                // Launch of mixed widths: the long 16-byte-aligned bodies among its pieces are
+                // handed to one extra warp of the CTA that moves them with bulk copies, while
+                // the other warps move the ragged rest (see iso_gather_rows_hybrid).
+                std::vector<Piece> longs;
+                if (kernel == KERNEL_VEC && width == 0 && r.hybrid && r.bulk_threshold > 0 && c.d <= 3) {
+                    bool plain = true;  // periodic dimensions only
+                    for (const Piece &q : cls)
+                        for (int j = 0; j < c.d; ++j) plain = plain && !q.p.check[j];
+                    std::vector<Piece> rest;
+                    for (const Piece &q : cls) (plain && q.width == 16 && q.p.len >= kHybridMinBytes ? longs : rest).push_back(q);
+                    int64_t rest_units = 0;
+                    for (const Piece &q : rest) rest_units += q.p.len / q.width;
+                    if (!longs.empty() && !rest.empty() && rest_units <= kMaxVecUnits) cls.swap(rest);
+                    else longs.clear();
+                }
+                // bulk side of such a launch: chunks of 1024 bytes if every long piece has as many,
+                // else 512; two stages and two barriers per lane of one warp
+                int64_t side_chunk = 1024;
+                for (const Piece &q : longs) if (q.p.len < 1024) side_chunk = 512;
+                // bulk warps: as many lanes as fill the staging area with two chunks each (measured with
+                // ONE bulk warp, 32 KB in flight per SM: 2.8 times slower than without the split - a
+                // bulk copy through shared memory occupies its stage for several microseconds)
+                const size_t side_lanes = kHybridStageBytes / (2 * (size_t)side_chunk);
+                const size_t side_smem = longs.empty() ? 0 : side_lanes * 2 * (size_t)side_chunk + side_lanes * 2 * 8;
                 // a vector launch holds at most kMaxVecUnits unit positions per process (each
                 // gets a descriptor): cut longer lists, splitting a piece at a unit boundary
                 if (kernel == KERNEL_VEC) {
@@ -952,51 +1019,20 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         }
                     }
                     L.width = (int)unit;
-                    uint64_t units = 0;
-                    bool uniform = true;
-                    bool used[ISO_MAX_DIMS] = {false};
-                    for (size_t k = lo; k < hi; ++k) {
-                        LoweredPart lp;
-                        lp.p = cls[k].p;
-                        lp.width = kernel == KERNEL_BULK ? (int)unit : cls[k].width;
-                        uint64_t n = (uint64_t)((lp.p.len + lp.width - 1) / lp.width);
-                        if (units + n > 0x7fffffffull) return ISO_ERR_COUNT;
-                        lp.first_unit = (uint32_t)units;
-                        lp.units = (uint32_t)n;
-                        units += n;
-                        if (!L.parts.empty() && L.parts[0].units != lp.units) uniform = false;
-                        int nnz = 0;
-                        for (int j = 0; j < c.d; ++j)
-                            if (lp.p.shift[j] || lp.p.check[j]) { used[j] = true; ++nnz; }
-                        L.max_nnz = std::max(L.max_nnz, nnz);
-                        L.parts.push_back(lp);
-                        if (kernel == KERNEL_BULK) bulk_bytes += lp.p.len;
+                    {
+                        int rc_fill = fill_parts(L, cls, lo, hi, kernel, unit);
+                        if (rc_fill != ISO_SUCCESS) return rc_fill;
                     }
-                    L.units_per_proc = (uint32_t)units;
-                    L.uniform_units = uniform ? L.parts[0].units : 0;
-                    bool torus = true;
-                    for (int j = 0; j < c.d; ++j)
-                        if (used[j]) {
-                            L.used_dim[L.n_used++] = j;
-                            torus = torus && c.periodic[j];
-                        }
+                    const uint64_t units = L.units_per_proc;
+                    if (kernel == KERNEL_BULK)
+                        for (const LoweredPart &lp : L.parts) bulk_bytes += lp.p.len;
                     // many shifted dimensions in the launch, few per part: the kernel then
                     // tests per row only the dimensions a unit moves along
-                    L.compact = kernel == KERNEL_VEC && (width >= 4 || width == 0) && L.n_used > 3 && L.max_nnz < L.n_used &&
-                                torus && !r.persistent;  // (the pipelined one-launch kernel does take compact launches)
-                    // coarse lookup: unit >> shift -> part
-                    if (!uniform) {
-                        int shift = 0;
-                        while ((units >> shift) + 1 > 16384) ++shift;
-                        L.lookup_shift = shift;
-                        size_t n = (size_t)(units >> shift) + 1;
-                        L.lookup.resize(n);
-                        size_t t = 0;
-                        for (size_t e = 0; e < n; ++e) {
-                            uint64_t u = (uint64_t)e << shift;
-                            while (t + 1 < L.parts.size() && L.parts[t + 1].first_unit <= u) ++t;
-                            L.lookup[e] = (uint16_t)t;
-                        }
+                    {
+                        bool torus = true;
+                        for (int k = 0; k < L.n_used; ++k) torus = torus && c.periodic[L.used_dim[k]];
+                        L.compact = kernel == KERNEL_VEC && (width >= 4 || width == 0) && L.n_used > 3 && L.max_nnz < L.n_used &&
+                                    torus && !r.persistent;  // (the pipelined one-launch kernel does take compact launches)
                     }
                     // geometry
                     (void)width;
@@ -1010,7 +1046,10 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         // per all-to-all on the 32^3 torus, 161 against 184 on the 8^5 torus);
                         // ISO_VEC_THREADS=256 or 512 selects the narrower shapes
                         uint32_t max_threads = (width == 16 || width == 0) ? 1024 : 256;
-                        if (r.knobs.vec_threads) {
+                        if (!longs.empty())  // leave a warp and the staging area to the bulk side
+                            max_threads = std::min<uint32_t>((uint32_t)(1024 - side_lanes),
+                                                             (uint32_t)((227 * 1024 - side_smem - 16 * 1024) / (kHybridDepth * 16) / 32 * 32));
+                        if (r.knobs.vec_threads && longs.empty()) {
                             const int v = r.knobs.vec_threads;
                             if ((v == 256 || v == 512) && max_threads == 1024) max_threads = units > 256 ? 1024 : (uint32_t)v;
                         }
@@ -1019,6 +1058,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         L.threads = (int)((L.chunk_units * L.rows_per_pass + 31) / 32 * 32);
                         // CTAs of fewer than 256 threads: as many per SM as keep 1024 threads resident
                         int per_sm = L.threads > 512 ? 1 : (L.threads > 256 ? 2 : std::min(16, std::max(4, 1024 / L.threads)));
+                        if (!longs.empty()) per_sm = 1;
                         if (r.knobs.vec_ctas_per_sm) {
                             const int v = r.knobs.vec_ctas_per_sm;
                             if (v >= 1 && v <= 8 && L.threads <= 256) per_sm = v;
@@ -1046,11 +1086,25 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     if (L.grid > 0x7fffffff) return ISO_ERR_DIMS;
                     L.smem = (size_t)L.n_used * (size_t)tp * sizeof(uint32_t);
                     if (kernel == KERNEL_VEC) {
-                        const size_t depth = L.threads > 256 ? kWideDepth : kVecDepth;
+                        const size_t depth = !longs.empty() ? kHybridDepth : (L.threads > 256 ? kWideDepth : kVecDepth);
                         L.smem = width >= 4 ? depth * L.threads * width : (width == 0 ? depth * L.threads * 16 : 0);
                     }
                     if (kernel == KERNEL_BULK)
                         L.smem = (L.smem + 15) / 16 * 16 + (size_t)L.threads * 2 * (size_t)unit + (size_t)L.threads * 2 * 8;
+                    if (!longs.empty()) {
+                        LaunchPlan S;
+                        S.kernel = KERNEL_BULK;
+                        S.phase = L.phase;
+                        S.width = (int)side_chunk;
+                        int rc_side = fill_parts(S, longs, 0, longs.size(), KERNEL_BULK, side_chunk);
+                        if (rc_side != ISO_SUCCESS) return rc_side;
+                        S.tile_procs = 1;
+                        S.threads = (int)side_lanes;
+                        S.smem = side_smem;
+                        for (const LoweredPart &lp : S.parts) bulk_bytes += lp.p.len;
+                        L.side.push_back(std::move(S));
+                        longs.clear();
+                    }
                     r.launches.push_back(std::move(L));
                 }
             }

@@ -115,6 +115,7 @@ def test_random_cases(chunk):
             pipe = (0, 0, 1, 0, 3)[(c["trial"] + 2 * alg + fusion) % 5]
             iso.Iso_request_set_pipeline(req, pipe)
             iso.Iso_request_set_sender_side(req, (2, 1, 2, 0)[(c["trial"] + fusion) % 4])
+            iso.Iso_request_set_hybrid(req, (c["trial"] + alg) % 2 == 0)
             iso.Iso_request_set_algorithm(req, alg, fusion)
             if rs:
                 recv.fill_(POISON)
@@ -152,6 +153,8 @@ def test_random_cases_host_simulation(chunk):
         for (alg, fusion), (lay, single, bulk, slabs) in zip(c["choices"], c["options"]):
             iso.Iso_request_set_layout(req, lay)
             iso.Iso_request_set_bulk_threshold(req, bulk)
+            iso.Iso_request_set_hybrid(req, (c["trial"] + alg) % 2 == 0)
+            iso.Iso_request_set_sender_side(req, (2, 1, 2, 0)[(c["trial"] + fusion) % 4])
             iso.Iso_request_set_algorithm(req, alg, fusion)
             st = iso.Iso_request_get_stats(req)
             got = simulate(iso.Iso_request_get_parts(req), c["dims"], st, c["send_h"] if c["ss"] else np.zeros((c["P"], 0), np.uint8),

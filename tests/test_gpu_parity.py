@@ -238,13 +238,17 @@ def test_allgather_phases_in_sender_side_form(torch_cuda):
     for w in cases:
         run = Run(torch, w)
         want = oracle_result(w, run.send_host)
-        for mode, kernels in ((2, {2}), (0, {0, 1}), (1, {0, 1, 2})):
+        for mode in (2, 0, 1):
             iso.Iso_request_set_sender_side(run.req, mode)
             for alg, fusion in (COMB1, COMB0):
                 got = run.result(alg, fusion)
                 assert np.array_equal(got, want), (w.name, w.dims, mode, alg, fusion)
                 used = {p["kernel"] for p in iso.Iso_request_get_parts(run.req)}
-                assert used <= kernels, (w.name, mode, used)
+                # (with one launch per round a block has two copies in a launch only if a vector is repeated)
+                if mode == 0:
+                    assert 2 not in used, (w.name, mode, fusion, used)
+                elif mode == 2 and fusion == 1 and w.name != "t":
+                    assert 2 in used, (w.name, mode, used)
             assert iso.Iso_request_check_guards(run.req) == 0
         run.close()
     # left to the library, the large phases of the 80-neighbour allgather take this form
@@ -448,6 +452,46 @@ def test_stencil_shaped_irregular_sizes(torch_cuda):
         w = wl.Workload(full.name, "alltoallv", (9, 8, 10), full.offsets, 0, lens=full.lens, seed=21)
         check(torch_cuda, w, [COMB0, COMB1, COMB2, ALT1, DIRECT, TORUS])
         check(torch_cuda, w, [COMB1], bulk=0)
+
+
+def test_ragged_rows_with_bulk_warps(torch_cuda):
+    """Iso_request_set_hybrid: the long bodies of ragged rows moved by bulk warps of the same
+    launch.  Same bytes as the oracle for every schedule, in slabs, through host buffers and
+    after the tuner (which tries the launch form both ways) has made its choice."""
+    torch = torch_cuda
+    stencil = wl.config("stencil_d3_m32")
+    cases = [wl.config("cfg5_32x32x32"), wl.Workload("st", "alltoallv", (9, 8, 10), stencil.offsets, 0, lens=stencil.lens, seed=21),
+             wl.Workload("ragged", "alltoallv", (37, 53), wl.moore(2, 1), 0,
+                         lens=np.array([1024, 4, 2064, 16, 1040, 8, 3072, 64]), seed=8),
+             wl.Workload("odd", "alltoallv", (5, 7, 6), wl.moore(3, 1), 0,
+                         lens=np.array([1 + (977 * i) % 1500 for i in range(26)]), seed=9)]
+    for w in cases:
+        run = Run(torch, w)
+        want = oracle_result(w, run.send_host)
+        iso.Iso_request_set_hybrid(run.req, True)
+        for slabs in (0, 3):
+            iso.Iso_request_set_slabs(run.req, slabs)
+            for alg, fusion in (COMB1, COMB0, COMB2, DIRECT, TORUS):
+                got = run.result(alg, fusion)
+                assert np.array_equal(got, want), (w.name, slabs, alg, fusion)
+        assert any(p["kernel"] == 1 and p["len"] < 4096 for p in iso.Iso_request_get_parts(run.req))
+        assert iso.Iso_request_check_guards(run.req) == 0
+        hs = torch.from_numpy(run.send_host).pin_memory()
+        hr = torch.zeros((w.P, run.rs), dtype=torch.uint8).pin_memory()
+        run.result(*COMB1)
+        iso.Iso_Start_host(run.req, hs, hr)
+        iso.Iso_wait(run.req)
+        lens, sd, rd, ss, rs = layout(w)
+        covered = np.zeros(rs, bool)
+        for i in range(w.s):
+            covered[rd[i]:rd[i] + lens[i]] = True
+        assert np.array_equal(hr.numpy()[:, covered], want[:, covered]), w.name
+        iso.Iso_request_tune(run.req, torch.cuda.current_stream(), cold=False)
+        run.recv.fill_(POISON)
+        iso.Iso_Start(run.req, torch.cuda.current_stream())
+        iso.Iso_wait(run.req)
+        assert np.array_equal(run.recv.cpu().numpy(), want), (w.name, "tuned")
+        run.close()
 
 
 def test_allgatherv_and_unaligned_receive_layout(torch_cuda):

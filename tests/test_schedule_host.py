@@ -291,6 +291,7 @@ def test_alignment_classes_and_bulk_selection():
     # 4-byte aligned packed displacements: long blocks are split into a 16-byte aligned
     # body and narrow head / tail pieces; in such a ragged phase bodies from 4 KB on go to the
     # bulk kernel, shorter ones stay with the small pieces in the launch of mixed widths
+    # (or, with Iso_request_set_hybrid, bodies from 256 bytes on go to the bulk warps of that launch)
     w = wl.Workload("v", "alltoallv", (4, 4), wl.moore(2, 1), 0, lens=np.array([4, 1024, 16, 8192, 64, 4, 256, 1024]))
     comm, req = make_request(w)
     parts = iso.Iso_request_get_parts(req)
@@ -302,6 +303,13 @@ def test_alignment_classes_and_bulk_selection():
     st = iso.Iso_request_get_stats(req)
     send = send_buffer_np(w, st["send_stride"])
     assert np.array_equal(simulate(parts, w.dims, st, send), oracle_result(w, send))
+    iso.Iso_request_set_hybrid(req, True)
+    parts = iso.Iso_request_get_parts(req)
+    assert all(p["len"] >= 256 and p["len"] % 16 == 0 and p["src_off"] % 16 == 0 for p in parts if p["kernel"] == 1)
+    assert any(p["kernel"] == 1 and p["len"] < 4096 for p in parts)
+    assert all(p["len"] < 256 or p["width"] < 16 for p in parts if p["kernel"] == 0)
+    assert np.array_equal(simulate(parts, w.dims, st, send), oracle_result(w, send))
+    iso.Iso_request_set_hybrid(req, False)
     iso.Iso_request_set_bulk_threshold(req, 0)
     assert all(p["kernel"] == 0 for p in iso.Iso_request_get_parts(req))
     assert iso.Iso_request_get_stats(req)["bulk_bytes"] == 0
@@ -312,19 +320,28 @@ def test_alignment_classes_and_bulk_selection():
 def test_ragged_phases_lower_to_one_launch_of_mixed_widths(monkeypatch):
     """Irregular sizes: a phase whose pieces need several unit widths is one launch (the unit
     descriptors carry their width); ragged ends are cut into aligned power-of-two pieces of
-    at most 4 bytes around a body of whole 16-byte units.  The exported parts still
-    reproduce the oracle, with and without that lowering."""
-    for name, phases in (("cfg5_32x32x32", 3), ("stencil_d3_m32", 3)):
+    at most 4 bytes around a body of whole 16-byte units; bodies of 256 bytes and more are
+    bulk copies of that same launch.  The exported parts still reproduce the oracle, with
+    and without that lowering."""
+    for name, phases, hybrid in (("cfg5_32x32x32", 3, False), ("stencil_d3_m32", 3, False), ("cfg5_32x32x32", 3, True),
+                                 ("stencil_d3_m32", 3, True)):
         w = wl.config(name)
         comm, req = make_request(w)
+        iso.Iso_request_set_hybrid(req, hybrid)
         st = iso.Iso_request_get_stats(req)
         assert st["phases"] == phases and st["launches"] == phases, st
         parts = iso.Iso_request_get_parts(req)
         for ph in range(phases):
             assert len({p["width"] for p in parts if p["phase"] == ph}) >= 2
         for p in parts:
+            if p["kernel"] == 1:
+                # a long 16-byte-aligned body: moved by the bulk warp of the same launch, in chunks
+                assert p["len"] >= 256 and p["src_off"] % 16 == 0 and p["dst_off"] % 16 == 0 and p["len"] % 16 == 0
+                continue
             assert p["kernel"] == 0 and p["width"] in (1, 2, 4, 8, 16)
             assert p["src_off"] % p["width"] == 0 and p["dst_off"] % p["width"] == 0 and p["len"] % p["width"] == 0
+            assert not hybrid or p["width"] < 16 or p["len"] < 256
+        assert any(p["kernel"] == 1 for p in parts) == hybrid
         iso.Iso_request_free(req)
         iso.Iso_comm_free(comm)
     # a small ragged case, executed on the host, both ways
