@@ -437,6 +437,7 @@ LaunchDev make_launch_args(const Request &r, const LaunchPlan &L)
     a.n_used = L.n_used;
     a.mesh_mask = 0;
     a.grid_share = 1;
+    a.col_split = (uint32_t)L.col_split;
     FastDiv f = make_fastdiv(L.units_per_proc);
     a.div_units = FastDivDev{f.m, f.s1, f.s2, f.div};
     f = make_fastdiv(L.uniform_units ? L.uniform_units : 1);
@@ -533,11 +534,13 @@ int build_wave(Request &r, unsigned char *blob, size_t launches_off, size_t item
 unsigned grid_for_rows(const LaunchPlan &L, const LaunchDev &a, int share = 1)
 {
     const long long rows = a.row_hi - a.row_lo;
-    if (rows >= a.P) return (unsigned)L.grid;
+    if (rows >= a.P && share <= 1) return (unsigned)L.grid;
     if (L.kernel == KERNEL_BULK) return (unsigned)((rows + L.tile_procs - 1) / L.tile_procs);
     const long long groups = (rows + L.rows_per_pass - 1) / L.rows_per_pass;
     // `share` launches of this kind run side by side: each takes its part of the CTA slots
     const long long full = std::max<long long>(1, L.grid / std::max(1, share));
+    if (L.col_split > 1)  // CTAs per column chunk x chunks
+        return (unsigned)(std::max<long long>(1, std::min<long long>(full / L.col_split, groups)) * L.col_split);
     const long long g = std::max<long long>(1, std::min<long long>(full, groups));
     return (unsigned)g;
 }
@@ -690,7 +693,7 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
         if ((L.width == 16 || L.width == 0) && L.threads > 256 && L.n_used > 0 && r.knobs.coord_table &&
             (L.compact || nu <= 2) && !a.mesh_mask) {
             const long long groups = (a.row_hi - a.row_lo + L.rows_per_pass - 1) / L.rows_per_pass;
-            const long long grid = grid_for_rows(L, a, a.grid_share);
+            const long long grid = grid_for_rows(L, a, a.grid_share) / std::max(1, L.col_split);  // CTAs that share the rows
             a.tab_iters = (uint32_t)((groups + grid - 1) / grid);
             a.tab_stride = L.n_used <= 4 ? 4 : 8;
             tab = L.smem + table_bytes(a) <= (size_t)kMaxDynamicSmem;
@@ -955,7 +958,7 @@ void choose_slab_plan(Request &r)
         long long rows_per_pass = 1;
         for (const LaunchPlan &L : r.launches) {
             if (L.kernel != KERNEL_VEC) return;
-            rows_per_pass = std::max<long long>(rows_per_pass, (long long)L.grid * L.rows_per_pass);
+            rows_per_pass = std::max<long long>(rows_per_pass, L.rows_hint > 0 ? (long long)L.rows_hint : (long long)L.grid * L.rows_per_pass);
         }
         const double est_us = (double)r.stats.bytes_moved / 5.5e6;
         const double per = est_us / (12.0 * (double)std::max<size_t>(1, r.launches.size()));

@@ -95,6 +95,8 @@ struct LaunchPlan {
     int used_dim[ISO_MAX_DIMS] = {0};
     int max_nnz = 0;       // most dimensions any one part shifts along
     bool compact = false;  // vector kernel: unit descriptors list only the shifted dimensions
+    int64_t rows_hint = 0; // vector kernel: rows the grid holds at a time when CTAs cover whole rows (slab heuristic)
+    int col_split = 1;     // vector kernel: column chunks of a row longer than a CTA, one CTA per chunk and row (1: none)
     std::vector<LaunchPlan> side;  // mixed-width vector launch: at most one bulk-copy plan for the long bodies of its rows,
                                    // run by one extra warp of the same CTAs
     std::vector<FanParent> fans;  // KERNEL_FAN: the launch as parents and their destinations (parts: the same copies, one per destination)
@@ -121,6 +123,7 @@ struct Knobs {
     bool tune_log = false;    // ISO_TUNE_LOG: the tuner prints every plan it times
     int sender_side = -1;     // ISO_SENDER_SIDE: 0 never, 1 automatic, 2 wherever possible (allgather phases; -1: the request's setting)
     int hybrid = -1;          // ISO_HYBRID: 1 = long bodies of ragged rows through bulk warps, 0 = not (-1: the request's setting)
+    bool col_split = true;    // ISO_COL_SPLIT=0: rows longer than a CTA are covered in passes instead of column chunks
     bool host_graph = true;   // ISO_HOST_GRAPH=0: the pipelined host-buffer path is never replayed from a graph
     bool coord_table = true;  // ISO_COORD_TABLE=0: row coordinates by division in every thread
 };

@@ -75,6 +75,7 @@ struct LaunchDev {
     uint32_t tab_iters;      // coordinate table: row groups a CTA visits at most (0: no table)
     uint32_t tab_stride;     // coordinate table: 32-bit words per row (4 or 8)
     uint32_t side_offset;    // hybrid kernel, bulk side: byte offset of its staging area in shared memory
+    uint32_t col_split;      // vector kernel: column chunks the CTAs are dealt to (0 or 1: a CTA covers whole rows)
     FastDivDev div_units;    // division by units_per_proc
     FastDivDev div_uniform;  // division by uniform_units
     int used_dim[ISO_MAX_DIMS];
@@ -296,9 +297,16 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
     const uint32_t CU = L.chunk_units, U = L.units_per_proc;
     const int G = (int)L.rows_per_pass;
     const int g = (int)(threadIdx.x / CU);
-    const uint32_t ul = threadIdx.x - (uint32_t)g * CU;
+    // Rows longer than a CTA (col_split = n > 1): instead of covering a row in n passes - each
+    // a fresh ramp and drain of the ring over the few rows a CTA has - the CTAs are dealt to n
+    // column chunks: CTA b owns chunk b mod n and takes every (grid / n)-th row, in one pass.
+    const uint32_t ncol = L.col_split > 1 ? L.col_split : 1;
+    const uint32_t col = cta % ncol;
+    cta /= ncol;
+    n_cta /= ncol;
+    const uint32_t ul = threadIdx.x - (uint32_t)g * CU + col * CU;
     const long long r0 = L.row_lo + (long long)G * cta + g;
-    const bool active = g < G && r0 < L.row_hi && ul < U;
+    const bool active = g < G && r0 < L.row_hi && ul < U && threadIdx.x < (uint32_t)G * CU;
     const long long rstep = (long long)G * n_cta;
     // the tables are not produced by kernels: fetch the first descriptor before ordering
     // behind the previous kernel
@@ -330,7 +338,7 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
     const long long r_end = L.row_hi;
     const uint32_t tab_step = (uint32_t)G * NT;
 
-    for (uint32_t u = ul; u < U; u += CU) {
+    for (uint32_t u = ul; u < U; u += (ncol > 1 ? U : CU)) {
         const UnitRegs R = u == ul ? R_first : load_unit(L, u);
         // used dimension tested in position e: e itself (dense) or the unit's own list
         auto dim_of = [&](int e) -> int {

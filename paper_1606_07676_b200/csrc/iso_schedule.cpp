@@ -63,6 +63,7 @@ Knobs read_knobs()
     k.coord_table = num("ISO_COORD_TABLE", 1) != 0;
     k.host_graph = num("ISO_HOST_GRAPH", 1) != 0;
     k.hybrid = (int)num("ISO_HYBRID", -1);
+    k.col_split = num("ISO_COL_SPLIT", 1) != 0;
     return k;
 }
 
@@ -1038,6 +1039,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                     (void)width;
                     int64_t tp;
                     int64_t grid;
+                    uint32_t whole_row_slots = 1;  // rows a CTA would hold if it covered whole rows
                     if (kernel == KERNEL_VEC) {
                         // a row slot covers up to 256 unit positions; short rows share a CTA
                         // 16-byte launches with long rows use CTAs of up to 1024 threads
@@ -1055,6 +1057,23 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         }
                         L.chunk_units = (uint32_t)std::min<uint64_t>(units, max_threads);
                         L.rows_per_pass = std::max<uint32_t>(1, max_threads / L.chunk_units);
+                        whole_row_slots = L.rows_per_pass;
+                        // rows longer than a CTA: equal column chunks, the CTAs dealt to them (not in the
+                        // one-launch modes, whose grids are sized elsewhere, nor with a bulk side)
+                        // Measured on launches that shift along one dimension: shells 3.59 -> 3.21 ms, Moore d=3
+                        // r=3 0.617 -> 0.544 ms, shells allgather 0.879 -> 0.797 ms; the one-pass direct launches
+                        // (three wrap tests per row) lost 4 % and keep whole rows.  Splitting shorter rows to
+                        // fill the CTA's thread slots (690 unit positions as 3 chunks x 4 rows), or into more
+                        // chunks than needed, measured slower (irregular 64x64x32: 1.54 -> 1.60 ms; Moore r=3
+                        // allgather 0.204 -> 0.235 ms).
+                        L.col_split = 1;
+                        if (max_threads == 1024 && units > max_threads && L.n_used <= 2 && longs.empty() && !r.persistent &&
+                            r.wave_request == 0 && r.knobs.col_split) {
+                            const uint32_t ncol = (uint32_t)((units + max_threads - 1) / max_threads);
+                            L.col_split = (int)ncol;
+                            L.chunk_units = (uint32_t)(((units + ncol - 1) / ncol + 31) / 32 * 32);
+                            L.rows_per_pass = 1;
+                        }
                         L.threads = (int)((L.chunk_units * L.rows_per_pass + 31) / 32 * 32);
                         // CTAs of fewer than 256 threads: as many per SM as keep 1024 threads resident
                         int per_sm = L.threads > 512 ? 1 : (L.threads > 256 ? 2 : std::min(16, std::max(4, 1024 / L.threads)));
@@ -1067,6 +1086,11 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         grid = std::min<int64_t>((c.P + L.rows_per_pass - 1) / L.rows_per_pass,
                                                  (int64_t)r.sm_count * per_sm);
                         grid = std::max<int64_t>(grid, 1);
+                        L.rows_hint = std::min<int64_t>((c.P + whole_row_slots - 1) / whole_row_slots, (int64_t)r.sm_count * per_sm) *
+                                      whole_row_slots;
+                        if (L.col_split > 1)  // a multiple of the column chunks
+                            grid = std::max<int64_t>(1, std::min<int64_t>((c.P + L.rows_per_pass - 1) / L.rows_per_pass,
+                                                                          r.sm_count / L.col_split)) * L.col_split;
                         tp = 1;
                     } else {
                         int threads = (int)(196608 / (2 * unit)) / 32 * 32;
