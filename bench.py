@@ -206,14 +206,14 @@ class OracleSample:
     6 GB workload costs a few hundred MB of host memory.  Only the CPU-baseline leg and the
     reference arm use this."""
 
-    def __init__(self, w, max_out_bytes=192 << 20):
+    def __init__(self, w, max_out_bytes=192 << 20, whole_below=512 << 20):
         from paper_1606_07676_b200 import workloads as wl
         self.w = w
         self.lens, self.sd, self.rd, self.ss, self.rs = wl.layout(w)
         P, p0 = w.P, w.dims[0]
         plane = P // p0
         planes = max(1, min(p0, max_out_bytes // max(1, plane * self.rs)))
-        if planes >= p0 or P * self.ss <= (512 << 20):
+        if planes >= p0 or P * self.ss <= whole_below:
             self.r0, self.r1 = 0, P
             self.send = wl.send_buffer_np(w, self.ss)
             self.what = "the whole workload (%d processes x %d blocks)" % (P, w.s)
