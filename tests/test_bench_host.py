@@ -73,6 +73,8 @@ def test_traffic_entries_are_ignored_once_the_kernels_change(tmp_path, monkeypat
     assert got and got["bytes_per_step"] == 20626400000.0 and got["launches"] == 2
     assert bench.recorded_traffic("cfg2_alltoall", "combining") is None      # stamped with other sources
     assert bench.recorded_traffic("cfg3_m4096", "direct") is None
-    # the tracked file itself is current
+    # the tracked file is well formed: workload, schedule, launches, bytes, mode, scaling, 16-hex stamp, commit
     monkeypatch.undo()
-    assert bench.recorded_traffic("cfg3_m4096", "combining") is not None
+    rows = [ln.split() for ln in open(bench.TRAFFIC_FILE) if ln.strip() and not ln.startswith("#")]
+    assert rows and all(len(f) == 8 and int(f[2]) > 0 and float(f[3]) > 0 and len(f[6]) == 16 for f in rows)
+    assert any(f[0] == bench.HEADLINE and f[1] == "combining" for f in rows)
