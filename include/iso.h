@@ -298,8 +298,9 @@ int Iso_request_set_graph(Iso_request request, int enable);
  * buffers; with it a scratch buffer of twice the L2 size is overwritten before every timed
  * start (allocated for the duration of the call), as when other work runs between the
  * starts.  With ISO_TUNE_SCHEDULE the schedule is chosen as well: the message-combining
- * schedule with one and with two dimensions per phase and the direct schedule are all timed,
- * each under every execution plan, and the request is left on the fastest (on one device
+ * schedule with one and with two dimensions per phase (for an allgather in both visiting
+ * orders of the dimensions, see Iso_request_set_dimension_order) and the direct schedule are
+ * all timed, each under every execution plan, and the request is left on the fastest (on one device
  * the direct schedule usually wins: it moves the fewest bytes); Iso_request_get_stats then
  * reports the algorithm and fusion level in use, Iso_request_get_execution the plan.
  * Without it the request keeps its schedule.  The collective is executed many times meanwhile:
@@ -340,6 +341,19 @@ int Iso_request_set_hybrid(Iso_request request, int enable);
  * Iso_request_get_stats counts a block read once per load in bytes_moved.
  */
 int Iso_request_set_sender_side(Iso_request request, int mode);
+
+/* Allgather, message-combining schedule: the order in which the prefix trie visits the
+ * dimensions (Section III-B leaves it open; the received data never depends on it, the number
+ * of parts may for neighbourhoods that are not symmetric in the dimensions).  order[k] is the
+ * dimension visited k-th, a permutation of 0..d-1 (host array, read during the call).  Stored
+ * for the other collectives but without effect there.  Rebuilds the schedule; waits for a
+ * start in flight first.  ISO_ERR_ARG if `order` is not a permutation. */
+int Iso_request_set_dimension_order(Iso_request request, const int order[]);
+/* The order in use: d values written to `order` (host array).  Default for the allgather:
+ * last dimension first when the neighbours have at most 8 distinct non-zero coordinates in
+ * dimension 0 (the last phase then copies runs of consecutive receive slots), first to last
+ * otherwise; 0..d-1 for the other collectives. */
+int Iso_request_get_dimension_order(Iso_request request, int order[]);
 
 /* Parts of at least `bytes` bytes whose addresses and length are multiples of 16 are moved
  * by the bulk-copy kernel (asynchronous bulk copies staged through shared memory), the rest

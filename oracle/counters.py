@@ -99,10 +99,15 @@ def direct_volume(offsets, d, dims=None) -> int:
     return sum(direct_hops(offsets, d, dims))
 
 
-def allgather_direct_volume(offsets, d, dims=None) -> int:
+def allgather_direct_volume(offsets, d, dims=None, order=None) -> int:
     """Blocks received per process by the direct-communication allgather: one per
-    trie edge with a non-zero weight (a zero edge forwards nothing)."""
+    trie edge with a non-zero weight (a zero edge forwards nothing).  `order` is the
+    order in which the trie visits the dimensions (Section III-B leaves it open;
+    default 0..d-1): the count depends on it unless the neighbourhood is symmetric
+    in the dimensions."""
     vs = residues(offsets, dims) if dims is not None else _vectors(offsets, d)
+    if order is not None:
+        vs = [tuple(v[k] for k in order) for v in vs]
     prefixes = set()
     for v in vs:
         for j in range(1, d + 1):

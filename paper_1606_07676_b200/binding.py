@@ -31,7 +31,7 @@ EXPORTS = (
     "Iso_neighborhood_create", "Iso_comm_free", "Iso_comm_set_periodic",
     "Iso_neighbor_alltoall_init", "Iso_neighbor_allgather_init", "Iso_neighbor_alltoallv_init",
     "Iso_neighbor_allgatherv_init", "Iso_request_set_algorithm", "Iso_request_set_layout", "Iso_request_set_single_launch", "Iso_request_set_slabs", "Iso_request_set_pipeline", "Iso_request_set_chains", "Iso_request_set_graph", "Iso_request_tune", "Iso_request_get_execution", "Iso_request_set_bulk_threshold",
-    "Iso_request_set_hybrid", "Iso_request_set_sender_side", "Iso_request_check_guards", "Iso_request_get_host_transfer_ms", "Iso_request_set_wait_limit", "Iso_request_test_skew_arrivals", "Iso_measure_launch_floor",
+    "Iso_request_set_hybrid", "Iso_request_set_sender_side", "Iso_request_set_dimension_order", "Iso_request_get_dimension_order", "Iso_request_check_guards", "Iso_request_get_host_transfer_ms", "Iso_request_set_wait_limit", "Iso_request_test_skew_arrivals", "Iso_measure_launch_floor",
     "Iso_Start", "Iso_Start_host", "Iso_wait", "Iso_request_get_stats", "Iso_request_get_parts",
     "Iso_neighbor_alltoall_static", "Iso_request_free", "Iso_error_string", "Iso_last_cuda_error", "Iso_selftest",
 )
@@ -103,6 +103,8 @@ def load_library() -> ctypes.CDLL:
         "Iso_request_set_bulk_threshold": [vp, i64],
         "Iso_request_set_hybrid": [vp, ci],
         "Iso_request_set_sender_side": [vp, ci],
+        "Iso_request_set_dimension_order": [vp, ctypes.POINTER(ci)],
+        "Iso_request_get_dimension_order": [vp, ctypes.POINTER(ci)],
         "Iso_request_check_guards": [vp, ctypes.POINTER(i64)],
         "Iso_request_get_host_transfer_ms": [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                                              ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ci)],
@@ -306,6 +308,17 @@ def Iso_request_set_hybrid(request: int, enable: bool) -> None:
 
 def Iso_request_set_sender_side(request: int, mode: int) -> None:
     _check(load_library().Iso_request_set_sender_side(request, mode), "Iso_request_set_sender_side")
+
+
+def Iso_request_set_dimension_order(request: int, order) -> None:
+    arr = (ctypes.c_int * len(order))(*[int(x) for x in order])
+    _check(load_library().Iso_request_set_dimension_order(request, arr), "Iso_request_set_dimension_order")
+
+
+def Iso_request_get_dimension_order(request: int, d: int):
+    arr = (ctypes.c_int * d)()
+    _check(load_library().Iso_request_get_dimension_order(request, arr), "Iso_request_get_dimension_order")
+    return [int(x) for x in arr]
 
 
 def Iso_request_check_guards(request: int) -> int:

@@ -134,6 +134,7 @@ Iso_request_s *new_request(Iso_comm comm, int kind, const void *sendbuf, void *r
     r->knobs = read_knobs();
     if (r->knobs.sender_side >= 0 && r->knobs.sender_side <= 2) r->sender_side = r->knobs.sender_side;
     if (r->knobs.hybrid >= 0) r->hybrid = r->knobs.hybrid != 0;
+    default_dimension_order(*r);
     r->send = static_cast<const unsigned char *>(sendbuf);
     r->recv = static_cast<unsigned char *>(recvbuf);
     r->s = comm->s;
@@ -1360,8 +1361,12 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
         }
     }
     const bool log = r.knobs.tune_log;
-    struct Choice { int slabs, chains, graph, alg, fusion, hybrid; };
-    const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0, r.alg, r.fusion, r.hybrid ? 1 : 0};
+    // order: visiting order of the allgather's trie (-1: as it was, 0: first dimension first, 1: last first)
+    struct Choice { int slabs, chains, graph, alg, fusion, hybrid, order; };
+    const Choice before{r.slab_request, r.chains_request, r.graph_request ? 1 : 0, r.alg, r.fusion, r.hybrid ? 1 : 0, -1};
+    int order_before[ISO_MAX_DIMS];
+    std::copy(r.dim_order, r.dim_order + ISO_MAX_DIMS, order_before);
+    int order_now = -1;
     Choice best = before;
     float best_ms = -1.0f;
     int rc = ISO_SUCCESS;
@@ -1372,16 +1377,28 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
         r.graph_request = c.graph != 0;
         r.hybrid = c.hybrid != 0;
         r.dirty = true;
+        if (c.order != order_now) {
+            int order[ISO_MAX_DIMS];
+            for (int k = 0; k < r.comm->d; ++k) order[k] = c.order < 0 ? order_before[k] : (c.order ? r.comm->d - 1 - k : k);
+            order_now = c.order;
+            r.alg = c.alg;
+            r.fusion = c.fusion;
+            return Iso_request_set_dimension_order(request, order);  // rebuilds the schedule
+        }
         if (c.alg != r.alg || c.fusion != r.fusion) return Iso_request_set_algorithm(request, c.alg, c.fusion);
         return ISO_SUCCESS;
     };
     // the schedules to try: the present one, or - when asked - the message-combining schedule
     // with the hops of 1 and of 2 consecutive dimensions per phase, and the direct schedule
-    std::vector<std::pair<int, int>> schedules(1, std::make_pair(r.alg, r.fusion));
+    // (the allgather's message-combining schedule in both visiting orders of the dimensions)
+    struct Sched { int first, second, order; };
+    std::vector<Sched> schedules(1, Sched{r.alg, r.fusion, -1});
     if (flags & ISO_TUNE_SCHEDULE) {
-        schedules.assign(1, std::make_pair((int)ISO_ALG_COMBINING, 1));
-        if (r.comm->d >= 3) schedules.push_back(std::make_pair((int)ISO_ALG_COMBINING, 2));
-        schedules.push_back(std::make_pair((int)ISO_ALG_DIRECT, 1));
+        const bool orders = r.kind == ISO_KIND_ALLGATHER && r.comm->d >= 2;
+        schedules.assign(1, Sched{(int)ISO_ALG_COMBINING, 1, orders ? 0 : -1});
+        if (orders) schedules.push_back(Sched{(int)ISO_ALG_COMBINING, 1, 1});
+        if (r.comm->d >= 3) schedules.push_back(Sched{(int)ISO_ALG_COMBINING, 2, -1});
+        schedules.push_back(Sched{(int)ISO_ALG_DIRECT, 1, -1});
     }
     // time `reps` starts back to back (the collective only reads the send buffers, so
     // repeating it leaves the same result)
@@ -1410,7 +1427,7 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
         // ragged rows only: does the lowering hand anything to bulk warps?
         r.hybrid = true;
         if (r.started) rc = Iso_wait(request);
-        if (rc == ISO_SUCCESS) rc = apply(Choice{1, 1, 0, sched.first, sched.second, 1});
+        if (rc == ISO_SUCCESS) rc = apply(Choice{1, 1, 0, sched.first, sched.second, 1, sched.order});
         if (rc == ISO_SUCCESS) rc = lower_schedule(r, (uintptr_t)r.send, (uintptr_t)r.recv, (uintptr_t)r.d_inter);
         bool any = false;
         for (const LaunchPlan &L : r.launches) any = any || !L.side.empty();
@@ -1423,11 +1440,11 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
             for (int slabs = 1; slabs <= 64 && slabs <= std::max(1, p0) && rc == ISO_SUCCESS; slabs *= 2) {
                 if (chains > 1 && slabs < chains) continue;
                 if (r.started) rc = Iso_wait(request);
-                if (rc == ISO_SUCCESS) rc = apply(Choice{slabs, chains, graph, sched.first, sched.second, hybrid});
+                if (rc == ISO_SUCCESS) rc = apply(Choice{slabs, chains, graph, sched.first, sched.second, hybrid, sched.order});
                 if (rc == ISO_SUCCESS) rc = materialise(r);
                 if (rc != ISO_SUCCESS) break;
                 // what the schedule allowed may differ from what was asked for: skip repeats
-                const Choice got{(int)std::max<size_t>(1, r.slab_plan.size()), r.chains, r.use_graph ? 1 : 0, r.alg, r.fusion, hybrid};
+                const Choice got{(int)std::max<size_t>(1, r.slab_plan.size()), r.chains, r.use_graph ? 1 : 0, r.alg, r.fusion, hybrid, sched.order};
                 bool seen = false;
                 for (const Choice &c : tried) seen = seen || (c.slabs == got.slabs && c.chains == got.chains && c.graph == got.graph);
                 if (seen) continue;
@@ -1439,12 +1456,12 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
                 rc = measure(reps, ms);
                 if (rc != ISO_SUCCESS) break;
                 if (log)
-                    std::fprintf(stderr, "iso tune: alg %d fusion %d hybrid %d slabs %d chains %d graph %d: %.4f ms\n", got.alg,
-                                 got.fusion, got.hybrid, got.slabs, got.chains, got.graph, ms);
+                    std::fprintf(stderr, "iso tune: alg %d fusion %d order %d hybrid %d slabs %d chains %d graph %d: %.4f ms\n", got.alg,
+                                 got.fusion, got.order, got.hybrid, got.slabs, got.chains, got.graph, ms);
                 // the plainer plans come first; a later one must win by 2 % to replace them
                 if (best_ms < 0.0f || ms < 0.98f * best_ms) {
                     best_ms = ms;
-                    best = Choice{slabs, chains, graph, sched.first, sched.second, hybrid};
+                    best = Choice{slabs, chains, graph, sched.first, sched.second, hybrid, sched.order};
                 }
             }
         }
@@ -1489,6 +1506,45 @@ int Iso_request_set_sender_side(Iso_request request, int mode)
     int rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
     request->dirty = true;
     return rc;
+    });
+}
+
+int Iso_request_set_dimension_order(Iso_request request, const int order[])
+{
+    return guarded([&]() -> int {
+    if (check_handle(request) || !order) return ISO_ERR_ARG;
+    const int d = request->comm->d;
+    bool seen[ISO_MAX_DIMS] = {false};
+    for (int k = 0; k < d; ++k) {
+        if (order[k] < 0 || order[k] >= d || seen[order[k]]) return ISO_ERR_ARG;
+        seen[order[k]] = true;
+    }
+    if (request->started) {
+        int rc = Iso_wait(request);
+        if (rc != ISO_SUCCESS) return rc;
+    }
+    int old[ISO_MAX_DIMS];
+    std::copy(request->dim_order, request->dim_order + ISO_MAX_DIMS, old);
+    std::copy(order, order + d, request->dim_order);
+    int rc = build_schedule(*request);
+    if (rc == ISO_SUCCESS)
+        rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
+    if (rc != ISO_SUCCESS) {
+        std::copy(old, old + ISO_MAX_DIMS, request->dim_order);
+        build_schedule(*request);
+        lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
+    }
+    request->dirty = true;
+    return rc;
+    });
+}
+
+int Iso_request_get_dimension_order(Iso_request request, int order[])
+{
+    return guarded([&]() -> int {
+    if (check_handle(request) || !order) return ISO_ERR_ARG;
+    std::copy(request->dim_order, request->dim_order + request->comm->d, order);
+    return ISO_SUCCESS;
     });
 }
 

@@ -126,6 +126,7 @@ struct Knobs {
     bool col_split = true;    // ISO_COL_SPLIT=0: rows longer than a CTA are covered in passes instead of column chunks
     bool host_graph = true;   // ISO_HOST_GRAPH=0: the pipelined host-buffer path is never replayed from a graph
     bool coord_table = true;  // ISO_COORD_TABLE=0: row coordinates by division in every thread
+    int ag_order = -1;        // ISO_AG_ORDER=0/1: allgather visits the dimensions first-to-last / last-to-first
 };
 Knobs read_knobs();
 
@@ -135,6 +136,7 @@ struct Request {
     int kind = ISO_KIND_ALLTOALL;
     int alg = ISO_ALG_COMBINING;
     int fusion = 1;
+    int dim_order[ISO_MAX_DIMS] = {0, 1, 2, 3, 4, 5, 6, 7};  // allgather: dimension visited k-th (Section III-B)
     int64_t bulk_threshold = 512;
     int layout = ISO_LAYOUT_PACKED;
     int slab_request = 0;     // slabs of dimension 0 Iso_Start runs one after the other (0: automatic, 1: none)
@@ -195,6 +197,8 @@ struct Request {
 
 // Builds r.parts, r.inter_stride and the schedule statistics from r.comm, r.kind, r.alg,
 // r.fusion and the block layout.  Returns an ISO_* code.
+// Default visiting order of the allgather's prefix trie for this neighbourhood (fills r.dim_order).
+void default_dimension_order(Request &r);
 int build_schedule(Request &r);
 
 // Splits parts into aligned pieces, groups them into kernel launches and fills the launch

@@ -64,6 +64,19 @@ def test_fig1_trie_shape():
     assert counters.allgather_direct_volume(leaves, 3) == 13
 
 
+def test_trie_volume_under_another_visiting_order():
+    # Section III-B leaves the order in which the trie visits the dimensions open.  Worked by
+    # hand: {(1,1), (2,1)} has the non-zero edges 1, 1-1, 2, 2-1 first-to-last (4 blocks) and
+    # 1, 1-1, 1-2 last-to-first (3 blocks: the two vectors then share their first edge)
+    pair = [[1, 1], [2, 1]]
+    assert counters.allgather_direct_volume(pair, 2) == 4
+    assert counters.allgather_direct_volume(pair, 2, order=(0, 1)) == 4
+    assert counters.allgather_direct_volume(pair, 2, order=(1, 0)) == 3
+    # a Moore neighbourhood is symmetric in the dimensions: s blocks in any order
+    for order in ((0, 1, 2), (2, 1, 0), (1, 0, 2), (2, 0, 1)):
+        assert counters.allgather_direct_volume(wl.moore(3, 2), 3, order=order) == 124
+
+
 def test_small_torus_aliasing():
     # coordinates that are equal modulo p_j share a round; a multiple of p_j needs no hop
     offs = [[1], [4], [-2], [3], [0]]

@@ -4,6 +4,7 @@ import numpy as np
 import pytest
 
 import oracle
+from oracle import counters
 from paper_1606_07676_b200 import binding as iso
 from paper_1606_07676_b200 import workloads as wl
 from schedule_sim import POISON, layout, make_request, oracle_result, send_buffer_np
@@ -256,6 +257,58 @@ def test_allgather_phases_in_sender_side_form(torch_cuda):
     run.result(*COMB1)
     assert {p["phase"] for p in iso.Iso_request_get_parts(run.req) if p["kernel"] == 2} == {2, 3}
     run.close()
+
+
+def test_allgather_visiting_orders(torch_cuda):
+    """The allgather's trie may visit the dimensions in any order (Section III-B): every order
+    gives the oracle's bytes, on the configuration, on a neighbourhood that is not symmetric in
+    the dimensions (where the number of parts depends on the order), with intermediate storage,
+    on a mesh, in both forms of the phases; the tuner may pick either order."""
+    torch = torch_cuda
+    lop = np.array([(0, 0, 0), (0, 0, 1), (1, 0, 0), (1, 1, 0), (1, 1, 1), (3, 2, 0), (3, 3, 2), (4, 0, 1), (4, 0, 2),
+                    (4, 1, 1), (-2, 5, 1), (1, 1, 1)], np.int32)
+    cases = [(wl.config("cfg2_allgather"), None), (wl.Workload("lop", "allgather", (9, 8, 7), lop, 48, seed=8), None),
+             (wl.Workload("sh", "allgather", (16, 15, 17), wl.shells(3, (3, 7)), 16, seed=3), None),
+             (wl.Workload("mesh", "allgather", (6, 5, 7), wl.moore(3, 1), 32, seed=9), [0, 1, 0]),
+             (wl.Workload("d4", "allgather", (5, 4, 6, 3), wl.moore(4, 1), 16, seed=10), None)]
+    for w, periodic in cases:
+        run = Run(torch, w, periodic=periodic)
+        want = oracle_result(w, run.send_host, periodic=periodic)
+        d = len(w.dims)
+        default = iso.Iso_request_get_dimension_order(run.req, d)
+        assert sorted(default) == list(range(d))
+        orders = [list(range(d)), list(range(d))[::-1], [1, 0] + list(range(2, d)), list(range(1, d)) + [0]]
+        for order in orders:
+            iso.Iso_request_set_dimension_order(run.req, order)
+            assert iso.Iso_request_get_dimension_order(run.req, d) == order
+            for mode in (0, 2):
+                iso.Iso_request_set_sender_side(run.req, mode)
+                got = run.result(*COMB1)
+                assert np.array_equal(got, want), (w.name, order, mode)
+            if periodic is None:
+                st = iso.Iso_request_get_stats(run.req)
+                # one part per non-zero edge of the trie, and one more per repetition of a vector
+                repeats = len(w.offsets) - len({tuple(v) for v in w.offsets.tolist()})
+                assert st["parts"] == counters.allgather_direct_volume(w.offsets, d, w.dims, order) + repeats
+            assert iso.Iso_request_check_guards(run.req) == 0
+        run.close()
+    run = Run(torch, wl.config("moore_d4r1_allgather"))
+    want = oracle_result(run.w, run.send_host)
+    assert iso.Iso_request_get_dimension_order(run.req, 4) == [3, 2, 1, 0]
+    iso.Iso_request_tune(run.req, None, schedule=True)
+    assert sorted(iso.Iso_request_get_dimension_order(run.req, 4)) == [0, 1, 2, 3]
+    run.recv.fill_(POISON)
+    torch.cuda.synchronize()
+    iso.Iso_Start(run.req, None)
+    iso.Iso_wait(run.req)
+    assert np.array_equal(run.recv.cpu().numpy(), want)
+    run.close()
+    with pytest.raises(iso.IsoError):
+        r2 = Run(torch, wl.config("cfg1"))
+        try:
+            iso.Iso_request_set_dimension_order(r2.req, [0, 0])
+        finally:
+            r2.close()
 
 
 @pytest.mark.parametrize("m", [4, 64, 512])

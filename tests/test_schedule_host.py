@@ -235,8 +235,25 @@ def test_allgather_statistics_follow_the_trie():
                                   (4, 0, 1), (4, 0, 2), (4, 1, 1)], np.int32), (8, 8, 8))]:
         w = wl.Workload("ag", "allgather", dims, offs, 64)
         comm, req = make_request(w)
+        # the trie may visit the dimensions in any order (Section III-B): same rounds, same result,
+        # and as many parts as the trie over the permuted vectors has non-zero edges
+        send0 = send_buffer_np(w, 64)
+        for order in itertools.permutations(range(3)):
+            iso.Iso_request_set_dimension_order(req, order)
+            assert iso.Iso_request_get_dimension_order(req, 3) == list(order)
+            st = iso.Iso_request_get_stats(req)
+            assert st["parts"] == counters.allgather_direct_volume(offs, 3, dims, order)
+            assert st["rounds"] == counters.direct_rounds(offs, 3, dims)
+            if w.P <= 4096:
+                assert np.array_equal(simulate(iso.Iso_request_get_parts(req), w.dims, st, send0), oracle_result(w, send0))
+        # default: last dimension first for these neighbourhoods (at most 8 distinct coordinates in dimension 0)
+        iso.Iso_request_free(req)
+        iso.Iso_comm_free(comm)
+        comm, req = make_request(w)
+        order = iso.Iso_request_get_dimension_order(req, 3)
+        assert order == [2, 1, 0]
         st = iso.Iso_request_get_stats(req)
-        assert st["parts"] == counters.allgather_direct_volume(offs, 3, dims)
+        assert st["parts"] == counters.allgather_direct_volume(offs, 3, dims, order)
         assert st["rounds"] == counters.direct_rounds(offs, 3, dims)
         assert st["bytes_moved"] == 2 * w.P * 64 * (st["parts"] + st["local_copies"])
         # sender-side launches: a parent block is read once for up to four of the places it is
