@@ -92,6 +92,13 @@ def expected(c):
     return _expected(c["kind"], c["dims"], c["offs"], c["lens"], c["sd"], c["rd"], c["ss"], c["rs"], c["send_h"], c["periodic"])
 
 
+def visiting_order(c, salt):
+    """A permutation of the dimensions, drawn from the case's trial number (the allgather's
+    trie may visit them in any order; the other collectives ignore it)."""
+    d = len(c["dims"])
+    return [int(x) for x in np.random.default_rng(1000 * c["trial"] + salt).permutation(d)]
+
+
 @pytest.mark.gpu
 @pytest.mark.parametrize("chunk", range(12))
 def test_random_cases(chunk):
@@ -116,6 +123,7 @@ def test_random_cases(chunk):
             iso.Iso_request_set_pipeline(req, pipe)
             iso.Iso_request_set_sender_side(req, (2, 1, 2, 0)[(c["trial"] + fusion) % 4])
             iso.Iso_request_set_hybrid(req, (c["trial"] + alg) % 2 == 0)
+            iso.Iso_request_set_dimension_order(req, visiting_order(c, alg + fusion))
             iso.Iso_request_set_algorithm(req, alg, fusion)
             if rs:
                 recv.fill_(POISON)
@@ -155,6 +163,7 @@ def test_random_cases_host_simulation(chunk):
             iso.Iso_request_set_bulk_threshold(req, bulk)
             iso.Iso_request_set_hybrid(req, (c["trial"] + alg) % 2 == 0)
             iso.Iso_request_set_sender_side(req, (2, 1, 2, 0)[(c["trial"] + fusion) % 4])
+            iso.Iso_request_set_dimension_order(req, visiting_order(c, alg + fusion))
             iso.Iso_request_set_algorithm(req, alg, fusion)
             st = iso.Iso_request_get_stats(req)
             got = simulate(iso.Iso_request_get_parts(req), c["dims"], st, c["send_h"] if c["ss"] else np.zeros((c["P"], 0), np.uint8),
