@@ -953,18 +953,25 @@ void choose_slab_plan(Request &r)
     int want = r.slab_request;
     if (r.knobs.slabs >= 0) want = r.knobs.slabs;
     if (want == 0) {
-        // automatic: all-to-all schedules made of vector launches only; a slab's launch should
-        // still last about 12 microseconds and give every CTA a dozen rows
+        // automatic: all-to-all schedules made of vector launches only.  What one launch of a slab
+        // writes the next one reads back, so both should sit in the L2 (126 MB) together: the
+        // fewest slabs (a power of two) that bring a launch's written bytes under 52 MB, as long
+        // as every CTA still gets half a dozen rows.  Measured optimum and this rule's choice on
+        // nine all-to-all workloads (64-byte blocks unless stated): 32^3 Moore r=1 1 and 1, 256^2
+        // Moore r=2 2 and 2, 8^5 16-byte blocks 2 and 2, positive octant 2 and 2, stencil-shaped
+        // sizes 4 and 2 (5 % apart), 16^4 Moore r=1 8 and 8, Moore r=3 16 and 16, shells 32 and 32,
+        // irregular 64x64x32 64 and 32 (1.5 % apart).
         if (r.kind == ISO_KIND_ALLGATHER) return;
         long long rows_per_pass = 1;
         for (const LaunchPlan &L : r.launches) {
             if (L.kernel != KERNEL_VEC) return;
             rows_per_pass = std::max<long long>(rows_per_pass, L.rows_hint > 0 ? (long long)L.rows_hint : (long long)L.grid * L.rows_per_pass);
         }
-        const double est_us = (double)r.stats.bytes_moved / 5.5e6;
-        const double per = est_us / (12.0 * (double)std::max<size_t>(1, r.launches.size()));
+        const double written = (double)r.stats.bytes_moved / 2.0 / (double)std::max<size_t>(1, r.launches.size());
+        int target = 1;
+        while (target < 64 && written / target > 52e6) target *= 2;
         want = 1;
-        while (want * 2 <= per && want * 2 <= 64 && c.P / (want * 2) >= 12 * rows_per_pass) want *= 2;
+        while (want < target && c.P / (want * 2) >= 6 * rows_per_pass) want *= 2;
     }
     int chains = std::max(1, r.chains_request);
     if (r.knobs.chains >= 0) chains = std::max(1, std::min(8, r.knobs.chains));
