@@ -532,7 +532,14 @@ def end_to_end(torch, iso, b, moved, minimum, steps, dist, world):
             "host_result_equals_device_result": same}
 
 
-SCHEDULES = (("combining", "ISO_ALG_COMBINING", 1), ("direct", "ISO_ALG_DIRECT", 1), ("torus", "ISO_ALG_TORUS", 1))
+SCHEDULES = (("combining", "ISO_ALG_COMBINING", 1), ("direct", "ISO_ALG_DIRECT", 1), ("torus", "ISO_ALG_TORUS", 1),
+             ("combining_2", "ISO_ALG_COMBINING", 2))   # two dimensions per phase (from three dimensions on)
+
+
+def skipped(key, w):
+    """Schedules a workload does not have: Algorithm 1 is an all-to-all schedule; with two
+    dimensions per phase a torus of fewer than three dimensions has the direct schedule."""
+    return (key == "torus" and w.collective == "allgather") or (key == "combining_2" and len(w.dims) < 3)
 
 
 def row(st, times, peak, ok):
@@ -552,7 +559,8 @@ def steps_for(est_ms, floor_steps):
 
 def config_table(torch, iso, wl, peak, args, names, have=None):
     """Every configuration under the combining schedule (one launch per dimension), the
-    one-pass direct schedule and the hop-by-hop schedule of Algorithm 1, each timed as
+    one-pass direct schedule, the hop-by-hop schedule of Algorithm 1 and the combining schedule
+    with two dimensions per phase, each timed as
     repeated runs until `--detail-ms` of device time and then checked against the oracle.
     `have` holds rows measured elsewhere (the headline workload)."""
     out = dict(have or {})
@@ -562,8 +570,8 @@ def config_table(torch, iso, wl, peak, args, names, have=None):
         reps = Replicas(torch, iso, wl, name)
         rows = {}
         for key, alg_name, fusion in SCHEDULES:
-            if key == "torus" and reps.items[0].w.collective == "allgather":
-                rows[key] = None        # Algorithm 1 is an all-to-all schedule
+            if skipped(key, reps.items[0].w):
+                rows[key] = None
                 continue
             st = reps.set(getattr(iso, alg_name), fusion)
             est = time_run(torch, reps.start, 8, 3)
@@ -679,7 +687,7 @@ def run_ours(args):
                                                   replicas=len(reps.items), execution=reps.execution())}}
         if args.alg == "combining" and not args.no_detail:
             for key, alg_name, fusion in SCHEDULES[1:]:
-                if key == "torus" and b.w.collective == "allgather":
+                if skipped(key, b.w):
                     have[args.workload][key] = None
                     continue
                 s2 = reps.set(getattr(iso, alg_name), fusion)
