@@ -536,7 +536,7 @@ unsigned grid_for_rows(const LaunchPlan &L, const LaunchDev &a, int share = 1)
 {
     const long long rows = a.row_hi - a.row_lo;
     if (rows >= a.P && share <= 1) return (unsigned)L.grid;
-    if (L.kernel == KERNEL_BULK) return (unsigned)((rows + L.tile_procs - 1) / L.tile_procs);
+    if (L.kernel == KERNEL_BULK) return (unsigned)((rows + a.tile_procs - 1) / a.tile_procs);
     const long long groups = (rows + L.rows_per_pass - 1) / L.rows_per_pass;
     // `share` launches of this kind run side by side: each takes its part of the CTA slots
     const long long full = std::max<long long>(1, L.grid / std::max(1, share));
@@ -644,6 +644,12 @@ int launch_one(const Request &r, const LaunchPlan &L, cudaStream_t stream, bool 
         a.row_lo = row_lo;
         a.row_hi = row_hi;
         if (row_hi <= row_lo) return ISO_SUCCESS;
+    }
+    // bulk kernel on a range of rows (a slab): its tiles were sized for the whole torus; keep at
+    // least two CTAs per SM busy on the range (a smaller tile needs less of the planned shared memory)
+    if (L.kernel == KERNEL_BULK && a.row_hi - a.row_lo < a.P) {
+        const long long per = std::max<long long>(1, (a.row_hi - a.row_lo) / ((long long)r.sm_count * 2));
+        a.tile_procs = (int)std::max<long long>(1, std::min<long long>(L.tile_procs, per));
     }
     // slab-serial execution: the intermediate buffer only holds one slab, addressed from
     // the slab's first row
@@ -1295,7 +1301,8 @@ int Iso_request_set_slabs(Iso_request request, int slabs)
     }
     request->slab_request = slabs;
     request->dirty = true;
-    return ISO_SUCCESS;
+    // (which kernel moves the longer parts depends on who chooses the slabs)
+    return lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
     });
 }
 
@@ -1428,6 +1435,22 @@ int Iso_request_tune(Iso_request request, void *cuda_stream, int flags)
         ms /= (float)reps;
         return ISO_SUCCESS;
     };
+    // the plan the request came with is the first candidate (with the slab count left to the
+    // library it may use kernels that no explicit slab count below selects)
+    {
+        if (r.started) rc = Iso_wait(request);
+        if (rc == ISO_SUCCESS) rc = materialise(r);
+        float ms = 0.0f;
+        if (rc == ISO_SUCCESS) rc = measure(3, ms);
+        if (rc == ISO_SUCCESS) {
+            const int reps = (int)std::max(5.0f, std::min(200.0f, 2.0f / std::max(ms, 1e-3f)));
+            rc = measure(reps, ms);
+        }
+        if (rc == ISO_SUCCESS) {
+            best_ms = ms;
+            if (log) std::fprintf(stderr, "iso tune: as it came: %.4f ms\n", ms);
+        }
+    }
     for (const auto &sched : schedules)
     for (int hybrid = 0; hybrid <= 1 && rc == ISO_SUCCESS; ++hybrid) {
     if (hybrid) {
@@ -1563,7 +1586,7 @@ int Iso_request_set_bulk_threshold(Iso_request request, int64_t bytes)
         int rc = Iso_wait(request);
         if (rc != ISO_SUCCESS) return rc;
     }
-    request->bulk_threshold = bytes;
+    request->bulk_threshold_asked = bytes;
     int rc = lower_schedule(*request, (uintptr_t)request->send, (uintptr_t)request->recv, (uintptr_t)request->d_inter);
     request->dirty = true;
     return rc;
@@ -2055,7 +2078,7 @@ extern "C" int Iso_neighbor_alltoall_static(int d, const int dims[], int s, cons
     r.alg = ISO_ALG_COMBINING;
     r.fusion = 1;
     r.layout = ISO_LAYOUT_PACKED;
-    r.bulk_threshold = 0;  // vector kernel only: no error flag, nothing that must start at zero
+    r.bulk_threshold_asked = 0;  // vector kernel only: no error flag, nothing that must start at zero
     r.send = static_cast<const unsigned char *>(sendbuf);
     r.recv = static_cast<unsigned char *>(recvbuf);
     r.s = s;

@@ -137,7 +137,8 @@ struct Request {
     int alg = ISO_ALG_COMBINING;
     int fusion = 1;
     int dim_order[ISO_MAX_DIMS] = {0, 1, 2, 3, 4, 5, 6, 7};  // allgather: dimension visited k-th (Section III-B)
-    int64_t bulk_threshold = 512;
+    int64_t bulk_threshold = 512;        // in force (set by lower_schedule)
+    int64_t bulk_threshold_asked = -1;   // Iso_request_set_bulk_threshold; -1: chosen by the library
     int layout = ISO_LAYOUT_PACKED;
     int slab_request = 0;     // slabs of dimension 0 Iso_Start runs one after the other (0: automatic, 1: none)
     bool persistent = false;  // run all phases in one cooperative launch when the schedule allows

@@ -743,9 +743,36 @@ int common_alignment(std::initializer_list<int64_t> xs)
 
 }  // namespace
 
+// Whether the schedule can run slab by slab (see plan_slabs in iso_api.cu): every part that
+// shifts along dimension 0 reads the send buffer, all dimensions periodic, at least four planes.
+static bool slabs_possible(const Request &r)
+{
+    const Comm &c = *r.comm;
+    if (c.d < 2 || c.dims[0] < 4) return false;
+    for (int j = 0; j < c.d; ++j)
+        if (!c.periodic[j]) return false;
+    for (const Part &p : r.parts)
+        if (p.shift[0] != 0 && p.src_buf != ISO_BUF_SEND) return false;
+    return true;
+}
+
 int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr_t inter_addr)
 {
     const Comm &c = *r.comm;
+    // From which part length on the bulk-copy kernel is used.  Asked for, or: 512 bytes (the
+    // measured crossover of one launch against one launch), but 4096 where the library may run
+    // the schedule in slabs of its own choice - an all-to-all with intermediate blocks - because
+    // only the vector kernel runs well in launches of a slab's size, and a slab's intermediate
+    // blocks are then read back out of the L2.  Measured on the 256x256 torus, Moore r=2, bulk
+    // kernel in one launch per phase against vector kernel in slabs: 512-byte blocks 438 against
+    // 391 microseconds, 1 KB 820 against 783, 2 KB 1668 against 1569, 4 KB 3295 against 3703.
+    if (r.bulk_threshold_asked >= 0) {
+        r.bulk_threshold = r.bulk_threshold_asked;
+    } else {
+        const bool own_slabs = r.kind != ISO_KIND_ALLGATHER && r.inter_stride > 0 && r.slab_request == 0 && r.knobs.slabs < 0 &&
+                               !r.persistent && r.wave_request == 0 && slabs_possible(r);
+        r.bulk_threshold = own_slabs ? 4096 : 512;
+    }
     const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
     const int64_t addr[3] = {(int64_t)send_addr, (int64_t)recv_addr, (int64_t)inter_addr};
     r.launches.clear();
