@@ -726,8 +726,8 @@ def run_ours(args):
                 for key, r_ in (detail["configs"].get(name) or {}).items():
                     if r_:
                         r_["launch_floor_ms"] = r_["launches"] * detail["launch_floor_us"]["dependent_launches"] * 1e-3
-            # DRAM traffic of the small configuration whose intermediate blocks stay in L2
-            for name in ("cfg2_alltoall", "cfg3_m64"):
+            # DRAM traffic of the configurations whose intermediate blocks stay in L2
+            for name in ("cfg2_alltoall", "cfg3_m64", "cfg3_m512"):
                 rec2 = recorded_traffic(name, "combining")
                 r_ = (detail["configs"].get(name) or {}).get("combining")
                 if rec2 and r_:
