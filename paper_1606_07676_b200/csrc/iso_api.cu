@@ -975,7 +975,7 @@ void choose_slab_plan(Request &r)
         }
         const double written = (double)r.stats.bytes_moved / 2.0 / (double)std::max<size_t>(1, r.launches.size());
         int target = 1;
-        while (target < 64 && written / target > 52e6) target *= 2;
+        while (target < kMaxOwnSlabs && written / target > kSlabLaunchBytes) target *= 2;
         want = 1;
         while (want < target && c.P / (want * 2) >= 6 * rows_per_pass) want *= 2;
     }

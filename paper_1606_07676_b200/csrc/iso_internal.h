@@ -70,7 +70,9 @@ struct FanParent {
 };
 constexpr int kFanDsts = 4;  // destinations per descriptor; a parent with more is listed several times
 constexpr int64_t kHybridMinBytes = 256;  // 16-byte-aligned pieces of a ragged row from which bulk copies take over
-constexpr int kMaxVecUnits = 4096;  // unit positions per process in one vector launch
+constexpr int kMaxOwnSlabs = 128;          // most slabs of dimension 0 the library chooses by itself
+constexpr double kSlabLaunchBytes = 52e6;  // what one launch of a slab may write so that it and its reader share the L2
+constexpr int kMaxVecUnits = 8192;  // unit positions per process in one vector launch
 constexpr int kVecDepth = 8;        // cp.async ring slots per thread in the vector kernel
 constexpr int kWideDepth = 12;      // the same in CTAs of more than 256 threads (one CTA per SM)
 constexpr int kHybridDepth = 6;     // the same for the vector warps of a hybrid launch (most of the shared memory stages bulk copies)

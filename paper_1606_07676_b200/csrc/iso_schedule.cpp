@@ -760,18 +760,27 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
 {
     const Comm &c = *r.comm;
     // From which part length on the bulk-copy kernel is used.  Asked for, or: 512 bytes (the
-    // measured crossover of one launch against one launch), but 4096 where the library may run
-    // the schedule in slabs of its own choice - an all-to-all with intermediate blocks - because
-    // only the vector kernel runs well in launches of a slab's size, and a slab's intermediate
-    // blocks are then read back out of the L2.  Measured on the 256x256 torus, Moore r=2, bulk
-    // kernel in one launch per phase against vector kernel in slabs: 512-byte blocks 438 against
-    // 391 microseconds, 1 KB 820 against 783, 2 KB 1668 against 1569, 4 KB 3295 against 3703.
+    // measured crossover of one launch against one launch) - except where the library may run
+    // the schedule in slabs of its own choice (an all-to-all with intermediate blocks) and can
+    // make the slabs small enough for the L2 (choose_slab_plan: 52 MB written per launch, at
+    // most 128 slabs of at least two planes and 512 processes): there the vector kernel moves
+    // everything, because only it runs well in launches of a slab's size, and a slab's
+    // intermediate blocks are then read back out of the L2.  Measured on the 256x256 torus,
+    // Moore r=2, bulk kernel in one launch per phase against vector kernel in slabs: 512-byte
+    // blocks 438 against 391 microseconds, 1 KB 820 against 783, 2 KB 1668 against 1566, 4 KB
+    // 3295 against 3157 (128 slabs).
     if (r.bulk_threshold_asked >= 0) {
         r.bulk_threshold = r.bulk_threshold_asked;
     } else {
-        const bool own_slabs = r.kind != ISO_KIND_ALLGATHER && r.inter_stride > 0 && r.slab_request == 0 && r.knobs.slabs < 0 &&
-                               !r.persistent && r.wave_request == 0 && slabs_possible(r);
-        r.bulk_threshold = own_slabs ? 4096 : 512;
+        bool own_slabs = r.kind != ISO_KIND_ALLGATHER && r.inter_stride > 0 && r.slab_request == 0 && r.knobs.slabs < 0 &&
+                         !r.persistent && r.wave_request == 0 && slabs_possible(r);
+        if (own_slabs) {
+            const double written = (double)r.stats.bytes_moved / 2.0 / (double)std::max(1, r.stats.phases);
+            int64_t need = 1;
+            while (need < kMaxOwnSlabs && written / (double)need > kSlabLaunchBytes) need *= 2;
+            own_slabs = written / (double)need <= kSlabLaunchBytes && need * 2 <= c.dims[0] && c.P / need >= 512;
+        }
+        r.bulk_threshold = own_slabs ? 0 : 512;
     }
     const int64_t stride[3] = {r.send_stride, r.recv_stride, r.inter_stride};
     const int64_t addr[3] = {(int64_t)send_addr, (int64_t)recv_addr, (int64_t)inter_addr};
@@ -1026,7 +1035,7 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                 // handed to one extra warp of the CTA that moves them with bulk copies, while
                 // the other warps move the ragged rest (see iso_gather_rows_hybrid).
                 std::vector<Piece> longs;
-                if (kernel == KERNEL_VEC && width == 0 && r.hybrid && r.bulk_threshold > 0 && c.d <= 3) {
+                if (kernel == KERNEL_VEC && width == 0 && r.hybrid && r.bulk_threshold_asked != 0 && c.d <= 3) {
                     bool plain = true;  // periodic dimensions only
                     for (const Piece &q : cls)
                         for (int j = 0; j < c.d; ++j) plain = plain && !q.p.check[j];
@@ -1163,9 +1172,11 @@ int lower_schedule(Request &r, uintptr_t send_addr, uintptr_t recv_addr, uintptr
                         grid = std::max<int64_t>(grid, 1);
                         L.rows_hint = std::min<int64_t>((c.P + whole_row_slots - 1) / whole_row_slots, (int64_t)r.sm_count * per_sm) *
                                       whole_row_slots;
-                        if (L.col_split > 1)  // a multiple of the column chunks
+                        if (L.col_split > 1) {  // a multiple of the column chunks; the CTAs of one chunk share the rows
                             grid = std::max<int64_t>(1, std::min<int64_t>((c.P + L.rows_per_pass - 1) / L.rows_per_pass,
                                                                           r.sm_count / L.col_split)) * L.col_split;
+                            L.rows_hint = std::max<int64_t>(1, r.sm_count / L.col_split);
+                        }
                         tp = 1;
                     } else {
                         int threads = (int)(196608 / (2 * unit)) / 32 * 32;

@@ -346,13 +346,21 @@ def test_cfg3_4096_sampled(torch_cuda):
     ranks = sorted({0, 1, 255, 256, 257, 511, P - 1, P - 256, P - 257, *rng.integers(0, P, 24).tolist()})
     host_send = None
     try:
-        for alg, fusion in (COMB1, DIRECT):
+        # the combining schedule as the library plans it (vector kernel in 128 slabs of two
+        # planes, so that a slab's intermediate blocks stay in the L2), the same schedule through
+        # the bulk-copy kernel (threshold asked for), and the direct schedule (bulk-copy kernel)
+        for alg, fusion, bulk in (COMB1 + (None,), COMB1 + (512,), DIRECT + (None,)):
+            if bulk is not None:
+                iso.Iso_request_set_bulk_threshold(req, bulk)
             iso.Iso_request_set_algorithm(req, alg, fusion)
             recv.fill_(POISON)
             iso.Iso_Start(req)
             iso.Iso_wait(req)
             st = iso.Iso_request_get_stats(req)
-            assert st["bulk_bytes"] == st["bytes_moved"]       # 4 KB blocks use the bulk kernel
+            if alg == iso.ISO_ALG_COMBINING and bulk is None:
+                assert st["bulk_bytes"] == 0 and iso.Iso_request_get_execution(req)["slabs"] == 128
+            else:
+                assert st["bulk_bytes"] == st["bytes_moved"]
             for r in ranks:
                 got = recv[r * stride:(r + 1) * stride].cpu().numpy().reshape(s, m)
                 for i in range(s):
