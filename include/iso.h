@@ -282,8 +282,9 @@ int Iso_request_set_chains(Iso_request request, int chains);
  * a change of the request captures its launches into a CUDA graph on a stream of the
  * library's own and every Iso_Start replays that graph on the caller's stream: one
  * submission per start instead of one per launch, which pays for schedules of many short
- * launches and costs a few microseconds on schedules of few long ones.  Default off.
- * Ignored in single-launch mode.  The result never depends on it.
+ * launches and costs a few microseconds on schedules of few long ones.  With `enable` == 0
+ * (the default) the library replays from a graph only where a start has 128 launches or
+ * more.  Ignored in single-launch mode.  The result never depends on it.
  */
 int Iso_request_set_graph(Iso_request request, int enable);
 

@@ -997,6 +997,10 @@ void choose_slab_plan(Request &r)
         r.use_graph = true;
         rows *= chains;
     }
+    // a start of very many launches is replayed from a graph unless the environment says otherwise
+    // (4 KB blocks on the 256x256 torus, 256 launches per start: 3.16 -> 3.10 ms; at 96 launches
+    // per start and below replay measured no gain)
+    if (r.knobs.graph < 0 && r.slab_plan.size() * r.launches.size() >= 128) r.use_graph = true;
     // the pipelined host-buffer path cuts dimension 0 into slabs of its own (plan_slabs)
     std::vector<SlabPlan> host;
     plan_slabs(r, host);
