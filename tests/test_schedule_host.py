@@ -334,6 +334,39 @@ def test_alignment_classes_and_bulk_selection():
     iso.Iso_comm_free(comm)
 
 
+def test_bulk_threshold_left_to_the_library():
+    """Which kernel moves large blocks when nobody says: the vector kernel where the library may
+    run the all-to-all in slabs of its own that fit the L2, the bulk-copy kernel from 512 bytes
+    elsewhere (a slab count asked for, slabs that would be too small, the direct schedule, the
+    allgather), and whatever threshold the caller sets."""
+    def kernels(req):
+        return {p["kernel"] for p in iso.Iso_request_get_parts(req)}
+    for name, want in (("cfg3_m512", {0}), ("cfg3_m4096", {0}), ("cfg3_m8192", {1}), ("cfg3_m512_8x256", {0}),
+                       ("cfg3_m4096_2x256", {1})):
+        comm, req = make_request(wl.config(name))
+        assert kernels(req) == want, name
+        if want == {0}:
+            assert iso.Iso_request_get_stats(req)["bulk_bytes"] == 0
+            iso.Iso_request_set_slabs(req, 2)            # the caller's slabs: back to the crossover of single launches
+            assert kernels(req) == {1}, name
+            iso.Iso_request_set_slabs(req, 0)
+            assert kernels(req) == {0}, name
+            set_alg(req, iso.ISO_ALG_DIRECT, 1)          # nothing to reuse: bulk copies
+            assert kernels(req) == {1}, name
+            set_alg(req, iso.ISO_ALG_COMBINING, 1)
+            iso.Iso_request_set_bulk_threshold(req, 512)
+            assert kernels(req) == {1}, name
+            iso.Iso_request_set_bulk_threshold(req, 0)
+            assert kernels(req) == {0}, name
+        iso.Iso_request_free(req)
+        iso.Iso_comm_free(comm)
+    w = wl.Workload("ag", "allgather", (16, 16, 16), wl.moore(3, 1), 1024)
+    comm, req = make_request(w)
+    assert kernels(req) == {1}
+    iso.Iso_request_free(req)
+    iso.Iso_comm_free(comm)
+
+
 def test_ragged_phases_lower_to_one_launch_of_mixed_widths(monkeypatch):
     """Irregular sizes: a phase whose pieces need several unit widths is one launch (the unit
     descriptors carry their width); ragged ends are cut into aligned power-of-two pieces of
