@@ -128,6 +128,7 @@ struct Knobs {
     bool col_split = true;    // ISO_COL_SPLIT=0: rows longer than a CTA are covered in passes instead of column chunks
     bool host_graph = true;   // ISO_HOST_GRAPH=0: the pipelined host-buffer path is never replayed from a graph
     bool coord_table = true;  // ISO_COORD_TABLE=0: row coordinates by division in every thread
+    bool l2_keep = true;      // ISO_L2_KEEP=0: no eviction-priority hint on stores into the intermediate buffer
     int ag_order = -1;        // ISO_AG_ORDER=0/1: allgather visits the dimensions first-to-last / last-to-first
 };
 Knobs read_knobs();

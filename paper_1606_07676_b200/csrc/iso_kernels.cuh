@@ -76,6 +76,7 @@ struct LaunchDev {
     uint32_t tab_stride;     // coordinate table: 32-bit words per row (4 or 8)
     uint32_t side_offset;    // hybrid kernel, bulk side: byte offset of its staging area in shared memory
     uint32_t col_split;      // vector kernel: column chunks the CTAs are dealt to (0 or 1: a CTA covers whole rows)
+    uint32_t keep_inter;     // vector kernel, 16-byte units: stores into the intermediate buffer ask the L2 to evict them last
     FastDivDev div_units;    // division by units_per_proc
     FastDivDev div_uniform;  // division by uniform_units
     int used_dim[ISO_MAX_DIMS];
@@ -218,6 +219,23 @@ template <int W> __device__ __forceinline__ void store_unit(unsigned char *dst, 
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// L2 eviction priority for the blocks a slab keeps for its next phase: written with the
+// evict_last policy they outlast the streamed send and receive lines around them, are read
+// back out of the L2 and are overwritten there by the next slab instead of being written
+// back to device memory in between.  A hint only: the data path is the same store.
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ void store_16_hinted(unsigned char *dst, const uint4 &v, uint64_t policy)
+{
+    asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w),
+                 "l"(policy)
+                 : "memory");
+}
+
 // What a thread keeps about the unit position it owns.
 struct UnitRegs {
     const unsigned char *A;  // source base: buffer + src_term
@@ -227,6 +245,7 @@ struct UnitRegs {
     uint32_t nnz;
     uint32_t width;
     uint32_t dims_lo, dims_hi;  // dim[0..3], dim[4..7], one byte each
+    bool to_inter;              // the destination is the intermediate buffer
 };
 
 __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
@@ -244,6 +263,7 @@ __device__ __forceinline__ UnitRegs load_unit(const LaunchDev &L, uint32_t u)
     R.c[0] = (int)b.x; R.c[1] = (int)b.y; R.c[2] = (int)b.z; R.c[3] = (int)b.w;
     R.c[4] = (int)c.x; R.c[5] = (int)c.y; R.c[6] = (int)c.z; R.c[7] = (int)c.w;
     R.nnz = (d.x >> 16) & 0xff;
+    R.to_inter = db == 2;  // ISO_BUF_INTER
     R.width = d.x >> 24;
     if (R.width < 4) R.width |= ((uint32_t)(uintptr_t)R.A & 3u) << 8;  // offset inside the aligned word
     R.dims_lo = d.y;
@@ -349,6 +369,8 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
 #pragma unroll
         for (int e = 0; e < NU; ++e) wrap_bytes[e] = (long long)L.used_wrap[dim_of(e)] * R.stride_s;
         const long long src_step = rstep * R.stride_s, dst_step = rstep * R.stride_d;
+        const bool keep = W == 16 && L.keep_inter && R.to_inter;
+        const uint64_t policy = keep ? l2_policy_evict_last() : 0;
 
         // `row`: the row's entry of the coordinate table (TAB), unused otherwise
         auto source = [&](const unsigned char *nowrap, long long r, const uint32_t *row, const unsigned char *&src) -> bool {
@@ -404,7 +426,11 @@ __device__ __forceinline__ void gather_rows_body(const LaunchDev &L, unsigned ch
                 valid = source(nullptr, r, row_st, ignored);
                 row_st += tab_step;
             }
-            if (valid) store_unit<W>(dst, slot, R.width);
+            if (W == 16 && keep) {
+                if (valid) store_16_hinted(dst, *reinterpret_cast<const uint4 *>(slot), policy);
+            } else if (valid) {
+                store_unit<W>(dst, slot, R.width);
+            }
             dst += dst_step;
             if (r_ld < r_end) {
                 const unsigned char *src;

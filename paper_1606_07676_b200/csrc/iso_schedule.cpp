@@ -65,6 +65,7 @@ Knobs read_knobs()
     k.hybrid = (int)num("ISO_HYBRID", -1);
     k.col_split = num("ISO_COL_SPLIT", 1) != 0;
     k.ag_order = num("ISO_AG_ORDER", -1);
+    k.l2_keep = num("ISO_L2_KEEP", 1) != 0;
     return k;
 }
 
